@@ -1,0 +1,185 @@
+/*
+ * httm.h - C ABI of the B200 (sm_100a) library for one VGGT-style global-attention
+ * layer with head-wise temporal token merging (HTTM).
+ *
+ * The path behind these calls is Algorithm 1 of the HTTM paper without its
+ * projections and without outlier filtering:
+ *   temporal reorder (Sec. 3.3) -> per-head, per-block cosine matching of Q and of K
+ *   (Eq. 1) -> mean merge of Q, K, V (V follows K, Sec. 3.2) -> softmax attention on
+ *   the merged sets (Eq. 3-4) -> head-wise unmerge (Eq. 5-7) + inverse reorder.
+ *
+ * Conventions common to all calls
+ *   - S frames; every frame has n_camera + n_register special tokens followed by a
+ *     grid_h x grid_w patch grid (row-major).  P = specials + grid_h*grid_w tokens per
+ *     frame, N = S*P tokens, token index i = frame*P + index_in_frame.
+ *   - Q, K, V are bf16 DEVICE tensors addressed as ptr[head*stride_head +
+ *     token*stride_token + channel], strides in ELEMENTS, channels contiguous.
+ *     ptr must be 16-byte aligned and both strides multiples of 8 elements.
+ *   - The output is bf16, addressed the same way; the paper's concatenated layout
+ *     [N][heads*head_dim] (Eq. 7) is stride_head = head_dim, stride_token =
+ *     heads*head_dim.  It must not overlap an input.
+ *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream) and return without waiting for it.  The caller
+ *     owns the tensors and keeps them alive until the stream has passed the call.
+ *   - The context owns all scratch memory (sized at httm_create; nothing is allocated
+ *     in the attention calls) and is not thread-safe; separate contexts are independent.
+ *   - Every function returns HTTM_OK (0) or a negative httm_status.  Arguments are
+ *     checked on the host before anything is launched.  Nothing aborts or throws.
+ */
+#ifndef HTTM_H_
+#define HTTM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HTTM_OK = 0,
+    HTTM_ERR_INVALID_ARG = -1, /* null pointer, value out of range, overlapping output */
+    HTTM_ERR_UNSUPPORTED = -2, /* head_dim != 64, block of more than 256 tokens, ...  */
+    HTTM_ERR_ALIGNMENT = -3,   /* pointer not 16-byte aligned / stride not multiple of 8 */
+    HTTM_ERR_NOMEM = -4,       /* device or host allocation failed                     */
+    HTTM_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed (see last_error)  */
+    HTTM_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (status word set)  */
+} httm_status;
+
+typedef struct httm_ctx httm_ctx; /* opaque; created and destroyed by the library */
+
+typedef struct {
+    int32_t frames;               /* S >= 1                                            */
+    int32_t n_camera, n_register; /* special tokens per frame (VGGT: 1 and 4); >= 0    */
+    int32_t grid_h, grid_w;       /* patch grid, >= 1                                  */
+    int32_t heads, head_dim;      /* head_dim must be 64                               */
+    int32_t blk_frames, blk_h, blk_w; /* merging block: frames x patch window, >= 1;
+                                     blocks are clipped at the grid / sequence end     */
+    double ratio_q, ratio_kv;     /* fraction of tokens merged away, in [0, 1)         */
+    int32_t device;               /* CUDA device ordinal                               */
+} httm_config;
+
+typedef struct {
+    void* ptr;            /* device pointer to bf16 data (inputs are only read)        */
+    int64_t stride_head;  /* elements between heads                                    */
+    int64_t stride_token; /* elements between tokens                                   */
+} httm_tensor;
+
+/* httm_query selectors */
+enum {
+    HTTM_Q_TOKENS = 0,          /* N                                                   */
+    HTTM_Q_MERGED_Q = 1,        /* M_q: merged query length (same for every head)      */
+    HTTM_Q_MERGED_K = 2,        /* M_k: merged key/value length                        */
+    HTTM_Q_BLOCKS = 3,          /* merging blocks per head                             */
+    HTTM_Q_WORKSPACE_BYTES = 4, /* device bytes owned by the context                   */
+    HTTM_Q_MAX_BLOCK_TOKENS = 5,
+    HTTM_Q_DEVICE_STATUS = 6    /* syncs the device; 0 or the first device-side error   */
+};
+
+/* httm_export selectors: intermediates of the LAST httm_global_attention call.
+ * Index arrays are int32, tensors bf16 bit patterns (uint16). */
+enum {
+    HTTM_X_PI = 0,         /* [N]       reordered position -> original token index      */
+    HTTM_X_PI_INV = 1,     /* [N]       original token index -> reordered position      */
+    HTTM_X_BLOCK_START = 2,/* [blocks+1] reordered position of each block's first token */
+    HTTM_X_ASSIGN_Q = 3,   /* [H][N]    reordered position each token is merged into     */
+    HTTM_X_ASSIGN_K = 4,
+    HTTM_X_RANK_Q = 5,     /* [H][N]    merged row of each reordered token               */
+    HTTM_X_Q_REORDERED = 6,/* [H][N][D]                                                  */
+    HTTM_X_K_REORDERED = 7,
+    HTTM_X_V_REORDERED = 8,
+    HTTM_X_Q_MERGED = 9,   /* [H][M_q][D]                                                */
+    HTTM_X_K_MERGED = 10,  /* [H][M_k][D]                                                */
+    HTTM_X_V_MERGED = 11,
+    HTTM_X_O_MERGED = 12   /* [H][M_q][D] attention output before unmerge               */
+};
+
+/* httm_launch_stage selectors: the five launches httm_global_attention is made of. */
+enum {
+    HTTM_STAGE_REORDER = 0,
+    HTTM_STAGE_MATCH = 1,
+    HTTM_STAGE_MERGE = 2,
+    HTTM_STAGE_ATTENTION = 3,
+    HTTM_STAGE_UNMERGE = 4
+};
+
+/*
+ * Create a context for one problem geometry (Algorithm 1's inputs: block shape
+ * B_s x B_t and the merge budgets).  Host work only plus device allocation and a few
+ * small uploads: builds the reorder index pi (Sec. 3.3), the block table and the
+ * per-block merge budget r = min(floor(ratio*n + 1e-9), n-1) with
+ * n_dst = min(ceil(n/4), n-r) evenly spaced destination tokens (Sec. 3.2).
+ * On success *out owns the context; free it with httm_destroy.
+ * Errors: INVALID_ARG, UNSUPPORTED, NOMEM, CUDA.  On error *out is NULL.
+ */
+int httm_create(const httm_config* cfg, httm_ctx** out);
+
+/*
+ * HTTM global attention (Algorithm 1 between the QKV and output projections).
+ * q, k, v: device tensors of the context's geometry; out: device output, all N
+ * tokens, every head.  Five kernels are enqueued on `stream`:
+ *   reorder (Sec. 3.3) -> match Q, K (Eq. 1, top-r of Sec. 3.2) -> merge Q, K, V
+ *   (mean of constituents) -> attention on merged sets (Eq. 3-4) -> unmerge +
+ *   inverse reorder + head concat (Eq. 5-7).
+ * With ratio_q = ratio_kv = 0 the result equals httm_dense_attention up to rounding.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA (launch failure); device-side wait time-outs
+ * are reported by the next httm_query(HTTM_Q_DEVICE_STATUS) / httm_export.
+ */
+int httm_global_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out,
+                          void* cuda_stream);
+
+/*
+ * Exact multi-head softmax attention over all N tokens (the unmerged baseline the
+ * paper's speed-ups are measured against, Sec. 4.1), same attention kernel, output
+ * written directly in `out`'s layout.  Same argument rules and errors as above.
+ */
+int httm_dense_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out,
+                         void* cuda_stream);
+
+/*
+ * The same two operations for callers whose tensors live in HOST memory (pinned memory
+ * makes the copies asynchronous).  q, k, v: bf16 [heads][N][head_dim] contiguous;
+ * out: bf16 [N][heads*head_dim] contiguous.  Each call copies the inputs to
+ * context-owned device buffers (allocated at the first such call), runs the path and
+ * copies the result back, all on `stream`; the caller synchronises the stream before
+ * reading `out`.  dense != 0 selects httm_dense_attention.
+ * Errors: INVALID_ARG, NOMEM, CUDA.
+ */
+int httm_attention_host(httm_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                        void* out_host, int dense, void* cuda_stream);
+
+/*
+ * Enqueue one of the five stages of httm_global_attention on its own, reading and
+ * writing the context's intermediates of the previous stages (for per-kernel timing
+ * and profiling; calling stages 0..4 in order equals httm_global_attention).
+ * q, k, v are read by HTTM_STAGE_REORDER only, out is written by HTTM_STAGE_UNMERGE only;
+ * the other stages ignore them.
+ */
+int httm_launch_stage(httm_ctx* ctx, int stage, httm_tensor q, httm_tensor k, httm_tensor v,
+                      httm_tensor out, void* cuda_stream);
+
+/* Sizes and status, see HTTM_Q_*.  Errors: INVALID_ARG, CUDA, TIMEOUT (device status). */
+int httm_query(httm_ctx* ctx, int what, int64_t* value);
+
+/*
+ * Copy an intermediate of the last call (HTTM_X_*) to host memory.  Waits for `stream`
+ * first.  `bytes` must be exactly the size of the item (int32 or bf16 elements).
+ * Errors: INVALID_ARG (wrong size / selector), CUDA, TIMEOUT (device status word set).
+ */
+int httm_export(httm_ctx* ctx, int what, void* host_dst, size_t bytes, void* cuda_stream);
+
+/* Message of the last error on this context (or of the last failed httm_create when ctx
+ * is NULL).  The string is owned by the library and valid until the next call. */
+const char* httm_last_error(const httm_ctx* ctx);
+
+/* Number of kernels launched by the library on this context since it was created. */
+int64_t httm_launch_count(const httm_ctx* ctx);
+
+/* Free the context and everything it owns.  The caller first synchronises every stream
+ * the context was used on.  NULL is accepted. */
+int httm_destroy(httm_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HTTM_H_ */

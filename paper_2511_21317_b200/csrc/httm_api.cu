@@ -1,0 +1,535 @@
+// C ABI of libhttm: context (plan + workspace), argument checks, stage launches, exports.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/httm.h"
+#include "httm_internal.h"
+
+using namespace httm;
+
+namespace {
+thread_local std::string g_create_error;
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+}  // namespace
+
+struct httm_ctx {
+    httm_config cfg{};
+    int32_t n_special = 0, tokens_per_frame = 0, n_tokens = 0, n_blocks = 0, max_block = 0;
+    int32_t m_q = 0, m_k = 0;
+    int sm_count = 148;
+    std::vector<int32_t> pi, pi_inv, blk_start;
+    std::vector<BlockInfo> blocks;
+    // device workspace
+    int32_t *d_pi = nullptr, *d_pi_inv = nullptr, *d_assign_q = nullptr, *d_assign_k = nullptr, *d_rank_q = nullptr;
+    int32_t* d_status = nullptr;
+    BlockInfo* d_blocks = nullptr;
+    __nv_bfloat16 *d_qr = nullptr, *d_kr = nullptr, *d_vr = nullptr;
+    __nv_bfloat16 *d_qm = nullptr, *d_km = nullptr, *d_vm = nullptr, *d_om = nullptr;
+    // staging for the host-buffer entry point (allocated on first use)
+    __nv_bfloat16 *d_hq = nullptr, *d_hk = nullptr, *d_hv = nullptr, *d_hout = nullptr;
+    int64_t workspace_bytes = 0;
+    int64_t launches = 0;
+    std::string error;
+
+    int fail(int code, const char* fmt, ...) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        error = buf;
+        return code;
+    }
+    template <typename T>
+    int alloc(T** p, size_t count) {
+        const size_t bytes = (count ? count : 1) * sizeof(T);
+        cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
+        if (e != cudaSuccess) {
+            *p = nullptr;
+            cudaGetLastError();
+            return fail(e == cudaErrorMemoryAllocation ? HTTM_ERR_NOMEM : HTTM_ERR_CUDA, "cudaMalloc(%zu bytes): %s", bytes,
+                        cudaGetErrorString(e));
+        }
+        workspace_bytes += (int64_t)bytes;
+        return HTTM_OK;
+    }
+    void release() {
+        void* ptrs[] = {d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
+                        d_vr, d_qm,     d_km,       d_vm,       d_om,     d_hq,     d_hk,     d_hv, d_hout};
+        for (void* p : ptrs)
+            if (p) cudaFree(p);
+    }
+};
+
+namespace {
+
+int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Merge budget of a block of n tokens (Sec. 3.2, r = N - M): r src tokens are merged away,
+// n_dst evenly spaced tokens act as destinations.
+void block_budget(int n, double ratio, int32_t* r, int32_t* nd) {
+    int64_t rr = (int64_t)std::floor(ratio * (double)n + 1e-9);
+    if (rr > n - 1) rr = n - 1;
+    if (rr < 0) rr = 0;
+    int64_t d = ceil_div64(n, 4);
+    if (d > n - rr) d = n - rr;
+    *r = (int32_t)rr;
+    *nd = (int32_t)d;
+}
+
+int check_cuda(httm_ctx* c, cudaError_t e, const char* what) {
+    if (e == cudaSuccess) return HTTM_OK;
+    cudaGetLastError();
+    return c->fail(HTTM_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool overlaps(const void* a, int64_t a_bytes, const void* b, int64_t b_bytes) {
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + (uintptr_t)b_bytes && b0 < a0 + (uintptr_t)a_bytes;
+}
+
+int64_t span_bytes(const httm_ctx* c, const httm_tensor& t) {
+    return ((int64_t)(c->cfg.heads - 1) * t.stride_head + (int64_t)(c->n_tokens - 1) * t.stride_token + kHeadDim) * 2;
+}
+
+int check_tensor(httm_ctx* c, const httm_tensor& t, const char* name) {
+    if (!t.ptr) return c->fail(HTTM_ERR_INVALID_ARG, "%s: null pointer", name);
+    if (((uintptr_t)t.ptr & 15u) != 0) return c->fail(HTTM_ERR_ALIGNMENT, "%s: pointer is not 16-byte aligned", name);
+    if (t.stride_head % 8 != 0 || t.stride_token % 8 != 0)
+        return c->fail(HTTM_ERR_ALIGNMENT, "%s: strides must be multiples of 8 elements", name);
+    if (t.stride_token < kHeadDim || t.stride_head < 0)
+        return c->fail(HTTM_ERR_INVALID_ARG, "%s: stride_token must be >= head_dim and stride_head >= 0", name);
+    if (c->cfg.heads > 1 && t.stride_head < kHeadDim)
+        return c->fail(HTTM_ERR_INVALID_ARG, "%s: stride_head must be >= head_dim", name);
+    return HTTM_OK;
+}
+
+int check_io(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out) {
+    int rc;
+    if ((rc = check_tensor(c, q, "q")) || (rc = check_tensor(c, k, "k")) || (rc = check_tensor(c, v, "v")) ||
+        (rc = check_tensor(c, out, "out")))
+        return rc;
+    const httm_tensor* in[3] = {&q, &k, &v};
+    for (const httm_tensor* t : in)
+        if (overlaps(out.ptr, span_bytes(c, out), t->ptr, span_bytes(c, *t)))
+            return c->fail(HTTM_ERR_INVALID_ARG, "out overlaps an input tensor");
+    return HTTM_OK;
+}
+
+TensorView view(const httm_tensor& t) {
+    return TensorView{reinterpret_cast<const __nv_bfloat16*>(t.ptr), t.stride_head, t.stride_token};
+}
+TensorView view(const __nv_bfloat16* p, int64_t rows) { return TensorView{p, rows * kHeadDim, kHeadDim}; }
+
+float scale_log2() { return 1.4426950408889634f / std::sqrt((float)kHeadDim); }
+
+int stage_reorder(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, cudaStream_t s) {
+    ReorderArgs a{};
+    a.src[0] = view(q);
+    a.src[1] = view(k);
+    a.src[2] = view(v);
+    a.dst[0] = c->d_qr;
+    a.dst[1] = c->d_kr;
+    a.dst[2] = c->d_vr;
+    a.pi = c->d_pi;
+    a.n_tokens = c->n_tokens;
+    a.heads = c->cfg.heads;
+    c->launches++;
+    return check_cuda(c, launch_reorder(a, s), "reorder launch");
+}
+
+int stage_match(httm_ctx* c, cudaStream_t s) {
+    MatchArgs a{};
+    a.xr[0] = c->d_qr;
+    a.xr[1] = c->d_kr;
+    a.assign[0] = c->d_assign_q;
+    a.assign[1] = c->d_assign_k;
+    a.blocks = c->d_blocks;
+    a.n_blocks = c->n_blocks;
+    a.n_tokens = c->n_tokens;
+    a.heads = c->cfg.heads;
+    a.status = c->d_status;
+    c->launches++;
+    return check_cuda(c, launch_match(a, c->max_block, c->sm_count, s), "match launch");
+}
+
+int stage_merge(httm_ctx* c, cudaStream_t s) {
+    MergeArgs a{};
+    a.xr[0] = c->d_qr;
+    a.xr[1] = c->d_kr;
+    a.xr[2] = c->d_vr;
+    a.assign[0] = c->d_assign_q;
+    a.assign[1] = c->d_assign_k;
+    a.merged[0] = c->d_qm;
+    a.merged[1] = c->d_km;
+    a.merged[2] = c->d_vm;
+    a.rank_q = c->d_rank_q;
+    a.blocks = c->d_blocks;
+    a.n_blocks = c->n_blocks;
+    a.n_tokens = c->n_tokens;
+    a.heads = c->cfg.heads;
+    a.n_special_total = c->cfg.frames * c->n_special;
+    a.m_q = c->m_q;
+    a.m_k = c->m_k;
+    a.status = c->d_status;
+    c->launches++;
+    return check_cuda(c, launch_merge(a, c->max_block, c->sm_count, s), "merge launch");
+}
+
+int stage_attention(httm_ctx* c, cudaStream_t s) {
+    AttentionArgs a{};
+    a.q = view(c->d_qm, c->m_q);
+    a.k = view(c->d_km, c->m_k);
+    a.v = view(c->d_vm, c->m_k);
+    a.out = c->d_om;
+    a.out_stride_head = (int64_t)c->m_q * kHeadDim;
+    a.out_stride_token = kHeadDim;
+    a.m_q = c->m_q;
+    a.m_k = c->m_k;
+    a.heads = c->cfg.heads;
+    a.scale_log2 = scale_log2();
+    a.status = c->d_status;
+    c->launches++;
+    return check_cuda(c, launch_attention(a, c->sm_count, s), "attention launch");
+}
+
+int stage_unmerge(httm_ctx* c, const httm_tensor& out, cudaStream_t s) {
+    UnmergeArgs a{};
+    a.o_m = c->d_om;
+    a.rank_q = c->d_rank_q;
+    a.pi_inv = c->d_pi_inv;
+    a.out = reinterpret_cast<__nv_bfloat16*>(out.ptr);
+    a.out_stride_head = out.stride_head;
+    a.out_stride_token = out.stride_token;
+    a.n_tokens = c->n_tokens;
+    a.heads = c->cfg.heads;
+    a.m_q = c->m_q;
+    a.status = c->d_status;
+    c->launches++;
+    return check_cuda(c, launch_unmerge(a, s), "unmerge launch");
+}
+
+int dense_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out,
+               cudaStream_t s) {
+    AttentionArgs a{};
+    a.q = view(q);
+    a.k = view(k);
+    a.v = view(v);
+    a.out = reinterpret_cast<__nv_bfloat16*>(out.ptr);
+    a.out_stride_head = out.stride_head;
+    a.out_stride_token = out.stride_token;
+    a.m_q = c->n_tokens;
+    a.m_k = c->n_tokens;
+    a.heads = c->cfg.heads;
+    a.scale_log2 = scale_log2();
+    a.status = c->d_status;
+    c->launches++;
+    return check_cuda(c, launch_attention(a, c->sm_count, s), "dense attention launch");
+}
+
+int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out,
+                cudaStream_t s) {
+    int rc;
+    if ((rc = stage_reorder(c, q, k, v, s))) return rc;
+    if ((rc = stage_match(c, s))) return rc;
+    if ((rc = stage_merge(c, s))) return rc;
+    if ((rc = stage_attention(c, s))) return rc;
+    return stage_unmerge(c, out, s);
+}
+
+int device_status(httm_ctx* c, int32_t* value) {
+    cudaError_t e = cudaMemcpy(value, c->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost);   // syncs
+    return check_cuda(c, e, "read device status");
+}
+
+}  // namespace
+
+extern "C" {
+
+int httm_create(const httm_config* cfg, httm_ctx** out) {
+    if (out) *out = nullptr;
+    if (!cfg || !out) {
+        g_create_error = "httm_create: null argument";
+        return HTTM_ERR_INVALID_ARG;
+    }
+    auto bad = [&](int code, const char* msg) {
+        g_create_error = std::string("httm_create: ") + msg;
+        return code;
+    };
+    if (cfg->frames < 1 || cfg->n_camera < 0 || cfg->n_register < 0 || cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->heads < 1 ||
+        cfg->blk_frames < 1 || cfg->blk_h < 1 || cfg->blk_w < 1)
+        return bad(HTTM_ERR_INVALID_ARG, "sizes must be positive (special-token counts non-negative)");
+    if (!(cfg->ratio_q >= 0.0 && cfg->ratio_q < 1.0) || !(cfg->ratio_kv >= 0.0 && cfg->ratio_kv < 1.0))
+        return bad(HTTM_ERR_INVALID_ARG, "merge ratios must lie in [0, 1)");
+    if (cfg->head_dim != kHeadDim) return bad(HTTM_ERR_UNSUPPORTED, "head_dim must be 64");
+    if (cfg->heads > 65535) return bad(HTTM_ERR_UNSUPPORTED, "at most 65535 heads");
+    const int64_t per_frame = (int64_t)cfg->n_camera + cfg->n_register + (int64_t)cfg->grid_h * cfg->grid_w;
+    const int64_t n_tokens = per_frame * cfg->frames;
+    if (n_tokens > (1ll << 24) || n_tokens * cfg->heads > (1ll << 31) - 1)
+        return bad(HTTM_ERR_UNSUPPORTED, "too many tokens (N <= 2^24 and N*heads < 2^31)");
+    const int64_t bf = std::min<int64_t>(cfg->blk_frames, cfg->frames), bh = std::min<int64_t>(cfg->blk_h, cfg->grid_h),
+                  bw = std::min<int64_t>(cfg->blk_w, cfg->grid_w);
+    if (bf * bh * bw > kMaxBlockTokens) return bad(HTTM_ERR_UNSUPPORTED, "a merging block may hold at most 256 tokens");
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) {
+        cudaGetLastError();
+        return bad(HTTM_ERR_INVALID_ARG, "device ordinal out of range (or no CUDA device)");
+    }
+
+    httm_ctx* c = new (std::nothrow) httm_ctx();
+    if (!c) return bad(HTTM_ERR_NOMEM, "host allocation failed");
+    c->cfg = *cfg;
+    c->n_special = cfg->n_camera + cfg->n_register;
+    c->tokens_per_frame = (int32_t)per_frame;
+    c->n_tokens = (int32_t)n_tokens;
+
+    // --- reorder index pi (Sec. 3.3): specials first (frame-major), then the blocks
+    //     (frame group, window row, window column), inside a block frame / y / x.
+    const int S = cfg->frames, h = cfg->grid_h, w = cfg->grid_w, nsp = c->n_special, P = c->tokens_per_frame;
+    c->pi.resize(n_tokens);
+    c->pi_inv.resize(n_tokens);
+    int32_t pos = 0;
+    for (int s = 0; s < S; ++s)
+        for (int j = 0; j < nsp; ++j) c->pi[pos++] = s * P + j;
+    int32_t moff_q = pos, moff_k = pos;
+    for (int g0 = 0; g0 < S; g0 += cfg->blk_frames) {
+        const int f = std::min(cfg->blk_frames, S - g0);
+        for (int y0 = 0; y0 < h; y0 += cfg->blk_h) {
+            const int hh = std::min(cfg->blk_h, h - y0);
+            for (int x0 = 0; x0 < w; x0 += cfg->blk_w) {
+                const int ww = std::min(cfg->blk_w, w - x0);
+                BlockInfo bi{};
+                bi.start = pos;
+                bi.n = f * hh * ww;
+                block_budget(bi.n, cfg->ratio_q, &bi.r_q, &bi.nd_q);
+                block_budget(bi.n, cfg->ratio_kv, &bi.r_k, &bi.nd_k);
+                bi.moff_q = moff_q;
+                bi.moff_k = moff_k;
+                moff_q += bi.n - bi.r_q;
+                moff_k += bi.n - bi.r_k;
+                c->max_block = std::max(c->max_block, bi.n);
+                c->blk_start.push_back(pos);
+                c->blocks.push_back(bi);
+                for (int tl = 0; tl < f; ++tl)
+                    for (int yl = 0; yl < hh; ++yl)
+                        for (int xl = 0; xl < ww; ++xl) c->pi[pos++] = (g0 + tl) * P + nsp + (y0 + yl) * w + (x0 + xl);
+            }
+        }
+    }
+    c->blk_start.push_back(pos);
+    c->n_blocks = (int32_t)c->blocks.size();
+    c->m_q = moff_q;
+    c->m_k = moff_k;
+    for (int32_t p = 0; p < c->n_tokens; ++p) c->pi_inv[c->pi[p]] = p;
+
+    DeviceGuard guard(cfg->device);
+    int rc = HTTM_OK;
+    auto done = [&](int code) -> int {
+        if (code != HTTM_OK) {
+            g_create_error = "httm_create: " + c->error;
+            c->release();
+            delete c;
+            return code;
+        }
+        *out = c;
+        return HTTM_OK;
+    };
+    if (!guard.ok) return done(c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed"));
+    cudaDeviceProp prop{};
+    if ((rc = check_cuda(c, cudaGetDeviceProperties(&prop, cfg->device), "cudaGetDeviceProperties"))) return done(rc);
+    if (prop.major != 10) return done(c->fail(HTTM_ERR_UNSUPPORTED, "device is sm_%d%d; this library is built for sm_100a only",
+                                               prop.major, prop.minor));
+    c->sm_count = prop.multiProcessorCount;
+    if ((rc = check_cuda(c, configure_kernels(), "cudaFuncSetAttribute"))) return done(rc);
+
+    const size_t H = cfg->heads, N = c->n_tokens;
+    if ((rc = c->alloc(&c->d_pi, N)) || (rc = c->alloc(&c->d_pi_inv, N)) || (rc = c->alloc(&c->d_blocks, c->blocks.size())) ||
+        (rc = c->alloc(&c->d_status, 4)) || (rc = c->alloc(&c->d_assign_q, H * N)) || (rc = c->alloc(&c->d_assign_k, H * N)) ||
+        (rc = c->alloc(&c->d_rank_q, H * N)) || (rc = c->alloc(&c->d_qr, H * N * kHeadDim)) ||
+        (rc = c->alloc(&c->d_kr, H * N * kHeadDim)) || (rc = c->alloc(&c->d_vr, H * N * kHeadDim)) ||
+        (rc = c->alloc(&c->d_qm, H * c->m_q * kHeadDim)) || (rc = c->alloc(&c->d_km, H * c->m_k * kHeadDim)) ||
+        (rc = c->alloc(&c->d_vm, H * c->m_k * kHeadDim)) || (rc = c->alloc(&c->d_om, H * c->m_q * kHeadDim)))
+        return done(rc);
+
+    // uploads; special tokens are never merged: their map entries are constants, written once
+    std::vector<int32_t> ident(H * N);
+    for (size_t hd = 0; hd < H; ++hd)
+        for (size_t p = 0; p < N; ++p) ident[hd * N + p] = (int32_t)p;
+    cudaError_t e = cudaSuccess;
+    auto up = [&](void* dst, const void* src, size_t bytes) {
+        if (e == cudaSuccess && bytes) e = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice);
+    };
+    up(c->d_pi, c->pi.data(), N * 4);
+    up(c->d_pi_inv, c->pi_inv.data(), N * 4);
+    up(c->d_blocks, c->blocks.data(), c->blocks.size() * sizeof(BlockInfo));
+    up(c->d_assign_q, ident.data(), H * N * 4);
+    up(c->d_assign_k, ident.data(), H * N * 4);
+    up(c->d_rank_q, ident.data(), H * N * 4);
+    if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 16);
+    if ((rc = check_cuda(c, e, "workspace upload"))) return done(rc);
+    return done(HTTM_OK);
+}
+
+int httm_global_attention(httm_ctx* c, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out, void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    int rc = check_io(c, q, k, v, out);
+    if (rc) return rc;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    return global_impl(c, q, k, v, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int httm_dense_attention(httm_ctx* c, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out, void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    int rc = check_io(c, q, k, v, out);
+    if (rc) return rc;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    return dense_impl(c, q, k, v, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int httm_attention_host(httm_ctx* c, const void* q_host, const void* k_host, const void* v_host, void* out_host, int dense,
+                        void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (!q_host || !k_host || !v_host || !out_host) return c->fail(HTTM_ERR_INVALID_ARG, "null host pointer");
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    const size_t elems = (size_t)c->cfg.heads * c->n_tokens * kHeadDim;
+    int rc;
+    if (!c->d_hq) {
+        if ((rc = c->alloc(&c->d_hq, elems)) || (rc = c->alloc(&c->d_hk, elems)) || (rc = c->alloc(&c->d_hv, elems)) ||
+            (rc = c->alloc(&c->d_hout, elems)))
+            return rc;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemcpyAsync(c->d_hq, q_host, elems * 2, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_hk, k_host, elems * 2, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_hv, v_host, elems * 2, cudaMemcpyHostToDevice, s);
+    if ((rc = check_cuda(c, e, "host to device copy"))) return rc;
+    const int64_t N = c->n_tokens, H = c->cfg.heads;
+    httm_tensor q{c->d_hq, N * kHeadDim, kHeadDim}, k{c->d_hk, N * kHeadDim, kHeadDim}, v{c->d_hv, N * kHeadDim, kHeadDim};
+    httm_tensor o{c->d_hout, kHeadDim, H * kHeadDim};
+    rc = dense ? dense_impl(c, q, k, v, o, s) : global_impl(c, q, k, v, o, s);
+    if (rc) return rc;
+    return check_cuda(c, cudaMemcpyAsync(out_host, c->d_hout, elems * 2, cudaMemcpyDeviceToHost, s), "device to host copy");
+}
+
+int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out, void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    int rc;
+    switch (stage) {
+        case HTTM_STAGE_REORDER:
+            if ((rc = check_tensor(c, q, "q")) || (rc = check_tensor(c, k, "k")) || (rc = check_tensor(c, v, "v"))) return rc;
+            return stage_reorder(c, q, k, v, s);
+        case HTTM_STAGE_MATCH:
+            return stage_match(c, s);
+        case HTTM_STAGE_MERGE:
+            return stage_merge(c, s);
+        case HTTM_STAGE_ATTENTION:
+            return stage_attention(c, s);
+        case HTTM_STAGE_UNMERGE:
+            if ((rc = check_tensor(c, out, "out"))) return rc;
+            return stage_unmerge(c, out, s);
+        default:
+            return c->fail(HTTM_ERR_INVALID_ARG, "unknown stage %d", stage);
+    }
+}
+
+int httm_query(httm_ctx* c, int what, int64_t* value) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (!value) return c->fail(HTTM_ERR_INVALID_ARG, "null value pointer");
+    switch (what) {
+        case HTTM_Q_TOKENS: *value = c->n_tokens; return HTTM_OK;
+        case HTTM_Q_MERGED_Q: *value = c->m_q; return HTTM_OK;
+        case HTTM_Q_MERGED_K: *value = c->m_k; return HTTM_OK;
+        case HTTM_Q_BLOCKS: *value = c->n_blocks; return HTTM_OK;
+        case HTTM_Q_WORKSPACE_BYTES: *value = c->workspace_bytes; return HTTM_OK;
+        case HTTM_Q_MAX_BLOCK_TOKENS: *value = c->max_block; return HTTM_OK;
+        case HTTM_Q_DEVICE_STATUS: {
+            DeviceGuard guard(c->cfg.device);
+            int32_t st = 0;
+            int rc = device_status(c, &st);
+            if (rc) return rc;
+            *value = st;
+            if (st != kDevOk)
+                return c->fail(st == kDevBadIndex ? HTTM_ERR_CUDA : HTTM_ERR_TIMEOUT, "device status word = %d", st);
+            return HTTM_OK;
+        }
+        default: return c->fail(HTTM_ERR_INVALID_ARG, "unknown query %d", what);
+    }
+}
+
+int httm_export(httm_ctx* c, int what, void* host_dst, size_t bytes, void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (!host_dst) return c->fail(HTTM_ERR_INVALID_ARG, "null destination");
+    const size_t H = c->cfg.heads, N = c->n_tokens;
+    const void* src = nullptr;
+    size_t need = 0;
+    bool host_src = false;
+    switch (what) {
+        case HTTM_X_PI: src = c->pi.data(); need = N * 4; host_src = true; break;
+        case HTTM_X_PI_INV: src = c->pi_inv.data(); need = N * 4; host_src = true; break;
+        case HTTM_X_BLOCK_START: src = c->blk_start.data(); need = c->blk_start.size() * 4; host_src = true; break;
+        case HTTM_X_ASSIGN_Q: src = c->d_assign_q; need = H * N * 4; break;
+        case HTTM_X_ASSIGN_K: src = c->d_assign_k; need = H * N * 4; break;
+        case HTTM_X_RANK_Q: src = c->d_rank_q; need = H * N * 4; break;
+        case HTTM_X_Q_REORDERED: src = c->d_qr; need = H * N * kRowBytes; break;
+        case HTTM_X_K_REORDERED: src = c->d_kr; need = H * N * kRowBytes; break;
+        case HTTM_X_V_REORDERED: src = c->d_vr; need = H * N * kRowBytes; break;
+        case HTTM_X_Q_MERGED: src = c->d_qm; need = H * (size_t)c->m_q * kRowBytes; break;
+        case HTTM_X_K_MERGED: src = c->d_km; need = H * (size_t)c->m_k * kRowBytes; break;
+        case HTTM_X_V_MERGED: src = c->d_vm; need = H * (size_t)c->m_k * kRowBytes; break;
+        case HTTM_X_O_MERGED: src = c->d_om; need = H * (size_t)c->m_q * kRowBytes; break;
+        default: return c->fail(HTTM_ERR_INVALID_ARG, "unknown export %d", what);
+    }
+    if (bytes != need) return c->fail(HTTM_ERR_INVALID_ARG, "export %d needs %zu bytes, got %zu", what, need, bytes);
+    if (host_src) {
+        memcpy(host_dst, src, need);
+        return HTTM_OK;
+    }
+    DeviceGuard guard(c->cfg.device);
+    int rc;
+    if ((rc = check_cuda(c, cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)), "stream synchronize"))) return rc;
+    if ((rc = check_cuda(c, cudaMemcpy(host_dst, src, need, cudaMemcpyDeviceToHost), "export copy"))) return rc;
+    int32_t st = 0;
+    if ((rc = device_status(c, &st))) return rc;
+    if (st != kDevOk) return c->fail(st == kDevBadIndex ? HTTM_ERR_CUDA : HTTM_ERR_TIMEOUT, "device status word = %d", st);
+    return HTTM_OK;
+}
+
+const char* httm_last_error(const httm_ctx* c) { return c ? c->error.c_str() : g_create_error.c_str(); }
+
+int64_t httm_launch_count(const httm_ctx* c) { return c ? c->launches : 0; }
+
+int httm_destroy(httm_ctx* c) {
+    if (!c) return HTTM_OK;
+    {
+        DeviceGuard guard(c->cfg.device);
+        c->release();
+    }
+    delete c;
+    return HTTM_OK;
+}
+
+}  // extern "C"

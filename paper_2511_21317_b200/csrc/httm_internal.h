@@ -1,0 +1,89 @@
+// Internal declarations shared by the translation units of libhttm (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace httm {
+
+constexpr int kHeadDim = 64;          // channels per head the kernels are written for
+constexpr int kRowBytes = kHeadDim * 2;  // one token of one head, bf16
+constexpr int kMaxBlockTokens = 256;  // largest merging block the match / merge kernels stage
+
+// Device status word values (first error wins).
+enum : int {
+    kDevOk = 0,
+    kDevTimeoutMatchLoad = 1,   // match kernel: bulk copy of a block did not complete in time
+    kDevTimeoutAttention = 2,   // attention kernel: a pipeline barrier did not complete in time
+    kDevBadIndex = 3            // an index read from a map was out of range (skipped)
+};
+
+// One merging block (Sec. 3.3): tokens [start, start + n) of the reordered sequence.
+// r_* = number of src tokens merged away, nd_* = number of dst tokens,
+// moff_* = merged row of the block's first kept token (closed form: the per-block kept
+// count n - r is the same for every head).
+struct BlockInfo {
+    int32_t start, n;
+    int32_t r_q, nd_q, moff_q;
+    int32_t r_k, nd_k, moff_k;
+};
+
+struct TensorView {          // bf16, element strides
+    const __nv_bfloat16* ptr;
+    int64_t stride_head, stride_token;
+};
+
+struct ReorderArgs {
+    TensorView src[3];
+    __nv_bfloat16* dst[3];   // [H][N][64] contiguous
+    const int32_t* pi;       // [N]
+    int32_t n_tokens, heads;
+};
+
+struct MatchArgs {
+    const __nv_bfloat16* xr[2];   // reordered Q, K  [H][N][64]
+    int32_t* assign[2];           // A_q, A_k        [H][N]
+    const BlockInfo* blocks;
+    int32_t n_blocks, n_tokens, heads;
+    int32_t* status;
+};
+
+struct MergeArgs {
+    const __nv_bfloat16* xr[3];   // reordered Q, K, V
+    const int32_t* assign[2];     // A_q, A_k (V uses A_k)
+    __nv_bfloat16* merged[3];     // Q_m [H][M_q][64], K_m, V_m [H][M_k][64]
+    int32_t* rank_q;              // [H][N] merged row of every reordered token (written for Q)
+    const BlockInfo* blocks;
+    int32_t n_blocks, n_tokens, heads, n_special_total, m_q, m_k;
+    int32_t* status;
+};
+
+struct UnmergeArgs {
+    const __nv_bfloat16* o_m;     // [H][M_q][64]
+    const int32_t* rank_q;        // [H][N]
+    const int32_t* pi_inv;        // [N]
+    __nv_bfloat16* out;
+    int64_t out_stride_head, out_stride_token;
+    int32_t n_tokens, heads, m_q;
+    int32_t* status;
+};
+
+struct AttentionArgs {
+    TensorView q, k, v;
+    __nv_bfloat16* out;
+    int64_t out_stride_head, out_stride_token;
+    int32_t m_q, m_k, heads;
+    float scale_log2;             // log2(e) / sqrt(head_dim)
+    int32_t* status;
+};
+
+// Launchers (each enqueues exactly one kernel on `stream`; returns the CUDA error).
+cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream);
+cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
+cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
+cudaError_t launch_unmerge(const UnmergeArgs& a, cudaStream_t stream);
+cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);
+cudaError_t configure_kernels();   // one-time function attributes (dynamic shared memory sizes)
+
+}  // namespace httm

@@ -1,0 +1,135 @@
+"""Comparison of the CUDA path with the CPU oracle (used by the GPU tests, the smoke
+check and the benchmark's parity sample).  The rules:
+
+  * reorder permutation, reordered tensors: bit-exact;
+  * assignment maps: bit-exact, except inside blocks where the oracle's (double)
+    similarity margin to the runner-up - best vs second-best destination of a source,
+    or the r-th vs (r+1)-th best score - is below 1e-5; there the map under test must
+    still be a valid outcome within that margin;
+  * merged tensors: the bf16 value must be one of the two bf16 neighbours of the exact mean;
+  * attention output: max abs error <= 2e-2 x RMS of the oracle's output.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import httm_oracle as orc
+
+MARGIN = 1e-5
+OUT_TOL = 2e-2
+
+
+def bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def check_maps(g, rho, blk_start, xr_bits, a_oracle, margin_best, margin_sel, a_gpu, what=""):
+    """Returns the number of (head, block) pairs where the maps differ (all justified by the
+    margin rule); raises AssertionError otherwise."""
+    a_gpu = np.asarray(a_gpu, dtype=np.int64)
+    assert a_gpu.shape == a_oracle.shape, f"{what}: map shape {a_gpu.shape} != {a_oracle.shape}"
+    diff = a_gpu != a_oracle
+    if not diff.any():
+        return 0
+    nsp_total = int(blk_start[0])
+    assert not diff[:, :nsp_total].any(), f"{what}: special tokens must map to themselves"
+    n_bad_blocks = 0
+    for hd in np.flatnonzero(diff.any(axis=1)):
+        cols = np.flatnonzero(diff[hd])
+        blocks = np.unique(np.searchsorted(blk_start, cols, side="right") - 1)
+        for b in blocks:
+            lo, hi = int(blk_start[b]), int(blk_start[b + 1])
+            n = hi - lo
+            r, nd = orc.block_budget(n, rho)
+            ambiguous = margin_sel[hd, b] < MARGIN or (margin_best[hd, lo:hi] < MARGIN).any()
+            assert ambiguous, (f"{what}: head {hd} block {b}: map differs from the oracle but all margins are >= {MARGIN} "
+                               f"(min best-margin {margin_best[hd, lo:hi].min():.3e}, selection margin {margin_sel[hd, b]:.3e})")
+            # validity within the margin, from double-precision similarities
+            x = bits_to_f64(xr_bits[hd, lo:hi])
+            nrm = np.maximum(np.linalg.norm(x, axis=1, keepdims=True), 1e-12)
+            xn = x / nrm
+            dst = np.array([j for j in range(n) if ((j + 1) * nd) // n > (j * nd) // n])
+            src = np.array([j for j in range(n) if j not in set(dst.tolist())])
+            sim = xn[src] @ xn[dst].T
+            best = sim.max(axis=1)
+            loc = a_gpu[hd, lo:hi] - lo
+            assert ((loc >= 0) & (loc < n)).all(), f"{what}: head {hd} block {b}: target outside the block"
+            assert (loc[dst] == dst).all(), f"{what}: a dst token was merged away"
+            merged = loc[src] != src
+            assert merged.sum() == r, f"{what}: head {hd} block {b}: {merged.sum()} merged, budget {r}"
+            for ai in np.flatnonzero(merged):
+                tgt = loc[src[ai]]
+                assert tgt in dst, f"{what}: merge target is not a dst token"
+                assert sim[ai, np.flatnonzero(dst == tgt)[0]] >= best[ai] - MARGIN, f"{what}: target is not the best match"
+            if 0 < r < len(src):
+                assert best[merged].min() >= best[~merged].max() - MARGIN, f"{what}: selection is not top-r"
+            n_bad_blocks += 1
+    return n_bad_blocks
+
+
+def check_merged(gpu_bits: np.ndarray, exact: np.ndarray, what=""):
+    """The bf16 result must be the rounding of the exact (double) mean up to the fp32 summation
+    error of the kernel: |err| <= half a bf16 step (2^-8 |exact|) + 4e-6 x the largest magnitude."""
+    got = bits_to_f64(gpu_bits)
+    assert got.shape == exact.shape, f"{what}: shape {got.shape} != {exact.shape}"
+    err = np.abs(got - exact)
+    bound = np.abs(exact) * 2.0 ** -8 + 4e-6 * max(float(np.abs(exact).max()), 1e-30)
+    bad = err > bound
+    assert not bad.any(), f"{what}: {bad.sum()} merged values off by more than one bf16 step (max err {err.max():.3e})"
+    # and nearly all of them are the correctly rounded value
+    return float((err <= np.abs(exact) * 2.0 ** -8).mean())
+
+
+def check_output(gpu_bits: np.ndarray, expect: np.ndarray, rms: float | None = None, what="", peaky: bool = False):
+    """max |gpu - oracle| <= 2e-2 x RMS(oracle).  peaky=True (tiny adversarial geometries only, where a
+    few keys dominate a row and |value| is many times the RMS) adds the representation error of the
+    bf16 output itself, half a bf16 step = 2^-8 |oracle value|, element by element."""
+    got = bits_to_f64(gpu_bits)
+    assert got.shape == expect.shape, f"{what}: shape {got.shape} != {expect.shape}"
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    if rms is None:
+        rms = float(np.sqrt(np.mean(expect ** 2)))
+    err = np.abs(got - expect)
+    bound = OUT_TOL * rms + (2.0 ** -8 * np.abs(expect) if peaky else 0.0)
+    worst = float((err - bound).max())
+    assert worst <= 0, f"{what}: max abs err {err.max():.4e} exceeds {OUT_TOL} x RMS {rms:.4e} by {worst:.3e}"
+    return float(err.max()) / rms
+
+
+def full_check(g, rho_q, rho_kv, q, k, v, ex, out_bits, sample_tokens=None, what="", peaky=False):
+    """Element-by-element comparison of everything the library exposes.
+    ex: dict of exports (numpy) with keys pi, blk_start, qr, kr, vr, assign_q, assign_k, rank_q, q_m, k_m, v_m, o_m.
+    If sample_tokens is given, attention output is checked on those ORIGINAL tokens only."""
+    res = orc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
+    assert np.array_equal(ex["pi"].astype(np.int64), res.pi), f"{what}: reorder permutation differs"
+    assert np.array_equal(ex["blk_start"].astype(np.int64), res.blk_start), f"{what}: block table differs"
+    qr, kr, vr = orc.reorder(g, res.pi, q), orc.reorder(g, res.pi, k), orc.reorder(g, res.pi, v)
+    for name, ref in (("qr", qr), ("kr", kr), ("vr", vr)):
+        assert np.array_equal(ex[name], ref), f"{what}: reordered {name} is not bit-exact"
+    nq = check_maps(g, rho_q, res.blk_start, qr, res.assign_q, res.margin_best_q, res.margin_sel_q, ex["assign_q"], what + " A_q")
+    nk = check_maps(g, rho_kv, res.blk_start, kr, res.assign_k, res.margin_best_k, res.margin_sel_k, ex["assign_k"], what + " A_k")
+    if nq or nk:   # maps differ inside the margin: the oracle continues from the validated maps
+        res = orc.merged_attention_from_maps(g, res.pi, q, k, v, ex["assign_q"].astype(np.int64),
+                                             ex["assign_k"].astype(np.int64), attend=False)
+    assert np.array_equal(ex["rank_q"].astype(np.int64), res.rank_q), f"{what}: rank_q differs"
+    fr = [check_merged(ex[n], ref, f"{what} {n}") for n, ref in (("q_m", res.q_m), ("k_m", res.k_m), ("v_m", res.v_m))]
+    stats = {"ambiguous_blocks_q": nq, "ambiguous_blocks_k": nk, "merged_exactly_rounded": min(fr)}
+    if sample_tokens is None:
+        o_m = orc.attention(res.q_m, res.k_m, res.v_m)
+        out = orc.unmerge(g, res.pi, res.rank_q, o_m)
+        rms = float(np.sqrt(np.mean(out ** 2)))
+        stats["o_m_err"] = check_output(ex["o_m"], o_m, rms, what + " O_m", peaky)
+        stats["out_err"] = check_output(out_bits, out, rms, what + " out", peaky)
+    else:
+        rows = orc.attention_rows_for_tokens(g, res, sample_tokens)
+        rms = float(np.sqrt(np.mean(rows ** 2)))
+        stats["out_err"] = check_output(out_bits[sample_tokens], rows, rms, what + " out (sampled)", peaky)
+        # unmerge is a pure copy of O_m rows: check that on ALL tokens, bit-exactly
+        D = g.head_dim
+        inv = np.empty_like(res.pi)
+        inv[res.pi] = np.arange(len(res.pi))
+        for hd in range(g.heads):
+            assert np.array_equal(out_bits[:, hd * D:(hd + 1) * D], ex["o_m"][hd][res.rank_q[hd][inv]]), \
+                f"{what}: unmerge of head {hd} is not a pure copy"
+    stats["rms"] = rms
+    return stats

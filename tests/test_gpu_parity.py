@@ -1,0 +1,212 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+All tests here need a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import httm_oracle as orc
+from paper_2511_21317_b200 import binding as hb
+from paper_2511_21317_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def exports(ctx):
+    names = {"pi": hb.X_PI, "blk_start": hb.X_BLOCK_START, "qr": hb.X_Q_REORDERED, "kr": hb.X_K_REORDERED,
+             "vr": hb.X_V_REORDERED, "assign_q": hb.X_ASSIGN_Q, "assign_k": hb.X_ASSIGN_K, "rank_q": hb.X_RANK_Q,
+             "q_m": hb.X_Q_MERGED, "k_m": hb.X_K_MERGED, "v_m": hb.X_V_MERGED, "o_m": hb.X_O_MERGED}
+    return {k: ctx.export(v) for k, v in names.items()}
+
+
+def run_case(wl, q=None, k=None, v=None, sample=None, peaky=False):
+    if q is None:
+        q, k, v = synth.make_qkv(wl)
+    g = orc.Geometry.of(wl)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        assert ctx.n_tokens == wl.n_tokens
+        assert ctx.m_q == orc.merged_len(g, wl.ratio_q) and ctx.m_k == orc.merged_len(g, wl.ratio_kv)
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        out = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        ex = exports(ctx)
+        out_bits = hb.bits_from_bf16(out)
+        stats = parity.full_check(g, wl.ratio_q, wl.ratio_kv, q, k, v, ex, out_bits, sample, wl.name, peaky)
+        # determinism: a second call gives bit-identical results (catches races)
+        out2 = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert torch.equal(out, out2)
+        ex2 = exports(ctx)
+        for name in ex:
+            assert np.array_equal(ex[name], ex2[name]), f"{name} differs between two identical calls"
+    return stats
+
+
+def test_tiny_config_full_parity():
+    stats = run_case(synth.WORKLOADS["tiny"])
+    assert stats["out_err"] <= parity.OUT_TOL
+
+
+GEOMS = [
+    # name, frames, grid_h, grid_w, blk, ratio_q, ratio_kv, n_camera, n_register, heads
+    ("clipped_all_dims", 3, 5, 6, (2, 2, 4), 0.5, 0.7, 1, 1, 2),
+    ("window_1x1", 3, 3, 3, (2, 1, 1), 0.5, 0.5, 1, 4, 2),
+    ("single_token_blocks", 2, 2, 2, (1, 1, 1), 0.9, 0.9, 1, 0, 1),
+    ("no_specials", 4, 8, 8, (2, 4, 4), 0.5, 0.75, 0, 0, 3),
+    ("frames_not_divisible", 5, 9, 9, (4, 4, 4), 0.7, 0.8, 1, 4, 2),
+    ("ratio_zero_q", 4, 8, 8, (2, 4, 4), 0.0, 0.6, 1, 4, 2),
+    ("ratio_zero_kv", 4, 8, 8, (2, 4, 4), 0.6, 0.0, 1, 4, 2),
+    ("ratio_099", 4, 9, 9, (2, 4, 4), 0.99, 0.99, 1, 4, 2),
+    ("block_128", 4, 17, 19, (2, 8, 8), 0.7, 0.9, 1, 4, 2),
+    ("block_64", 9, 10, 10, (4, 4, 4), 0.5, 0.9, 1, 4, 2),
+    ("block_256_max", 5, 9, 8, (4, 8, 8), 0.8, 0.3, 1, 4, 1),
+    ("one_frame", 1, 12, 12, (2, 4, 4), 0.5, 0.5, 1, 4, 2),
+]
+
+
+@pytest.mark.parametrize("case", GEOMS, ids=[c[0] for c in GEOMS])
+def test_adversarial_geometries(case):
+    name, S, h, w, blk, rq, rkv, ncam, nreg, H = case
+    wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, n_camera=ncam, n_register=nreg, heads=H, seed=3)
+    run_case(wl, peaky=True)
+
+
+def test_random_uncorrelated_inputs():
+    wl = synth.Workload("gauss", 4, 11, 13, 2, 4, 4, 0.6, 0.6, heads=4)
+    rng = np.random.default_rng(5)
+    q, k, v = (synth.f32_to_bf16_bits(rng.standard_normal((wl.heads, wl.n_tokens, 64)).astype(np.float32)) for _ in range(3))
+    run_case(wl, q, k, v, peaky=True)
+
+
+def test_ties_and_zero_vectors():
+    wl = synth.Workload("ties", 2, 8, 8, 2, 4, 4, 0.5, 0.5, heads=2, n_camera=1, n_register=1)
+    x = synth.make_identical_block_tokens(wl, seed=4)       # every similarity inside a block is a tie
+    q, k, v = synth.make_qkv(wl)
+    z = q.copy()
+    z[:, 10:40, :] = 0                                         # zero vectors: norm clamp
+    run_case(wl, x, k, v, peaky=True)
+    run_case(wl, q, x, v, peaky=True)
+    run_case(wl, z, z, v, peaky=True)
+
+
+def test_ratio_zero_equals_dense_and_textbook():
+    wl = synth.Workload("r0", 3, 7, 9, 2, 4, 4, 0.0, 0.0, heads=3)
+    q, k, v = synth.make_qkv(wl)
+    g = orc.Geometry.of(wl)
+    ref = orc.dense_attention(g, q, k, v)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        assert ctx.m_q == wl.n_tokens == ctx.m_k
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        o_h = ctx.global_attention(dq, dk, dv)
+        o_d = ctx.dense_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        parity.check_output(hb.bits_from_bf16(o_d), ref, what="dense")
+        parity.check_output(hb.bits_from_bf16(o_h), ref, what="httm ratio 0")
+        # same kernel, same rows, same key order up to the permutation -> very close
+        d = (o_h.float() - o_d.float()).abs().max().item()
+        assert d <= 2e-2 * float(np.sqrt(np.mean(ref ** 2)))
+
+
+def test_dense_attention_small_config_sampled():
+    wl = synth.WORKLOADS["small"].replace(heads=4)
+    q, k, v = synth.make_qkv(wl)
+    g = orc.Geometry.of(wl)
+    rng = np.random.default_rng(0)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 96), [0, 1, 4, wl.n_tokens - 1, 10944, 10943]]))
+    ref = orc.dense_attention(g, q, k, v, toks)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        out = ctx.dense_attention(*(hb.bf16_from_bits(x, DEV) for x in (q, k, v)))
+        torch.cuda.synchronize()
+        bits = hb.bits_from_bf16(out)
+        assert np.isfinite(parity.bits_to_f64(bits)).all()
+        parity.check_output(bits[toks], ref, what="dense small")
+
+
+def test_strided_layouts_fused_qkv_and_head_major_output():
+    """Q/K/V as slices of one [N][3][H][D] projection output; output written as [H][N][D]."""
+    wl = synth.Workload("strided", 4, 9, 9, 2, 4, 4, 0.5, 0.7, heads=4)
+    q, k, v = synth.make_qkv(wl)
+    H, N, D = wl.heads, wl.n_tokens, 64
+    fused = torch.empty(N, 3, H, D, dtype=torch.bfloat16, device=DEV)
+    for i, x in enumerate((q, k, v)):
+        fused[:, i] = hb.bf16_from_bits(x, DEV).permute(1, 0, 2)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        ref = ctx.global_attention(*(hb.bf16_from_bits(x, DEV) for x in (q, k, v)))
+        views = [fused[:, i].permute(1, 0, 2) for i in range(3)]      # [H][N][D] views, token stride 3*H*D
+        assert not views[0].is_contiguous()
+        got = ctx.global_attention(*views)
+        out_hm = torch.zeros(H, N, D, dtype=torch.bfloat16, device=DEV)
+        lib_out = hb._Tensor(out_hm.data_ptr(), N * D, D)
+        rc = ctx._lib.httm_global_attention(ctx._h, ctx._tensor(views[0], "q"), ctx._tensor(views[1], "k"),
+                                            ctx._tensor(views[2], "v"), lib_out, ctx._stream(None))
+        assert rc == 0
+        torch.cuda.synchronize()
+        assert torch.equal(ref, got)
+        assert torch.equal(out_hm.permute(1, 0, 2).reshape(N, H * D), ref)
+        d_ref = ctx.dense_attention(*(hb.bf16_from_bits(x, DEV) for x in (q, k, v)))
+        d_got = ctx.dense_attention(*views)
+        torch.cuda.synchronize()
+        assert torch.equal(d_ref, d_got)
+
+
+def test_stage_calls_equal_the_fused_call_and_host_entry_point():
+    wl = synth.WORKLOADS["tiny"].replace(heads=4)
+    q, k, v = synth.make_qkv(wl)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        ref = ctx.global_attention(dq, dk, dv)
+        n0 = ctx.launch_count()
+        out = ctx.new_output().zero_()
+        for st in range(5):
+            ctx.launch_stage(st, dq, dk, dv, out)
+        torch.cuda.synchronize()
+        assert ctx.launch_count() == n0 + 5
+        assert torch.equal(ref, out)
+        hq, hk, hv = (hb.bf16_from_bits(x, pin=True) for x in (q, k, v))
+        hout = torch.empty(wl.n_tokens, wl.heads * 64, dtype=torch.bfloat16).pin_memory()
+        ctx.attention_host(hq, hk, hv, hout)
+        torch.cuda.synchronize()
+        assert torch.equal(hout, ref.cpu())
+        dref = ctx.dense_attention(dq, dk, dv)
+        ctx.attention_host(hq, hk, hv, hout, dense=True)
+        torch.cuda.synchronize()
+        assert torch.equal(hout, dref.cpu())
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    wl = synth.WORKLOADS["tiny"].replace(heads=2)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        H, N, D = wl.heads, wl.n_tokens, 64
+        good = [torch.zeros(H, N, D, dtype=torch.bfloat16, device=DEV) for _ in range(3)]
+        out = ctx.new_output()
+        n0 = ctx.launch_count()
+        T = hb._Tensor
+        t = lambda x: ctx._tensor(x, "x")
+        o = ctx._tensor(out, "out", True)
+        call = lambda q, k, v, oo: ctx._lib.httm_global_attention(ctx._h, q, k, v, oo, ctx._stream(None))
+        assert call(T(None, N * D, D), t(good[1]), t(good[2]), o) == hb.ERR_INVALID_ARG
+        assert call(T(good[0].data_ptr() + 2, N * D, D), t(good[1]), t(good[2]), o) == hb.ERR_ALIGNMENT
+        assert call(T(good[0].data_ptr(), N * D, D + 4), t(good[1]), t(good[2]), o) == hb.ERR_ALIGNMENT
+        assert call(T(good[0].data_ptr(), N * D, 32), t(good[1]), t(good[2]), o) == hb.ERR_INVALID_ARG
+        assert call(t(good[0]), t(good[1]), t(good[2]), T(good[0].data_ptr(), D, H * D)) == hb.ERR_INVALID_ARG   # aliasing
+        assert ctx._lib.httm_dense_attention(ctx._h, t(good[0]), t(good[1]), T(None, 0, 0), o, ctx._stream(None)) == hb.ERR_INVALID_ARG
+        assert b"null" in ctx._lib.httm_last_error(ctx._h)
+        assert ctx._lib.httm_launch_stage(ctx._h, 9, t(good[0]), t(good[1]), t(good[2]), o, ctx._stream(None)) == hb.ERR_INVALID_ARG
+        buf = np.empty(3, dtype=np.int32)
+        assert ctx._lib.httm_export(ctx._h, hb.X_PI, buf.ctypes.data, buf.nbytes, None) == hb.ERR_INVALID_ARG
+        assert ctx.launch_count() == n0
+        with pytest.raises(hb.HttmError):
+            ctx.global_attention(good[0].float(), good[1], good[2])
+        torch.cuda.synchronize()
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+
+
+def test_small_config_full_size_sampled():
+    """VGGT-shaped small scene at full size: maps and merged tensors in full, attention on sampled tokens."""
+    wl = synth.WORKLOADS["small"]
+    rng = np.random.default_rng(1)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 64), np.arange(5), [wl.n_tokens - 1]]))
+    stats = run_case(wl, sample=toks)
+    assert stats["merged_exactly_rounded"] > 0.99
