@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the HTTM global-attention layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload medium] [--impl ours|reference]
+
+One step = one pass of the whole hot path (reorder, match, merge, attention on the merged
+sets, unmerge + inverse reorder) over one synthetic VGGT-shaped scene.  Prints ONE JSON line.
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the
+same workload on its own GPU: the path has no exchange step, so there is no data-path collective.
+`--impl reference` times the CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_21317_b200 import synth  # noqa: E402
+
+METRIC = "httm_global_attention_layer_throughput"
+UNIT = "tokens/s"
+
+
+def workload_config(wl):
+    return {"workload": f"{wl.name}: S={wl.frames} frames x (5 + {wl.grid_h}x{wl.grid_w}) = {wl.n_tokens} tokens, "
+                        f"{wl.heads} heads x {wl.head_dim}, blocks {wl.blk_frames}x{wl.blk_h}x{wl.blk_w}, "
+                        f"merge ratio q={wl.ratio_q} kv={wl.ratio_kv}, noise sigma {wl.sigma}, seed {wl.seed}",
+            "tokens": wl.n_tokens, "heads": wl.heads, "head_dim": wl.head_dim,
+            "l2_policy": "inputs (Q/K/V %.0f MB) and streamed workspace are larger than the 126 MB L2; no flush"
+                         % (3 * wl.heads * wl.n_tokens * wl.head_dim * 2 / 1e6),
+            "parallelism": "replicas only (single-GPU path)"}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------ CPU oracle arm
+
+def oracle_layer_time(wl, q, k, v, sample_rows=48, keep=False):
+    """Times the oracle as it stands on the host cores.  Reorder, match, merge and unmerge run in
+    full; attention runs on `sample_rows` merged query rows per head against all merged keys and is
+    scaled by M_q / sample_rows.  Returns (seconds per layer, details)."""
+    from oracle import httm_oracle as orc
+    g = orc.Geometry.of(wl)
+    t = {}
+    t0 = time.perf_counter()
+    pi, bs = orc.temporal_reorder(g)
+    qr, kr, vr = orc.reorder(g, pi, q), orc.reorder(g, pi, k), orc.reorder(g, pi, v)
+    t["reorder"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    aq, mbq, msq = orc.match(g, bs, wl.ratio_q, qr)
+    ak, mbk, msk = orc.match(g, bs, wl.ratio_kv, kr)
+    t["match"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    rq, Mq = orc.merged_rank(g, aq)
+    rk, Mk = orc.merged_rank(g, ak)
+    qm, km, vm = orc.merge(g, rq, Mq, qr), orc.merge(g, rk, Mk, kr), orc.merge(g, rk, Mk, vr)
+    t["merge"] = time.perf_counter() - t0
+    rows = np.unique(np.linspace(0, Mq - 1, sample_rows).astype(np.int64))
+    t0 = time.perf_counter()
+    o_rows = orc.attention(qm, km, vm, rows)
+    t_attn = time.perf_counter() - t0
+    t["attention_sampled"] = t_attn
+    t["attention_extrapolated"] = t_attn * Mq / len(rows)
+    t0 = time.perf_counter()
+    om = np.zeros((g.heads, Mq, g.head_dim))
+    om[:, rows] = o_rows
+    out = orc.unmerge(g, pi, rq, om)
+    t["unmerge"] = time.perf_counter() - t0
+    total = t["reorder"] + t["match"] + t["merge"] + t["attention_extrapolated"] + t["unmerge"]
+    info = {"seconds": {k_: round(v_, 4) for k_, v_ in t.items()}, "cores": orc.threads(),
+            "sample": f"reorder, match, merge, unmerge in full; attention on {len(rows)} of {Mq} merged query rows per head "
+                      f"(all {Mk} keys), scaled by M_q/rows"}
+    kept = None
+    if keep:
+        kept = dict(g=g, pi=pi, bs=bs, qr=qr, kr=kr, aq=aq, ak=ak, mbq=mbq, msq=msq, mbk=mbk, msk=msk, rq=rq, rows=rows,
+                    o_rows=o_rows, Mq=Mq, Mk=Mk, out=out)
+    return total, info, kept
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    q, k, v = synth.make_qkv(wl)
+    times = []
+    info = None
+    for i in range(args.warmup + args.steps):
+        tot, info, _ = oracle_layer_time(wl, q, k, v, sample_rows=args.oracle_rows)
+        if i >= args.warmup:
+            times.append(tot)
+    sec = float(np.mean(times))
+    val = wl.n_tokens / sec
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": workload_config(wl),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": info["cores"], "kind": "oracle", "sample": info["sample"],
+                             "seconds": info["seconds"]},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ GPU arm
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in open(self.path):
+            p = [x.strip() for x in ln.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1]))
+                mx.append(float(p[2]))
+                pw.append(float(p[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, p[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(np.max(mx)), "power_w_max": float(np.max(pw)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_21317_b200 import binding as hb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the HTTM path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    q, k, v = synth.make_qkv(wl)
+    ctx = hb.Httm(hb.HttmConfig.of(wl, device=local))
+    dq, dk, dv = (hb.bf16_from_bits(x, dev) for x in (q, k, v))
+    out = ctx.new_output()
+    stream = torch.cuda.current_stream()
+    N, H, D, Mq, Mk = wl.n_tokens, wl.heads, wl.head_dim, ctx.m_q, ctx.m_k
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    # ---- warm-up, then the timed region: K calls of the public entry point
+    for _ in range(max(args.warmup, 3)):
+        ctx.global_attention(dq, dk, dv, out)
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    l0 = ctx.launch_count()
+    e0, e1 = ev(), ev()
+    e0.record(stream)
+    for _ in range(args.steps):
+        ctx.global_attention(dq, dk, dv, out)
+    e1.record(stream)
+    barrier()
+    launches = ctx.launch_count() - l0
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+
+    # ---- per-kernel durations: the same five launches with events between them
+    stage_ms = np.zeros(5)
+    evs = [[ev() for _ in range(6)] for _ in range(args.steps)]
+    for s in range(args.steps):
+        evs[s][0].record(stream)
+        for st in range(5):
+            ctx.launch_stage(st, dq, dk, dv, out)
+            evs[s][st + 1].record(stream)
+    torch.cuda.synchronize()
+    for s in range(args.steps):
+        for st in range(5):
+            stage_ms[st] += evs[s][st].elapsed_time(evs[s][st + 1])
+    stage_ms /= args.steps
+
+    # ---- dense baseline of the same run (same attention kernel on the unmerged tokens)
+    dsteps = max(3, min(args.steps, 10))
+    dout = ctx.new_output()
+    for _ in range(2):
+        ctx.dense_attention(dq, dk, dv, dout)
+    torch.cuda.synchronize()
+    d0, d1 = ev(), ev()
+    d0.record(stream)
+    for _ in range(dsteps):
+        ctx.dense_attention(dq, dk, dv, dout)
+    d1.record(stream)
+    torch.cuda.synchronize()
+    dense_ms = d0.elapsed_time(d1) / dsteps
+    clocks = sampler.stop()
+
+    # ---- end to end through the host-buffer entry point (pinned memory, copies inside the timed region)
+    hq, hk, hv = (hb.bf16_from_bits(x, pin=True) for x in (q, k, v))
+    hout = torch.empty(N, H * D, dtype=torch.bfloat16).pin_memory()
+    esteps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        ctx.attention_host(hq, hk, hv, hout)
+    barrier()
+    t0, t1 = ev(), ev()
+    t0.record(stream)
+    for _ in range(esteps):
+        ctx.attention_host(hq, hk, hv, hout)
+    t1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1) / esteps)
+    status = ctx.query(hb.Q_DEVICE_STATUS)
+    same = bool(torch.equal(hout, out.cpu()))
+
+    if rank == 0:
+        peaks = load_peaks()
+        b = 2
+        alg = {
+            "reorder": 2 * 3 * H * N * D * b,
+            "match": 2 * H * N * D * b + 2 * H * N * 4,
+            "merge": 3 * H * N * D * b + 2 * H * N * 4 + H * (Mq + 2 * Mk) * D * b + H * N * 4,
+            "unmerge": H * Mq * D * b + H * N * 4 + H * N * D * b,
+        }
+        attn_flops = 4.0 * H * Mq * Mk * D
+        kernels = {}
+        for i, name in enumerate(hb.STAGE_NAMES):
+            ms = float(stage_ms[i])
+            if name == "attention":
+                tf = attn_flops / (ms * 1e-3) / 1e12
+                kernels[name] = {"ms": ms, "tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                                 "frac_of_nominal_2250": tf / 2250.0}
+            else:
+                gbs = alg[name] / (ms * 1e-3) / 1e9
+                kernels[name] = {"ms": ms, "algorithmic_mb": alg[name] / 1e6, "gbs": gbs,
+                                 "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0}
+        attn_ms = float(stage_ms[3])
+        attn_tf = attn_flops / (attn_ms * 1e-3) / 1e12
+        roofline = {"kernel": "attention (merged sets)", "bound": "tensor", "achieved": attn_tf,
+                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": attn_tf / peaks["bf16_tflops_sustained"],
+                    "peak_source": peaks["source"] + " (sustained bf16 GEMM; kernel timed inside the step)",
+                    "traffic": None}
+        line = {
+            "metric": METRIC, "value": world * N / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(wl),
+            "clocks": clocks,
+            "e2e": {"value": world * N / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": 3 * H * N * D * b, "d2h_bytes_per_step": H * N * D * b, "steps": esteps,
+                    "matches_device_path": same},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "kernels": kernels,
+            "merged_tokens": {"M_q": Mq, "M_k": Mk},
+            "dense": {"ms": dense_ms, "tflops": 4.0 * H * N * N * D / (dense_ms * 1e-3) / 1e12, "steps": dsteps},
+            "speedup_vs_dense": dense_ms / ms_step,
+            "device_status": status,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            sec, info, kept = oracle_layer_time(wl, q, k, v, sample_rows=args.oracle_rows, keep=True)
+            line["cpu_baseline"] = {"value": N / sec, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
+                                    "sample": info["sample"], "seconds": info["seconds"], "ms_per_layer_extrapolated": sec * 1e3}
+            line["parity_sample"] = parity_sample(ctx, hb, wl, kept, out)
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def parity_sample(ctx, hb, wl, kept, out):
+    """Compare the benchmark's own GPU results with the oracle values the CPU-baseline leg just produced:
+    assignment maps in full (margin rule), attention output on the sampled merged rows."""
+    from tests import parity
+    try:
+        aq, ak = ctx.export(hb.X_ASSIGN_Q), ctx.export(hb.X_ASSIGN_K)
+        g = kept["g"]
+        nq = parity.check_maps(g, wl.ratio_q, kept["bs"], kept["qr"], kept["aq"], kept["mbq"], kept["msq"], aq, "A_q")
+        nk = parity.check_maps(g, wl.ratio_kv, kept["bs"], kept["kr"], kept["ak"], kept["mbk"], kept["msk"], ak, "A_k")
+        res = {"maps": "ok", "blocks_differing_inside_margin": [int(nq), int(nk)]}
+        if nq == 0 and nk == 0:
+            om = parity.bits_to_f64(ctx.export(hb.X_O_MERGED))[:, kept["rows"]]
+            rms = float(np.sqrt(np.mean(kept["o_rows"] ** 2)))
+            err = float(np.abs(om - kept["o_rows"]).max())
+            res["attention_rows_max_err_over_rms"] = err / rms
+            res["attention"] = "ok" if err <= parity.OUT_TOL * rms else "FAIL"
+        else:
+            res["attention"] = "skipped here (maps differ inside the margin; covered by tests)"
+        return res
+    except AssertionError as e:   # report, never hide
+        return {"maps": "FAIL", "error": str(e)[:300]}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="medium", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
+    ap.add_argument("--block", default=None, help="override block shape, e.g. 4x4x4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--oracle-rows", type=int, default=4096, help="merged query rows per head the CPU oracle attends (sample)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.ratio is not None:
+        wl = wl.replace(ratio_q=args.ratio, ratio_kv=args.ratio)
+    if args.block:
+        bt, bh, bw = (int(x) for x in args.block.lower().split("x"))
+        wl = wl.replace(blk_frames=bt, blk_h=bh, blk_w=bw)
+    if args.impl == "reference":
+        args.steps = 2 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, wl)
+    else:
+        args.steps = 50 if args.steps is None else args.steps
+        args.warmup = 5 if args.warmup is None else args.warmup
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
