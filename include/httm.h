@@ -175,6 +175,33 @@ const char* httm_last_error(const httm_ctx* ctx);
 /* Number of kernels launched by the library on this context since it was created. */
 int64_t httm_launch_count(const httm_ctx* ctx);
 
+/*
+ * (No counterpart in the paper: a packaging variant of httm_global_attention.)
+ * The same HTTM global attention for callers that cannot allocate device memory at the time
+ * of the call and therefore cannot use httm_create, which calls cudaMalloc: for example code
+ * that runs after a serving process has handed the whole device to its own memory pool, or a
+ * latency-critical loop in which cudaMalloc's device-wide synchronisation is not acceptable.
+ * This call allocates nothing on the device (no cudaMalloc / cudaFree, no library allocator):
+ * every intermediate of the path lives in one array of HTTM_STATIC_SCRATCH_BYTES that is built
+ * into the library's device image, so every GPU that loads the library holds that much memory
+ * until the process exits.
+ *   - cfg describes the problem exactly as for httm_create (cfg->device selects the GPU);
+ *     q, k, v, out follow the rules at the top of this file and stay owned by the caller.
+ *   - Problems whose intermediates do not fit the array (roughly heads * N * 128 bytes * 5;
+ *     the tiny 1044-token, 16-head configuration needs about 11 MiB) are rejected with
+ *     HTTM_ERR_UNSUPPORTED before anything is launched; use a context for those.
+ *   - The first call on a device looks up the array's device address and sets kernel
+ *     attributes; make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents (the call
+ *     resets what must start clean).  Two calls that overlap on the GPU, e.g. on different
+ *     streams, race on it: serialise them.  Calls are serialised on the host by a lock.
+ *   - Intermediates cannot be exported and the device status word is not reported.
+ * Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA; message via httm_last_error(NULL).
+ */
+#define HTTM_STATIC_SCRATCH_BYTES (16u << 20)
+int httm_global_attention_static(const httm_config* cfg, httm_tensor q, httm_tensor k, httm_tensor v,
+                                 httm_tensor out, void* cuda_stream);
+
 /* Free the context and everything it owns.  The caller first synchronises every stream
  * the context was used on.  NULL is accepted. */
 int httm_destroy(httm_ctx* ctx);

@@ -30,6 +30,7 @@ _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPO
 EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
+    "httm_global_attention_static",
 )
 
 
@@ -74,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     L.httm_launch_count.argtypes = [vp]
     L.httm_launch_count.restype = i64
     L.httm_destroy.argtypes = [vp]
+    L.httm_global_attention_static.argtypes = [ctypes.POINTER(_Config), _Tensor, _Tensor, _Tensor, _Tensor, vp]
     for name in EXPORTED_SYMBOLS:
         if name not in ("httm_last_error", "httm_launch_count"):
             getattr(L, name).restype = ctypes.c_int
@@ -230,6 +232,36 @@ class Httm:
         self._check(self._lib.httm_export(self._h, what, arr.ctypes.data_as(ctypes.c_void_p), arr.nbytes,
                                           self._stream(stream)))
         return arr
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def global_attention_static(cfg: HttmConfig, q, k, v, out, stream=None):
+    """HTTM global attention without any device allocation (see httm_global_attention_static in
+    include/httm.h): q, k, v are CUDA bf16 [heads][tokens][64], out is CUDA bf16 [tokens][heads*64],
+    all owned by the caller.  Only problems whose intermediates fit the library's built-in
+    16 MiB scratch array are accepted."""
+    lib = load_library()
+    H, D = cfg.heads, cfg.head_dim
+    N = cfg.frames * (cfg.n_camera + cfg.n_register + cfg.grid_h * cfg.grid_w)
+    for t, name in ((q, "q"), (k, "k"), (v, "v")):
+        if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (H, N, D) or t.stride(2) != 1:
+            raise HttmError(ERR_INVALID_ARG, f"{name}: expected CUDA bfloat16 [heads][tokens][head_dim]")
+    if not out.is_cuda or out.dtype != torch.bfloat16 or out.numel() != N * H * D:
+        raise HttmError(ERR_INVALID_ARG, "out: expected CUDA bfloat16 [tokens][heads*head_dim]")
+    o = out.view(N, H, D)
+    c = _Config(cfg.frames, cfg.n_camera, cfg.n_register, cfg.grid_h, cfg.grid_w, H, D, cfg.blk_frames, cfg.blk_h,
+                cfg.blk_w, float(cfg.ratio_q), float(cfg.ratio_kv), cfg.device)
+    if stream is None:
+        stream = torch.cuda.current_stream(cfg.device)
+    rc = lib.httm_global_attention_static(
+        ctypes.byref(c), _Tensor(q.data_ptr(), q.stride(0), q.stride(1)), _Tensor(k.data_ptr(), k.stride(0), k.stride(1)),
+        _Tensor(v.data_ptr(), v.stride(0), v.stride(1)), _Tensor(o.data_ptr(), o.stride(1), o.stride(0)),
+        ctypes.c_void_p(stream.cuda_stream))
+    if rc != OK:
+        raise HttmError(rc, (lib.httm_last_error(None) or b"").decode())
+    return out
 
 
 def bf16_from_bits(bits: np.ndarray, device=None, pin: bool = False) -> torch.Tensor:

@@ -262,6 +262,11 @@ int device_status(httm_ctx* c, int32_t* value) {
 
 }  // namespace
 
+namespace httm {
+// lets other translation units of the library report through httm_last_error(NULL)
+void set_global_error(const std::string& msg) { g_create_error = msg; }
+}  // namespace httm
+
 extern "C" {
 
 int httm_create(const httm_config* cfg, httm_ctx** out) {
