@@ -202,6 +202,16 @@ int64_t httm_launch_count(const httm_ctx* ctx);
 int httm_global_attention_static(const httm_config* cfg, httm_tensor q, httm_tensor k, httm_tensor v,
                                  httm_tensor out, void* cuda_stream);
 
+/*
+ * Diagnostic: one 128-row tile through the tensor-core building blocks of the attention kernel
+ * (Eq. 3-4 on a single tile): s_out[128][128] = Q K^T and o_out[128][64] = bf16(s_out) V in fp32,
+ * with q, k, v contiguous bf16 [128][64] DEVICE arrays (16-byte aligned), s_out / o_out / status_dev
+ * device arrays owned by the caller.  *status_dev is set non-zero if a bounded wait gave up.
+ * Errors: INVALID_ARG, CUDA.
+ */
+int httm_selftest_tensor_core(const void* q, const void* k, const void* v, float* s_out, float* o_out,
+                              int* status_dev, void* cuda_stream);
+
 /* Free the context and everything it owns.  The caller first synchronises every stream
  * the context was used on.  NULL is accepted. */
 int httm_destroy(httm_ctx* ctx);

@@ -30,7 +30,7 @@ _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPO
 EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
-    "httm_global_attention_static",
+    "httm_global_attention_static", "httm_selftest_tensor_core",
 )
 
 
@@ -76,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     L.httm_launch_count.restype = i64
     L.httm_destroy.argtypes = [vp]
     L.httm_global_attention_static.argtypes = [ctypes.POINTER(_Config), _Tensor, _Tensor, _Tensor, _Tensor, vp]
+    L.httm_selftest_tensor_core.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
         if name not in ("httm_last_error", "httm_launch_count"):
             getattr(L, name).restype = ctypes.c_int
@@ -232,6 +233,25 @@ class Httm:
         self._check(self._lib.httm_export(self._h, what, arr.ctypes.data_as(ctypes.c_void_p), arr.nbytes,
                                           self._stream(stream)))
         return arr
+
+
+def selftest_tensor_core(q, k, v):
+    """One 128 x 64 tile: returns (Q K^T [128][128], bf16(Q K^T) V [128][64]) as fp32 CUDA tensors."""
+    lib = load_library()
+    for t in (q, k, v):
+        if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (128, 64) or not t.is_contiguous():
+            raise HttmError(ERR_INVALID_ARG, "expected contiguous CUDA bfloat16 [128][64]")
+    s = torch.zeros(128, 128, dtype=torch.float32, device=q.device)
+    o = torch.zeros(128, 64, dtype=torch.float32, device=q.device)
+    st = torch.zeros(1, dtype=torch.int32, device=q.device)
+    rc = lib.httm_selftest_tensor_core(q.data_ptr(), k.data_ptr(), v.data_ptr(), s.data_ptr(), o.data_ptr(), st.data_ptr(),
+                                       ctypes.c_void_p(torch.cuda.current_stream(q.device).cuda_stream))
+    if rc != OK:
+        raise HttmError(rc, "tensor-core self test could not be launched")
+    torch.cuda.synchronize(q.device)
+    if int(st.item()) != 0:
+        raise HttmError(ERR_TIMEOUT, "tensor-core self test: a bounded wait gave up")
+    return s, o
 
 
 STATIC_SCRATCH_BYTES = 16 << 20

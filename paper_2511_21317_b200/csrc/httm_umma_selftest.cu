@@ -1,0 +1,160 @@
+// One-tile check of the tcgen05 building blocks the attention kernel is made of:
+//   S = Q K^T        (A, B from shared memory, both K-major, 128 x 128 x 64)
+//   O = bf16(S) V    (A from tensor memory, B from shared memory MN-major, 128 x 64 x 128)
+// with Q, K, V tiles brought in by TMA (128-byte swizzle).  Also holds the host-side tensor-map
+// encoder used by the attention kernel.
+#include <mutex>
+
+#include "../../include/httm.h"
+#include "tc_sm100.cuh"
+
+namespace httm {
+
+namespace {
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode = nullptr;
+std::once_flag g_encode_once;
+
+void resolve_encode() {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+        g_encode = reinterpret_cast<EncodeFn>(fn);
+    else
+        cudaGetLastError();
+}
+}  // namespace
+
+bool encode_rows_tensor_map(CUtensorMap* map, const void* base, int64_t rows, int64_t heads, int64_t stride_row,
+                            int64_t stride_head, int box_rows) {
+    std::call_once(g_encode_once, resolve_encode);
+    if (!g_encode) return false;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)heads};
+    // a single head has no meaningful head stride; any multiple of 16 bytes is accepted
+    const cuuint64_t strides[2] = {(cuuint64_t)stride_row * 2, (cuuint64_t)(heads > 1 ? stride_head : stride_row * rows) * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+namespace {
+
+__global__ void __launch_bounds__(128) umma_selftest_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                            const __grid_constant__ CUtensorMap map_k,
+                                                            const __grid_constant__ CUtensorMap map_v, float* s_out, float* o_out,
+                                                            int* status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* sq = smem;             // 128 x 128 B
+    unsigned char* sk = smem + 16384;
+    unsigned char* sv = smem + 32768;
+    __shared__ uint64_t bars[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const uint32_t bar_tma = tc::smem_addr(&bars[0]), bar_mma = tc::smem_addr(&bars[1]);
+
+    if (tid == 0) {
+        abort_flag = 0;
+        tc::mbar_init(bar_tma, 1);
+        tc::mbar_init(bar_mma, 1);
+        tc::fence_barrier_init();
+    }
+    if (warp == 0) tc::tmem_alloc(tc::smem_addr(&tmem_base_slot), 256);
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem = tmem_base_slot;
+    const uint32_t t_s = tmem, t_o = tmem + 128;
+
+    if (tid == 0) {
+        tc::mbar_expect_tx(bar_tma, 3 * 16384);
+        tc::tma_load_3d(tc::smem_addr(sq), &map_q, bar_tma, 0, 0, 0);
+        tc::tma_load_3d(tc::smem_addr(sk), &map_k, bar_tma, 0, 0, 0);
+        tc::tma_load_3d(tc::smem_addr(sv), &map_v, bar_tma, 0, 0, 0);
+    }
+    bool ok = tc::mbar_wait(bar_tma, 0, &abort_flag);
+    if (ok && tid == 0) {
+        const uint64_t dq = tc::smem_desc_sw128(tc::smem_addr(sq)), dk = tc::smem_desc_sw128(tc::smem_addr(sk));
+        constexpr uint32_t idesc = tc::idesc_bf16(128, 128, false, false);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) tc::mma_ss(t_s, dq + 2 * k, dk + 2 * k, idesc, k > 0);   // 16 channels = 32 bytes per step
+        tc::mma_commit(bar_mma);
+    }
+    ok = ok && tc::mbar_wait(bar_mma, 0, &abort_flag);
+    tc::fence_after_sync();
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    if (ok) {
+        uint32_t p[64];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld32(t_s + lane_base + c * 32, r);
+            tc::tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s_out[tid * 128 + c * 32 + i] = __uint_as_float(r[i]);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                p[c * 16 + i] = *reinterpret_cast<const uint32_t*>(&v);
+            }
+        }
+        // P (bf16 pairs) over the first 64 columns of S
+        tc::tmem_st32(t_s + lane_base, p);
+        tc::tmem_st32(t_s + lane_base + 32, p + 32);
+        tc::tmem_wait_st();
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    if (ok && tid == 0) {
+        const uint64_t dv = tc::smem_desc_sw128(tc::smem_addr(sv));
+        constexpr uint32_t idesc = tc::idesc_bf16(128, 64, false, true);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)   // 16 keys per step: 8 TMEM columns of P, 16 rows (2048 bytes) of V
+            tc::mma_ts(t_o, t_s + 8 * k, dv + (uint64_t)(k * 2048 >> 4), idesc, k > 0);
+        tc::mma_commit(bar_mma);
+    }
+    ok = ok && tc::mbar_wait(bar_mma, 1, &abort_flag);
+    tc::fence_after_sync();
+    if (ok) {
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld32(t_o + lane_base + c * 32, r);
+            tc::tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o_out[tid * 64 + c * 32 + i] = __uint_as_float(r[i]);
+        }
+    }
+    if (!ok && tid == 0) atomicCAS(status, 0, 2);
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tc::tmem_dealloc(tmem, 256);
+}
+
+}  // namespace
+}  // namespace httm
+
+extern "C" int httm_selftest_tensor_core(const void* q, const void* k, const void* v, float* s_out, float* o_out,
+                                         int* status_dev, void* cuda_stream) {
+    using namespace httm;
+    if (!q || !k || !v || !s_out || !o_out || !status_dev) return HTTM_ERR_INVALID_ARG;
+    CUtensorMap mq, mk, mv;
+    if (!encode_rows_tensor_map(&mq, q, 128, 1, 64, 0, 128) || !encode_rows_tensor_map(&mk, k, 128, 1, 64, 0, 128) ||
+        !encode_rows_tensor_map(&mv, v, 128, 1, 64, 0, 128))
+        return HTTM_ERR_CUDA;
+    const int smem = 3 * 16384 + 1024;
+    if (cudaFuncSetAttribute(umma_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return HTTM_ERR_CUDA;
+    }
+    umma_selftest_kernel<<<1, 128, smem, static_cast<cudaStream_t>(cuda_stream)>>>(mq, mk, mv, s_out, o_out, status_dev);
+    return cudaGetLastError() == cudaSuccess ? HTTM_OK : HTTM_ERR_CUDA;
+}
