@@ -83,7 +83,8 @@ cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream);
 cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
 cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
 cudaError_t launch_unmerge(const UnmergeArgs& a, cudaStream_t stream);
-cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);
+cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 / TMEM kernel
+cudaError_t configure_attention();
 cudaError_t configure_kernels();   // one-time function attributes (dynamic shared memory sizes)
 
 }  // namespace httm

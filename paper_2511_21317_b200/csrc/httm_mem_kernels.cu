@@ -476,7 +476,7 @@ cudaError_t configure_kernels() {
     HTTM_SET_SMEM(merge_kernel<4>, match_warps_per_cta(128) * merge_warp_smem_bytes(128));
     HTTM_SET_SMEM(merge_kernel<8>, match_warps_per_cta(256) * merge_warp_smem_bytes(256));
 #undef HTTM_SET_SMEM
-    return cudaSuccess;
+    return configure_attention();
 }
 
 }  // namespace httm
