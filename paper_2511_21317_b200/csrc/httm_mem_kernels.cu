@@ -99,41 +99,82 @@ cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream) {
 }
 
 // ------------------------------------------------------------------------------------
+// Task cursor: (tensor t, head h, unit u) of a linear task index that advances by a fixed
+// stride, kept up to date with carries instead of 64-bit divisions in the loop.
+// ------------------------------------------------------------------------------------
+struct TaskCursor {
+    int t, h, u;
+    int st, sh, su;        // the stride, decomposed the same way
+    int heads, units;
+    __device__ void init(int64_t first, int64_t stride, int heads_, int units_) {
+        heads = heads_;
+        units = units_;
+        const int64_t per_tensor = (int64_t)heads * units;
+        t = (int)(first / per_tensor);
+        int64_t rem = first - t * per_tensor;
+        h = (int)(rem / units);
+        u = (int)(rem - (int64_t)h * units);
+        st = (int)(stride / per_tensor);
+        rem = stride - st * per_tensor;
+        sh = (int)(rem / units);
+        su = (int)(rem - (int64_t)sh * units);
+    }
+    __device__ __forceinline__ void advance() {
+        u += su;
+        if (u >= units) {
+            u -= units;
+            ++h;
+        }
+        h += sh;
+        if (h >= heads) {
+            h -= heads;
+            ++t;
+        }
+        t += st;
+    }
+};
+
+// ------------------------------------------------------------------------------------
 // a2. Block-wise bipartite matching (Eq. 1; Sec. 3.2 top-r rule), one warp per
 //     (tensor in {Q, K}, head, block).  The block (n x 64 bf16, contiguous after the
 //     reorder) is staged in shared memory by a tiled TMA load with the 128-byte swizzle,
-//     double buffered per warp, so that lane j reads its own row j without bank conflicts.
-//     Every lane keeps its row in registers as fp32; the dst rows are written once, as fp32,
-//     to a small per-warp table that all src lanes then read with broadcast loads.
-//     Similarities are fp32 dot products of the raw bf16 values (products are exact; two
-//     per instruction with packed fp32 FMAs) scaled by the inverse norms.
+//     double buffered per warp.  The dot products of every token with every dst token are
+//     a small dense contraction (n x n_dst x 64): they run on the tensor cores as
+//     m16n8k16 bf16 MMAs with fp32 accumulation, operands fetched with ldmatrix straight
+//     from the swizzled stage (conflict free); the dst rows are gathered by giving
+//     ldmatrix their row addresses.  Products of bf16 values are exact in fp32, and the
+//     accumulation error measured on this hardware is below that of an fp32 FMA chain.
+//     Squared norms are the diagonal of the same kind of MMA (a tile of rows against
+//     itself).  Similarity = dot * inv_norm(src) * inv_norm(dst).
 //     argmax ties -> lowest dst; top-r ties -> lowest src.  The r merged src are found by
 //     min(r, n_src - r) rounds of a warp-wide max (or min) extraction.
+//     Token j of a block is owned, for the selection, by lane (j & 7) * 4 + ((j >> 3) & 1),
+//     slot j >> 4: the lane where the MMA accumulator layout leaves row j's results.
 // ------------------------------------------------------------------------------------
-constexpr int kDstRowFloats = 68;   // 64 channels + inverse norm + local position + 2 pad (272 B: conflict-free row stores)
-
 __host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 32 ? 8 : (nmax <= 128 ? 4 : 2); }
-__host__ __device__ constexpr int match_aux_bytes(int nmax) { return (nmax / 4) * kDstRowFloats * 4 + 16; }
+__host__ __device__ constexpr int match_aux_bytes(int nmax) { return nmax * 4 + 16; }   // inverse norms + 2 mbarriers
 __host__ __device__ constexpr int match_smem_bytes(int nmax) {
     return match_warps_per_cta(nmax) * (2 * nmax * kRowBytes + match_aux_bytes(nmax)) + 1024 /*alignment slack*/;
 }
 
-__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
-    float2 d;
-    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
-        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
-        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
-        "mov.b64 {%0, %1}, rd;\n\t}"
-        : "=f"(d.x), "=f"(d.y)
-        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
-    return d;
-}
 // tiled TMA load {64 channels, rows, heads} -> this CTA's shared memory; the channel coordinate is 0
 __device__ __forceinline__ void tma_rows_load(uint32_t dst_smem, const CUtensorMap* map, uint32_t mbar, int row, int head) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
                      dst_smem),
                  "l"(reinterpret_cast<uint64_t>(map)), "r"(mbar), "r"(0), "r"(row), "r"(head)
                  : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t* r, uint32_t saddr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr)
+                 : "memory");
+}
+// c (16x8 fp32) += a (16x16 bf16, row) * b (16x8 bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 // monotone map float -> uint32 (larger float <-> larger key); every real score maps to a key >= 1
 __device__ __forceinline__ uint32_t score_key(float s) {
@@ -146,15 +187,18 @@ __global__ void __launch_bounds__(match_warps_per_cta(32 * PASSES) * 32)
 match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const MatchArgs a) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = match_warps_per_cta(NMAX);
+    constexpr int MT = NMAX / 16;        // 16-token row tiles
+    constexpr int NT = NMAX / 32;        // 8-dst column tiles (n_dst <= NMAX / 4)
+    constexpr bool KEEP_A = PASSES == 1; // row-tile fragments stay in registers between the two passes
     constexpr uint32_t STAGE_BYTES = NMAX * kRowBytes;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* stage = smem + (size_t)warp * 2 * STAGE_BYTES;                                     // [2][NMAX][128], 1024-aligned
+    const int g = lane >> 2, tq = lane & 3;   // accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
     unsigned char* aux = smem + (size_t)WARPS * 2 * STAGE_BYTES + (size_t)warp * match_aux_bytes(NMAX);
-    float* dstf = reinterpret_cast<float*>(aux);                                                      // [NMAX/4][68]
-    uint64_t* mbar = reinterpret_cast<uint64_t*>(aux + (NMAX / 4) * kDstRowFloats * 4);               // [2]
-    const uint32_t mbar0 = smem_u32(mbar), stage0 = smem_u32(stage);
+    float* invn = reinterpret_cast<float*>(aux);                                   // [NMAX]
+    const uint32_t mbar0 = smem_u32(aux + NMAX * 4);                               // 2 mbarriers
+    const uint32_t stage0 = smem_u32(smem + (size_t)warp * 2 * STAGE_BYTES);       // [2][NMAX][128], 1024-aligned
 
     if (lane == 0) {
         mbar_init(mbar0, 1);
@@ -164,45 +208,36 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     }
     __syncwarp();
 
-    const int64_t per_tensor = (int64_t)a.heads * a.n_blocks;
-    const int64_t n_tasks = 2 * per_tensor;
+    const int64_t n_tasks = 2ll * a.heads * a.n_blocks;
     const int64_t stride = (int64_t)gridDim.x * WARPS;
     const int64_t first = (int64_t)blockIdx.x * WARPS + warp;
+    TaskCursor cur, nxt;   // the task being processed; the task whose load is issued next
+    cur.init(first, stride, a.heads, a.n_blocks);
+    nxt = cur;
 
-    auto issue = [&](int64_t task, int buf) {   // lane 0 only; the whole box is always transferred (rows past the head's end are zero filled)
-        const int t = (int)(task / per_tensor);
-        const int64_t rem = task - t * per_tensor;
-        const int h = (int)(rem / a.n_blocks), b = (int)(rem - (int64_t)h * a.n_blocks);
-        const int start = __ldg(&a.blocks[b].start);
+    auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only; the whole box is transferred (rows past the head's end are zero filled)
+        const int start = __ldg(&a.blocks[c.u].start);
         const uint32_t mb = mbar0 + 8 * buf;
         mbar_expect_tx(mb, STAGE_BYTES);
-        tma_rows_load(stage0 + buf * STAGE_BYTES, t == 0 ? &map_q : &map_k, mb, start, h);
+        tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : &map_k, mb, start, c.h);
     };
-    if (lane == 0) {
-        if (first < n_tasks) issue(first, 0);
-        if (first + stride < n_tasks) issue(first + stride, 1);
-    }
+    if (first < n_tasks && lane == 0) issue(nxt, 0);
+    nxt.advance();
+    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+    nxt.advance();
 
-    // row j of a stage buffer, as 64 fp32 values in channel order (16-byte chunk c sits at c ^ (j & 7))
-    auto load_row = [&](const unsigned char* blk, int j, float* x) {
-        const unsigned char* row = blk + j * kRowBytes;
-        const int sw = j & 7;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) unpack8(*reinterpret_cast<const uint4*>(row + ((c ^ sw) << 4)), x + 8 * c);
-    };
+    int cached_n = -1, cached_nd = -1;
+    uint32_t magic_n = 0, magic_nd = 0;
 
     int it = 0;
     bool failed = false;
-    for (int64_t task = first; task < n_tasks; task += stride, ++it) {
+    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
         const int buf = it & 1;
         const uint32_t parity = (it >> 1) & 1;
-        const int t = (int)(task / per_tensor);
-        const int64_t rem = task - t * per_tensor;
-        const int h = (int)(rem / a.n_blocks), b = (int)(rem - (int64_t)h * a.n_blocks);
-        const BlockInfo bi = a.blocks[b];
-        const int n = bi.n, r = t == 0 ? bi.r_q : bi.r_k, nd = t == 0 ? bi.nd_q : bi.nd_k;
-        int32_t* A = a.assign[t] + (int64_t)h * a.n_tokens + bi.start;
-        const unsigned char* blk = stage + buf * STAGE_BYTES;
+        const bool more = task + 2 * stride < n_tasks;
+        const BlockInfo bi = a.blocks[cur.u];
+        const int n = bi.n, r = cur.t == 0 ? bi.r_q : bi.r_k, nd = cur.t == 0 ? bi.nd_q : bi.nd_k;
+        int32_t* A = a.assign[cur.t] + (int64_t)cur.h * a.n_tokens + bi.start;
         if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
             failed = true;
             break;
@@ -214,143 +249,181 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 if (j < n) A[j] = bi.start + j;
             }
             __syncwarp();
-            if (lane == 0 && task + 2 * stride < n_tasks) issue(task + 2 * stride, buf);
+            if (more && lane == 0) issue(nxt, buf);
             continue;
         }
-        // floor(x / n) for x < (n + 1) * nd by multiplication: exact for n <= 256, nd <= 64
-        const uint32_t magic = (1u << 23) / (uint32_t)n + 1u;
-        auto div_n = [&](int x) { return (int)(((uint32_t)x * magic) >> 23); };
-
-        // ---- phase 1: norms of every token; fp32 copy of the dst rows
-        float x[64];
-        float inv[PASSES];
-        bool is_src[PASSES];
-#pragma unroll
-        for (int p = 0; p < PASSES; ++p) {
-            const int j = lane + 32 * p;
-            inv[p] = 0.f;
-            is_src[p] = false;
-            if (j < n) {
-                load_row(blk, j, x);
-                float2 s0 = make_float2(0.f, 0.f), s1 = s0;
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    s0 = ffma2(make_float2(x[4 * k], x[4 * k + 1]), make_float2(x[4 * k], x[4 * k + 1]), s0);
-                    s1 = ffma2(make_float2(x[4 * k + 2], x[4 * k + 3]), make_float2(x[4 * k + 2], x[4 * k + 3]), s1);
-                }
-                inv[p] = 1.0f / fmaxf(sqrtf((s0.x + s0.y) + (s1.x + s1.y)), 1e-12f);
-                const int d = div_n(j * nd);
-                if (div_n((j + 1) * nd) > d) {   // dst number d
-                    float4* o = reinterpret_cast<float4*>(dstf + d * kDstRowFloats);
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) o[k] = make_float4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
-                    o[16] = make_float4(inv[p], __int_as_float(j), 0.f, 0.f);
-                } else {
-                    is_src[p] = true;
-                }
-            }
+        // floor(x / n) and floor(x / n_dst) by multiplication: exact for the operand ranges below (n <= 256, n_dst <= 64)
+        if (n != cached_n || nd != cached_nd) {
+            cached_n = n;
+            cached_nd = nd;
+            magic_n = (1u << 23) / (uint32_t)n + 1u;
+            magic_nd = (1u << 23) / (uint32_t)nd + 1u;
         }
-        __syncwarp();
-        if (PASSES == 1) {   // the row lives in registers from here on: the stage buffer can be refilled
-            if (lane == 0 && task + 2 * stride < n_tasks) issue(task + 2 * stride, buf);
-        }
+        auto div_n = [&](int x) { return (int)(((uint32_t)x * magic_n) >> 23); };          // x < (n + 1) * n_dst
+        auto pos_of = [&](int d) { return (int)(((uint32_t)((d + 1) * n + nd - 1) * magic_nd) >> 23) - 1; };   // position of dst d
+        const uint32_t blk = stage0 + buf * STAGE_BYTES;
+        // ldmatrix address of 16-byte chunk `chunk` of row `row` (chunk c of row j sits at c ^ (j & 7))
+        auto chunk_addr = [&](int row, int chunk) { return blk + row * kRowBytes + ((chunk ^ (row & 7)) << 4); };
 
-        // ---- phase 2: best dst of every src
-        uint32_t key[PASSES];
-        int best[PASSES];
+        // ---- pass 1: squared norms of every token = diagonal of (row tile) x (row tile)^T
+        uint32_t af[KEEP_A ? MT : 1][4][4];   // [tile][k step][a0..a3]
+        auto load_a = [&](int mt, uint32_t (*dstf)[4]) {
+            // matrices of one ldmatrix.x4: rows 0-7 / 8-15 of the tile (lane bit 3), k chunk 2 ks / 2 ks + 1 (lane bit 4)
+            const int row = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-        for (int p = 0; p < PASSES; ++p) {
-            key[p] = 0;
-            best[p] = 0;
-            if (p * 32 < n) {   // warp-uniform
-                if (is_src[p]) {
-                    if (PASSES > 1) load_row(blk, lane + 32 * p, x);
-                    float top = -INFINITY;
-                    int arg = 0;
-                    auto dot = [&](const float4* dr) {
-                        float2 c0 = make_float2(0.f, 0.f), c1 = c0;
+            for (int ks = 0; ks < 4; ++ks) ldmatrix_x4(dstf[ks], chunk_addr(row, 2 * ks + (lane >> 4)));
+        };
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float4 u = dr[k];
-                            c0 = ffma2(make_float2(x[4 * k], x[4 * k + 1]), make_float2(u.x, u.y), c0);
-                            c1 = ffma2(make_float2(x[4 * k + 2], x[4 * k + 3]), make_float2(u.z, u.w), c1);
-                        }
-                        return ((c0.x + c0.y) + (c1.x + c1.y)) * dr[16].x;
-                    };
-                    int d = 0;
-                    for (; d + 1 < nd; d += 2) {   // two dst at a time: four independent FMA chains
-                        const float s0 = dot(reinterpret_cast<const float4*>(dstf + d * kDstRowFloats));
-                        const float s1 = dot(reinterpret_cast<const float4*>(dstf + (d + 1) * kDstRowFloats));
-                        if (s0 > top) {
-                            top = s0;
-                            arg = d;
-                        }
-                        if (s1 > top) {
-                            top = s1;
-                            arg = d + 1;
-                        }
-                    }
-                    if (d < nd) {
-                        const float s0 = dot(reinterpret_cast<const float4*>(dstf + d * kDstRowFloats));
-                        if (s0 > top) {
-                            top = s0;
-                            arg = d;
-                        }
-                    }
-                    key[p] = score_key(top * inv[p]);
-                    best[p] = __float_as_int(dstf[arg * kDstRowFloats + 65]);
+        for (int mt = 0; mt < MT; ++mt) {
+            if (mt * 16 < n) {   // warp-uniform
+                uint32_t(*fr)[4] = af[KEEP_A ? mt : 0];
+                load_a(mt, fr);
+                float lo[4] = {0.f, 0.f, 0.f, 0.f}, hi[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    mma_bf16_16816(lo, fr[ks], fr[ks][0], fr[ks][2]);   // against rows 0-7 of the tile
+                    mma_bf16_16816(hi, fr[ks], fr[ks][1], fr[ks][3]);   // against rows 8-15
+                }
+                if (tq == (g >> 1)) {   // this lane holds the diagonal entries of rows g and g + 8
+                    const float s_lo = (g & 1) ? lo[1] : lo[0], s_hi = (g & 1) ? hi[3] : hi[2];
+                    invn[mt * 16 + g] = 1.0f / fmaxf(sqrtf(s_lo), 1e-12f);
+                    invn[mt * 16 + 8 + g] = 1.0f / fmaxf(sqrtf(s_hi), 1e-12f);
                 }
             }
         }
+        // ---- dst fragments: column tile nt holds dst 8 nt .. 8 nt + 7, gathered by row address
+        uint32_t bf[NT][4][2];   // [tile][k step][b0, b1]
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            if (nt * 8 < nd) {
+                const int d = min(nt * 8 + (lane & 7), nd - 1);
+                const int row = pos_of(d);
+#pragma unroll
+                for (int kp = 0; kp < 2; ++kp) {   // one ldmatrix.x4 = k steps 2 kp and 2 kp + 1
+                    uint32_t rr[4];
+                    ldmatrix_x4(rr, chunk_addr(row, 4 * kp + (lane >> 3)));
+                    bf[nt][2 * kp][0] = rr[0];
+                    bf[nt][2 * kp][1] = rr[1];
+                    bf[nt][2 * kp + 1][0] = rr[2];
+                    bf[nt][2 * kp + 1][1] = rr[3];
+                }
+            }
+        }
+        __syncwarp();   // inverse norms visible; with one pass, every fragment is now in registers
+        if (KEEP_A) {
+            if (more && lane == 0) issue(nxt, buf);
+        }
 
-        // ---- phase 3: the r src with the best scores merge (ties: lowest position first)
+        // ---- pass 2: similarities, best dst of every token (kept by the owner lane of the token)
+        uint32_t key[MT];
+        int best[MT];
+        bool is_src[MT];
+        const int own_half = tq & 1;   // owner of rows g (tq == 0) or g + 8 (tq == 1); lanes with tq >= 2 own nothing
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            key[mt] = 0;
+            best[mt] = 0;
+            is_src[mt] = false;
+            if (mt * 16 < n) {
+                uint32_t(*fr)[4] = af[KEEP_A ? mt : 0];
+                if (!KEEP_A) load_a(mt, fr);
+                float top[2] = {-INFINITY, -INFINITY};   // rows g, g + 8
+                int arg[2] = {0, 0};
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    if (nt * 8 < nd) {
+                        float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) mma_bf16_16816(c, fr[ks], bf[nt][ks][0], bf[nt][ks][1]);
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int d = nt * 8 + 2 * tq + e;
+                            if (d < nd) {
+                                const float w = invn[pos_of(d)];
+                                const float s0 = c[e] * w, s1 = c[2 + e] * w;
+                                if (s0 > top[0]) {
+                                    top[0] = s0;
+                                    arg[0] = d;
+                                }
+                                if (s1 > top[1]) {
+                                    top[1] = s1;
+                                    arg[1] = d;
+                                }
+                            }
+                        }
+                    }
+                }
+                // combine the four lanes of a row (ties: lowest dst)
+#pragma unroll
+                for (int hrow = 0; hrow < 2; ++hrow) {
+#pragma unroll
+                    for (int off = 1; off <= 2; off <<= 1) {
+                        const float ov = __shfl_xor_sync(0xffffffffu, top[hrow], off);
+                        const int oa = __shfl_xor_sync(0xffffffffu, arg[hrow], off);
+                        if (ov > top[hrow] || (ov == top[hrow] && oa < arg[hrow])) {
+                            top[hrow] = ov;
+                            arg[hrow] = oa;
+                        }
+                    }
+                }
+                const int j = mt * 16 + own_half * 8 + g;
+                if (tq < 2 && j < n) {
+                    const int dj = div_n(j * nd);
+                    if (!(div_n((j + 1) * nd) > dj)) {   // not a dst position: a src token
+                        is_src[mt] = true;
+                        key[mt] = score_key((own_half ? top[1] : top[0]) * invn[j]);
+                        best[mt] = pos_of(own_half ? arg[1] : arg[0]);
+                    }
+                }
+            }
+        }
+
+        // ---- the r src with the best scores merge (ties: lowest position first)
         const int n_src = n - nd, n_out = n_src - r;
-        bool merged[PASSES];
+        bool merged[MT];
         if (r <= n_out) {
 #pragma unroll
-            for (int p = 0; p < PASSES; ++p) merged[p] = false;
+            for (int mt = 0; mt < MT; ++mt) merged[mt] = false;
             for (int round = 0; round < r; ++round) {
                 uint32_t loc = 0;
 #pragma unroll
-                for (int p = 0; p < PASSES; ++p) loc = max(loc, (is_src[p] && !merged[p]) ? key[p] : 0u);
+                for (int mt = 0; mt < MT; ++mt) loc = max(loc, (is_src[mt] && !merged[mt]) ? key[mt] : 0u);
                 const uint32_t m = __reduce_max_sync(0xffffffffu, loc);
-                bool done = false;
+                int cand = 0x7fffffff;   // lowest own position holding the maximum
 #pragma unroll
-                for (int p = 0; p < PASSES; ++p) {
-                    const unsigned ball = __ballot_sync(0xffffffffu, is_src[p] && !merged[p] && key[p] == m);
-                    if (!done && ball) {
-                        if (lane == __ffs(ball) - 1) merged[p] = true;
-                        done = true;
-                    }
-                }
+                for (int mt = MT - 1; mt >= 0; --mt)
+                    if (is_src[mt] && !merged[mt] && key[mt] == m) cand = mt * 16 + own_half * 8 + g;
+                const int win = __reduce_min_sync(0xffffffffu, cand);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+                    if (is_src[mt] && win == mt * 16 + own_half * 8 + g) merged[mt] = true;
             }
         } else {
 #pragma unroll
-            for (int p = 0; p < PASSES; ++p) merged[p] = is_src[p];
+            for (int mt = 0; mt < MT; ++mt) merged[mt] = is_src[mt];
             for (int round = 0; round < n_out; ++round) {
                 uint32_t loc = 0xffffffffu;
 #pragma unroll
-                for (int p = 0; p < PASSES; ++p) loc = min(loc, merged[p] ? key[p] : 0xffffffffu);
+                for (int mt = 0; mt < MT; ++mt) loc = min(loc, merged[mt] ? key[mt] : 0xffffffffu);
                 const uint32_t m = __reduce_min_sync(0xffffffffu, loc);
-                bool done = false;
+                int cand = -1;           // highest own position holding the minimum
 #pragma unroll
-                for (int p = PASSES - 1; p >= 0; --p) {
-                    const unsigned ball = __ballot_sync(0xffffffffu, merged[p] && key[p] == m);
-                    if (!done && ball) {
-                        if (lane == 31 - __clz(ball)) merged[p] = false;
-                        done = true;
-                    }
-                }
+                for (int mt = 0; mt < MT; ++mt)
+                    if (merged[mt] && key[mt] == m) cand = mt * 16 + own_half * 8 + g;
+                const int win = __reduce_max_sync(0xffffffffu, cand);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+                    if (merged[mt] && win == mt * 16 + own_half * 8 + g) merged[mt] = false;
             }
         }
 #pragma unroll
-        for (int p = 0; p < PASSES; ++p) {
-            const int j = lane + 32 * p;
-            if (j < n) A[j] = bi.start + (merged[p] ? best[p] : j);
+        for (int mt = 0; mt < MT; ++mt) {
+            const int j = mt * 16 + own_half * 8 + g;
+            if (tq < 2 && j < n) A[j] = bi.start + (merged[mt] ? best[mt] : j);
         }
-        __syncwarp();   // every lane is done with the dst table (and, with several passes, the stage buffer)
-        if (PASSES > 1) {
-            if (lane == 0 && task + 2 * stride < n_tasks) issue(task + 2 * stride, buf);
+        __syncwarp();   // every lane is done with the inverse norms (and, with several passes, the stage buffer)
+        if (!KEEP_A) {
+            if (more && lane == 0) issue(nxt, buf);
         }
     }
     if (failed) {
@@ -372,9 +445,10 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
         !encode_rows_tensor_map(&mk, a.xr[1], N, a.heads, kHeadDim, N * kHeadDim, NMAX))
         return cudaErrorInvalidValue;
     const int64_t n_tasks = 2ll * a.heads * a.n_blocks;
-    const int ctas_per_sm = (int)((224 * 1024) / (smem + 1024));
+    int ctas_per_sm = (int)((224 * 1024) / (smem + 1024));
+    ctas_per_sm = ctas_per_sm < 1 ? 1 : (ctas_per_sm > 32 / WARPS ? 32 / WARPS : ctas_per_sm);
     int64_t grid = (n_tasks + WARPS - 1) / WARPS;
-    const int64_t cap = (int64_t)sm_count * (ctas_per_sm < 1 ? 1 : ctas_per_sm);
+    const int64_t cap = (int64_t)sm_count * ctas_per_sm;
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
     match_kernel<PASSES><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
@@ -422,30 +496,30 @@ __global__ void __launch_bounds__(merge_warps_per_cta(32 * PASSES) * 32) merge_k
     // task -> (tensor t, head h, unit u); units 0 .. n_blocks-1 are merging blocks, the rest are
     // chunks of 32 special tokens (never merged: rows 0 .. n_special_total-1 are copied)
     const int sp_chunks = (a.n_special_total + 31) / 32;
-    const int64_t per_head = (int64_t)a.n_blocks + sp_chunks;
-    const int64_t per_tensor = (int64_t)a.heads * per_head;
-    const int64_t n_tasks = 3 * per_tensor;
+    const int per_head = a.n_blocks + sp_chunks;
+    const int64_t n_tasks = 3ll * a.heads * per_head;
     const int64_t stride = (int64_t)gridDim.x * WARPS;
     const int64_t first = (int64_t)blockIdx.x * WARPS + warp;
+    TaskCursor cur, nxt;   // the task being processed; the task whose load is issued next
+    cur.init(first, stride, a.heads, per_head);
+    nxt = cur;
 
     struct Unit {
         int t, h, start, n, r, moff;
         bool special;
     };
-    auto decode = [&](int64_t task) {
+    auto decode = [&](const TaskCursor& c) {
         Unit u;
-        u.t = (int)(task / per_tensor);
-        const int64_t rem = task - u.t * per_tensor;
-        u.h = (int)(rem / per_head);
-        const int idx = (int)(rem - (int64_t)u.h * per_head);
-        u.special = idx >= a.n_blocks;
+        u.t = c.t;
+        u.h = c.h;
+        u.special = c.u >= a.n_blocks;
         if (u.special) {
-            u.start = (idx - a.n_blocks) * 32;
+            u.start = (c.u - a.n_blocks) * 32;
             u.n = min(32, a.n_special_total - u.start);
             u.r = 0;
             u.moff = u.start;
         } else {
-            const BlockInfo bi = a.blocks[idx];
+            const BlockInfo bi = a.blocks[c.u];
             u.start = bi.start;
             u.n = bi.n;
             u.r = u.t == 0 ? bi.r_q : bi.r_k;
@@ -453,24 +527,24 @@ __global__ void __launch_bounds__(merge_warps_per_cta(32 * PASSES) * 32) merge_k
         }
         return u;
     };
-    auto issue = [&](int64_t task, int buf) {   // lane 0 only
-        const Unit u = decode(task);
+    auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only
+        const Unit u = decode(c);
         const uint32_t bytes = (uint32_t)u.n * kRowBytes;
         const uint32_t mb = mbar0 + 8 * buf;
         mbar_expect_tx(mb, bytes);
         bulk_load(stage0 + buf * STAGE_BYTES, a.xr[u.t] + ((int64_t)u.h * a.n_tokens + u.start) * kHeadDim, bytes, mb);
     };
-    if (lane == 0) {
-        if (first < n_tasks) issue(first, 0);
-        if (first + stride < n_tasks) issue(first + stride, 1);
-    }
+    if (first < n_tasks && lane == 0) issue(nxt, 0);
+    nxt.advance();
+    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+    nxt.advance();
 
     int it = 0;
     bool failed = false;
-    for (int64_t task = first; task < n_tasks; task += stride, ++it) {
+    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
         const int buf = it & 1;
         const uint32_t parity = (it >> 1) & 1;
-        const Unit u = decode(task);
+        const Unit u = decode(cur);
         const int n = u.n;
         const int m_len = u.t == 0 ? a.m_q : a.m_k;
         uint32_t* out = reinterpret_cast<uint32_t*>(a.merged[u.t] + ((int64_t)u.h * m_len + u.moff) * kHeadDim);
@@ -570,7 +644,7 @@ __global__ void __launch_bounds__(merge_warps_per_cta(32 * PASSES) * 32) merge_k
             }
         }
         __syncwarp();   // every lane is done reading this stage buffer
-        if (lane == 0 && task + 2 * stride < n_tasks) issue(task + 2 * stride, buf);
+        if (lane == 0 && task + 2 * stride < n_tasks) issue(nxt, buf);
     }
     if (failed) {
         mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
