@@ -183,7 +183,7 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 }
 
 template <int PASSES>
-__global__ void __launch_bounds__(match_warps_per_cta(32 * PASSES) * 32)
+__global__ void __launch_bounds__(match_warps_per_cta(32 * PASSES) * 32, PASSES == 1 ? 3 : 1)
 match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const MatchArgs a) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = match_warps_per_cta(NMAX);
@@ -286,8 +286,9 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 }
                 if (tq == (g >> 1)) {   // this lane holds the diagonal entries of rows g and g + 8
                     const float s_lo = (g & 1) ? lo[1] : lo[0], s_hi = (g & 1) ? hi[3] : hi[2];
-                    invn[mt * 16 + g] = 1.0f / fmaxf(sqrtf(s_lo), 1e-12f);
-                    invn[mt * 16 + 8 + g] = 1.0f / fmaxf(sqrtf(s_hi), 1e-12f);
+                    // 1 / max(|x|, 1e-12): rsqrt.approx is within 2 ulp, far inside the 1e-5 margin rule
+                    invn[mt * 16 + g] = fminf(rsqrtf(s_lo), 1e12f);
+                    invn[mt * 16 + 8 + g] = fminf(rsqrtf(s_hi), 1e12f);
                 }
             }
         }
@@ -315,6 +316,14 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         }
 
         // ---- pass 2: similarities, best dst of every token (kept by the owner lane of the token)
+        float wd[NT][2];   // inverse norms of this lane's dst columns
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int d = nt * 8 + 2 * tq + e;
+                wd[nt][e] = d < nd ? invn[pos_of(d)] : 0.f;
+            }
         uint32_t key[MT];
         int best[MT];
         bool is_src[MT];
@@ -339,7 +348,7 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                         for (int e = 0; e < 2; ++e) {
                             const int d = nt * 8 + 2 * tq + e;
                             if (d < nd) {
-                                const float w = invn[pos_of(d)];
+                                const float w = wd[nt][e];
                                 const float s0 = c[e] * w, s1 = c[2 + e] * w;
                                 if (s0 > top[0]) {
                                     top[0] = s0;
