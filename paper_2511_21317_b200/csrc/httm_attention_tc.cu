@@ -5,8 +5,8 @@
 //   warp 0      TMA producer: Q tiles once, then a ring of K and V tiles (128-byte swizzle)
 //   warp 1      issues every tcgen05.mma: S_X = Q_X K^T (operands in shared memory) and
 //               O_X += P_X V (P_X read from tensor memory, V MN-major from shared memory)
-//   warps 4-7   softmax of tile A: one thread per query row, S read from tensor memory,
-//               P written back over S as bf16 pairs; warps 8-11 the same for tile B
+//   warps 2-5   softmax of tile A: one thread per query row, S read from tensor memory,
+//               P written back over S as bf16 pairs; warps 6-9 the same for tile B
 // While one tile's softmax runs, the tensor core works on the other tile.  Accumulators live in
 // tensor memory: S_A, S_B (128 columns each), O_A, O_B (64 columns each).  Running maxima are
 // only raised when they grow by more than 2^8 (then the softmax threads rescale O in place), so
@@ -14,6 +14,8 @@
 // kDevTimeoutAttention in the status word, releases its tensor memory and returns.
 #include "httm_internal.h"
 #include "tc_sm100.cuh"
+
+#include <type_traits>
 
 namespace httm {
 
@@ -23,7 +25,7 @@ constexpr int BM = 128;            // rows per query tile
 constexpr int BN = 128;            // keys per tile
 constexpr int KV_STAGES = 3;
 constexpr int TILE_BYTES = BM * kRowBytes;   // 16 KB
-constexpr int NTHREADS = 384;
+constexpr int NTHREADS = 320;   // producer warp, MMA warp, 2 x 4 softmax warps: 192 registers per thread at launch
 constexpr int TMEM_COLS = 512;
 constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
@@ -57,7 +59,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __maxnreg__(192)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const TcParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -99,11 +101,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const uint32_t tmem = bars->tmem_base;
     // columns: S_A [0,128)  S_B [128,256)  O_A [256,320)  O_B [320,384); P_X overlays the first 64 columns of S_X
 
-    // Register budget: the softmax threads hold a whole 128-wide row of S; the producer, the MMA
-    // issuer and the two idle warps give most of their registers to them (128*80 + 256*208 <= 64K).
+    // Register budget: the softmax threads hold a whole 128-wide row of S; with ten warps every thread
+    // has 192 registers from launch, so no register reallocation between the roles is needed.  A warp
+    // reaches the 32 TMEM lanes 32 * (warp % 4) ..: any four consecutive warps cover a 128-row tile.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (lane == 0) {
             const uint32_t qb = tc::smem_addr(&bars->q_full);
             tc::mbar_expect_tx(qb, 2 * TILE_BYTES);
@@ -125,63 +127,77 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        // Every operand of a tcgen05.mma below is a loop-invariant base plus a compile-time offset (the
+        // ring stage is a template constant, the loop is unrolled over the three stages): operands that
+        // are recomputed per instruction at run time make the issue itself cost more than the MMA.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = tc::idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_pv = tc::idesc_bf16(BM, kHeadDim, false, true);
-            const uint64_t dq[2] = {tc::smem_desc_sw128(s_q), tc::smem_desc_sw128(s_q + TILE_BYTES)};
-            auto issue_qk = [&](int x, int st) {
-                const uint64_t dk = tc::smem_desc_sw128(s_k + st * TILE_BYTES);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) tc::mma_ss(tmem + x * BN, dq[x] + 2 * k, dk + 2 * k, idesc_qk, k > 0);
-                tc::mma_commit(tc::smem_addr(&bars->s_full[x]));
+            const uint64_t dq0 = tc::smem_desc_sw128(s_q), dq1 = tc::smem_desc_sw128(s_q + TILE_BYTES);
+            const uint64_t dk0 = tc::smem_desc_sw128(s_k), dv0 = tc::smem_desc_sw128(s_v);
+            constexpr uint64_t kStageStep = TILE_BYTES >> 4;   // descriptor address field counts 16-byte units
+            const uint32_t t_s0 = tmem, t_s1 = tmem + BN, t_o0 = tmem + 2 * BN, t_o1 = tmem + 2 * BN + kHeadDim;
+            const uint32_t b_sfull0 = tc::smem_addr(&bars->s_full[0]), b_sfull1 = tc::smem_addr(&bars->s_full[1]);
+            const uint32_t b_pfull0 = tc::smem_addr(&bars->p_full[0]), b_pfull1 = tc::smem_addr(&bars->p_full[1]);
+            // S_x = Q_x K^T: four K=16 steps, 32 bytes apart inside the 128-byte rows
+            auto issue_qk = [&](uint32_t t_s, uint64_t dq, uint64_t dk, uint32_t bar) {
+                tc::mma_ss_c<false>(t_s, dq, dk, idesc_qk);
+                tc::mma_ss_c<true>(t_s, dq + 2, dk + 2, idesc_qk);
+                tc::mma_ss_c<true>(t_s, dq + 4, dk + 4, idesc_qk);
+                tc::mma_ss_c<true>(t_s, dq + 6, dk + 6, idesc_qk);
+                tc::mma_commit(bar);
             };
-            auto issue_pv = [&](int x, int st, bool first) {
-                const uint64_t dv = tc::smem_desc_sw128(s_v + st * TILE_BYTES);
+            // O_x += P_x V: eight K=16 steps; P advances 8 columns (16 bf16), V 16 rows (2048 bytes).
+            // O starts at zero (written by the softmax threads), so every step accumulates.
+            auto issue_pv = [&](uint32_t t_o, uint32_t t_p, uint64_t dv) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    tc::mma_ts(tmem + 2 * BN + x * kHeadDim, tmem + x * BN + 8 * k, dv + (uint64_t)(k * 2048 >> 4), idesc_pv,
-                               (!first || k > 0) ? 1u : 0u);
+                for (int k = 0; k < 8; ++k) tc::mma_ts_c<true>(t_o, t_p + 8 * k, dv + (uint64_t)(k * 128), idesc_pv);
+            };
+            // one key tile j held in ring stage ST; returns false when a wait gave up
+            auto step = [&](auto st_c, int j, uint32_t ph) -> bool {
+                constexpr int ST = decltype(st_c)::value, ST1 = (ST + 1) % KV_STAGES;
+                const uint32_t ph1 = ST == KV_STAGES - 1 ? ph ^ 1u : ph;
+                const bool more = j + 1 < n_tiles;
+                if (!tc::mbar_wait(tc::smem_addr(&bars->v_full[ST]), ph, abort_flag)) return false;
+                if (!tc::mbar_wait(b_pfull0, j & 1, abort_flag)) return false;
+                tc::fence_after_sync();
+                issue_pv(t_o0, t_s0, dv0 + ST * kStageStep);
+                if (more) {
+                    if (!tc::mbar_wait(tc::smem_addr(&bars->k_full[ST1]), ph1, abort_flag)) return false;
+                    tc::fence_after_sync();
+                    issue_qk(t_s0, dq0, dk0 + ST1 * kStageStep, b_sfull0);
+                }
+                if (!tc::mbar_wait(b_pfull1, j & 1, abort_flag)) return false;
+                tc::fence_after_sync();
+                issue_pv(t_o1, t_s1, dv0 + ST * kStageStep);
+                tc::mma_commit(tc::smem_addr(&bars->v_empty[ST]));
+                if (more) {
+                    issue_qk(t_s1, dq1, dk0 + ST1 * kStageStep, b_sfull1);
+                    tc::mma_commit(tc::smem_addr(&bars->k_empty[ST1]));
+                }
+                return true;
             };
             bool ok = tc::mbar_wait(tc::smem_addr(&bars->q_full), 0, abort_flag) &&
                       tc::mbar_wait(tc::smem_addr(&bars->k_full[0]), 0, abort_flag);
             if (ok) {
                 tc::fence_after_sync();
-                issue_qk(0, 0);
-                issue_qk(1, 0);
+                issue_qk(t_s0, dq0, dk0, b_sfull0);
+                issue_qk(t_s1, dq1, dk0, b_sfull1);
                 tc::mma_commit(tc::smem_addr(&bars->k_empty[0]));
             }
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                const int st = j % KV_STAGES, st1 = (j + 1) % KV_STAGES;
-                const uint32_t ph = (uint32_t)(j / KV_STAGES) & 1u, ph1 = (uint32_t)((j + 1) / KV_STAGES) & 1u;
-                const bool more = j + 1 < n_tiles;
-                if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->v_full[st]), ph, abort_flag))) break;
-                if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->p_full[0]), j & 1, abort_flag))) break;
-                tc::fence_after_sync();
-                issue_pv(0, st, j == 0);
-                if (more) {
-                    if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->k_full[st1]), ph1, abort_flag))) break;
-                    tc::fence_after_sync();
-                    issue_qk(0, st1);
-                }
-                if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->p_full[1]), j & 1, abort_flag))) break;
-                tc::fence_after_sync();
-                issue_pv(1, st, j == 0);
-                tc::mma_commit(tc::smem_addr(&bars->v_empty[st]));
-                if (more) {
-                    issue_qk(1, st1);
-                    tc::mma_commit(tc::smem_addr(&bars->k_empty[st1]));
-                }
+            static_assert(KV_STAGES == 3, "the issue loop is unrolled over three ring stages");
+            uint32_t ph = 0;
+            for (int j = 0; ok && j < n_tiles; ph ^= 1u) {
+                ok = step(std::integral_constant<int, 0>{}, j++, ph);
+                if (ok && j < n_tiles) ok = step(std::integral_constant<int, 1>{}, j++, ph);
+                if (ok && j < n_tiles) ok = step(std::integral_constant<int, 2>{}, j++, ph);
             }
             if (ok) tc::mma_commit(tc::smem_addr(&bars->o_final));
         }
         __syncwarp();
-    } else if (warp < 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
-        const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
+        const int x = (warp - 2) >> 2;                 // 0: tile A (warps 2-5), 1: tile B (warps 6-9)
         const int row = (warp & 3) * 32 + lane;        // row inside the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_s = tmem + x * BN + lane_addr;
@@ -190,6 +206,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const float c = p.scale_log2;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
+        {   // the accumulator O starts at zero: every PV step accumulates (ordered before the first p_full arrival)
+            uint32_t z[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) z[i] = 0u;
+            tc::tmem_st32(t_o, z);
+            tc::tmem_st32(t_o + 32, z);
+        }
         for (int j = 0; j < n_tiles; ++j) {
             if (!(ok = tc::mbar_wait(sbar, j & 1, abort_flag))) break;
             tc::fence_after_sync();
@@ -203,9 +226,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 for (int i = 0; i < BN; ++i)
                     if (i >= valid) s[i] = 0xff800000u;   // -inf: keys past the end
             }
-            float mx = __uint_as_float(s[0]);
+            // row maximum: four independent chains of three-input maxima
+            float mx4[4];
 #pragma unroll
-            for (int i = 1; i < BN; ++i) mx = fmaxf(mx, __uint_as_float(s[i]));
+            for (int q = 0; q < 4; ++q) {
+                mx4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
+#pragma unroll
+                for (int i = 2; i < 32; i += 2)
+                    mx4[q] = tc::fmax3(mx4[q], __uint_as_float(s[32 * q + i]), __uint_as_float(s[32 * q + i + 1]));
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m, mx * c);
             if (j == 0) {
                 m = m_new;
@@ -215,32 +245,36 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const float f = exp2f(m - m_new);
                 l *= f;
                 m = m_new;
-#pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    uint32_t o[32];
-                    tc::tmem_ld32(t_o + cc * 32, o);
+#pragma unroll 1
+                for (int cc = 0; cc < 8; ++cc) {   // eight columns at a time: this rare path must not cost registers
+                    uint32_t o[8];
+                    tc::tmem_ld8(t_o + cc * 8, o);
                     tc::tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                    tc::tmem_st32(t_o + cc * 32, o);
+                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                    tc::tmem_st8(t_o + cc * 8, o);
                 }
             }
-            const float neg_m = -m;
-            float sum = 0.f;
+            const float2 c2 = make_float2(c, c), neg_m2 = make_float2(-m, -m);
+            float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0;
 #pragma unroll
             for (int cc = 0; cc < 8; ++cc) {
                 uint32_t pk[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const float a = fast_exp2(fmaf(__uint_as_float(s[cc * 16 + 2 * i]), c, neg_m));
-                    const float b = fast_exp2(fmaf(__uint_as_float(s[cc * 16 + 2 * i + 1]), c, neg_m));
-                    sum += a + b;
-                    pk[i] = pack_bf16(a, b);
+                    const float2 t = tc::ffma2(make_float2(__uint_as_float(s[cc * 16 + 2 * i]), __uint_as_float(s[cc * 16 + 2 * i + 1])), c2, neg_m2);
+                    const float2 e = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+                    if (i & 1)
+                        sum1 = tc::fadd2(sum1, e);
+                    else
+                        sum0 = tc::fadd2(sum0, e);
+                    pk[i] = pack_bf16(e.x, e.y);
                 }
                 asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(t_s + cc * 8),
                              "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7])
                              : "memory");
             }
+            const float sum = (sum0.x + sum0.y) + (sum1.x + sum1.y);
             l += sum;
             tc::tmem_wait_st();
             tc::fence_before_sync();
