@@ -3,15 +3,18 @@
 //
 // One CTA owns TWO 128-row query tiles (A, B) of one head and walks the keys in 128-key tiles.
 //   warp 0      TMA producer: Q tiles once, then a ring of K and V tiles (128-byte swizzle)
-//   warp 1      issues every tcgen05.mma: S_X = Q_X K^T (operands in shared memory) and
-//               O_X += P_X V (P_X read from tensor memory, V MN-major from shared memory)
+//   warp 1      issues every tcgen05.mma: S = Q_X K^T (operands in shared memory) and
+//               O_X += P V (P read from tensor memory, V MN-major from shared memory)
 //   warps 2-5   softmax of tile A: one thread per query row, S read from tensor memory,
 //               P written back over S as bf16 pairs; warps 6-9 the same for tile B
-// While one tile's softmax runs, the tensor core works on the other tile.  Accumulators live in
-// tensor memory: S_A, S_B (128 columns each), O_A, O_B (64 columns each).  Running maxima are
-// only raised when they grow by more than 2^8 (then the softmax threads rescale O in place), so
-// rescaling is rare after the first tiles.  Every wait is bounded; on expiry the kernel records
-// kDevTimeoutAttention in the status word, releases its tensor memory and returns.
+// Score tiles are numbered k = 2 j + x (key tile j, query tile x) and live in a ring of THREE
+// 128-column buffers of tensor memory shared by both query tiles (tile k in buffer k mod 3); the
+// accumulators O_A, O_B take the remaining 2 x 64 columns.  S(k+3) is issued right after P(k) V, into
+// the buffer that P(k) V releases, so the scores of a softmax warp's next tile are ready before it
+// finishes the current one: the softmax warps never wait for the tensor core in steady state.
+// Running maxima are only raised when they grow by more than 2^8 (then the softmax threads rescale O
+// in place), so rescaling is rare after the first tiles.  Every wait is bounded; on expiry the kernel
+// records kDevTimeoutAttention in the status word, releases its tensor memory and returns.
 #include "httm_internal.h"
 #include "tc_sm100.cuh"
 
@@ -25,7 +28,7 @@ constexpr int BM = 128;            // rows per query tile
 constexpr int BN = 128;            // keys per tile
 constexpr int KV_STAGES = 3;
 constexpr int TILE_BYTES = BM * kRowBytes;   // 16 KB
-constexpr int NTHREADS = 320;   // producer warp, MMA warp, 2 x 4 softmax warps: 192 registers per thread at launch
+constexpr int NTHREADS = 320;   // producer warp, MMA warp, 2 x 4 softmax warps: registers are granted per four warps, so 168 per thread as with twelve
 constexpr int TMEM_COLS = 512;
 constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
@@ -34,7 +37,8 @@ struct Barriers {
     uint64_t q_full;
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
-    uint64_t s_full[2], p_full[2];
+    uint64_t s_full[3], p_full[3];   // per score buffer
+    uint64_t o_done[2];              // per query tile: one completion per P V
     uint64_t o_final;
     uint32_t tmem_base;
     int abort_flag;
@@ -59,7 +63,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-__global__ void __maxnreg__(192)
+__global__ void __launch_bounds__(NTHREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const TcParams p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -84,10 +88,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             tc::mbar_init(tc::smem_addr(&bars->v_full[i]), 1);
             tc::mbar_init(tc::smem_addr(&bars->v_empty[i]), 1);
         }
-        for (int x = 0; x < 2; ++x) {
-            tc::mbar_init(tc::smem_addr(&bars->s_full[x]), 1);
-            tc::mbar_init(tc::smem_addr(&bars->p_full[x]), 128);
+        for (int b = 0; b < 3; ++b) {
+            tc::mbar_init(tc::smem_addr(&bars->s_full[b]), 1);
+            tc::mbar_init(tc::smem_addr(&bars->p_full[b]), 128);
         }
+        tc::mbar_init(tc::smem_addr(&bars->o_done[0]), 1);
+        tc::mbar_init(tc::smem_addr(&bars->o_done[1]), 1);
         tc::mbar_init(tc::smem_addr(&bars->o_final), 1);
         tc::fence_barrier_init();
         tc::prefetch_tensormap(&map_q);
@@ -99,10 +105,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     __syncthreads();
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
-    // columns: S_A [0,128)  S_B [128,256)  O_A [256,320)  O_B [320,384); P_X overlays the first 64 columns of S_X
+    // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the first 64 columns of its S
 
     // Register budget: the softmax threads hold a whole 128-wide row of S; with ten warps every thread
-    // has 192 registers from launch, so no register reallocation between the roles is needed.  A warp
+    // has 168 registers from launch, so no register reallocation between the roles is needed.  A warp
     // reaches the 32 TMEM lanes 32 * (warp % 4) ..: any four consecutive warps cover a 128-row tile.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -133,13 +139,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (lane == 0) {
             constexpr uint32_t idesc_qk = tc::idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_pv = tc::idesc_bf16(BM, kHeadDim, false, true);
-            const uint64_t dq0 = tc::smem_desc_sw128(s_q), dq1 = tc::smem_desc_sw128(s_q + TILE_BYTES);
+            const uint64_t dq0 = tc::smem_desc_sw128(s_q);
             const uint64_t dk0 = tc::smem_desc_sw128(s_k), dv0 = tc::smem_desc_sw128(s_v);
             constexpr uint64_t kStageStep = TILE_BYTES >> 4;   // descriptor address field counts 16-byte units
-            const uint32_t t_s0 = tmem, t_s1 = tmem + BN, t_o0 = tmem + 2 * BN, t_o1 = tmem + 2 * BN + kHeadDim;
-            const uint32_t b_sfull0 = tc::smem_addr(&bars->s_full[0]), b_sfull1 = tc::smem_addr(&bars->s_full[1]);
-            const uint32_t b_pfull0 = tc::smem_addr(&bars->p_full[0]), b_pfull1 = tc::smem_addr(&bars->p_full[1]);
-            // S_x = Q_x K^T: four K=16 steps, 32 bytes apart inside the 128-byte rows
+            const int n_score = 2 * n_tiles;                   // score tiles k = 2 j + x
+            // S(buffer) = Q_x K(stage)^T: four K=16 steps, 32 bytes apart inside the 128-byte rows
             auto issue_qk = [&](uint32_t t_s, uint64_t dq, uint64_t dk, uint32_t bar) {
                 tc::mma_ss_c<false>(t_s, dq, dk, idesc_qk);
                 tc::mma_ss_c<true>(t_s, dq + 2, dk + 2, idesc_qk);
@@ -147,50 +151,59 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 tc::mma_ss_c<true>(t_s, dq + 6, dk + 6, idesc_qk);
                 tc::mma_commit(bar);
             };
-            // O_x += P_x V: eight K=16 steps; P advances 8 columns (16 bf16), V 16 rows (2048 bytes).
+            // O_x += P(buffer) V(stage): eight K=16 steps; P advances 8 columns (16 bf16), V 16 rows (2048 bytes).
             // O starts at zero (written by the softmax threads), so every step accumulates.
             auto issue_pv = [&](uint32_t t_o, uint32_t t_p, uint64_t dv) {
 #pragma unroll
                 for (int k = 0; k < 8; ++k) tc::mma_ts_c<true>(t_o, t_p + 8 * k, dv + (uint64_t)(k * 128), idesc_pv);
             };
-            // one key tile j held in ring stage ST; returns false when a wait gave up
-            auto step = [&](auto st_c, int j, uint32_t ph) -> bool {
-                constexpr int ST = decltype(st_c)::value, ST1 = (ST + 1) % KV_STAGES;
-                const uint32_t ph1 = ST == KV_STAGES - 1 ? ph ^ 1u : ph;
-                const bool more = j + 1 < n_tiles;
-                if (!tc::mbar_wait(tc::smem_addr(&bars->v_full[ST]), ph, abort_flag)) return false;
-                if (!tc::mbar_wait(b_pfull0, j & 1, abort_flag)) return false;
+            // Score tile k = k0 + C with k0 a multiple of 6: buffer, query tile and ring stages are compile-time.
+            // round_par = parity of k0 / 6.  Returns false when a wait gave up.
+            auto step = [&](auto c_c, int k0, uint32_t round_par) -> bool {
+                constexpr int C = decltype(c_c)::value;
+                constexpr int B = C % 3, X = C % 2, ST = (C >> 1) % KV_STAGES;                 // this tile: P(k) V
+                constexpr int X3 = 1 - X, J3 = (C + 3) >> 1, ST3 = J3 % KV_STAGES;            // tile k + 3: next S in the same buffer
+                const uint32_t t_buf = tmem + B * BN, t_o = tmem + 3 * BN + X * kHeadDim;
+                if (X == 0 && !tc::mbar_wait(tc::smem_addr(&bars->v_full[ST]), round_par, abort_flag)) return false;
+                if (!tc::mbar_wait(tc::smem_addr(&bars->p_full[B]), (C / 3) & 1, abort_flag)) return false;
                 tc::fence_after_sync();
-                issue_pv(t_o0, t_s0, dv0 + ST * kStageStep);
-                if (more) {
-                    if (!tc::mbar_wait(tc::smem_addr(&bars->k_full[ST1]), ph1, abort_flag)) return false;
-                    tc::fence_after_sync();
-                    issue_qk(t_s0, dq0, dk0 + ST1 * kStageStep, b_sfull0);
-                }
-                if (!tc::mbar_wait(b_pfull1, j & 1, abort_flag)) return false;
-                tc::fence_after_sync();
-                issue_pv(t_o1, t_s1, dv0 + ST * kStageStep);
-                tc::mma_commit(tc::smem_addr(&bars->v_empty[ST]));
-                if (more) {
-                    issue_qk(t_s1, dq1, dk0 + ST1 * kStageStep, b_sfull1);
-                    tc::mma_commit(tc::smem_addr(&bars->k_empty[ST1]));
+                issue_pv(t_o, t_buf, dv0 + ST * kStageStep);
+                tc::mma_commit(tc::smem_addr(&bars->o_done[X]));
+                if (X == 1) tc::mma_commit(tc::smem_addr(&bars->v_empty[ST]));
+                if (k0 + C + 3 < n_score) {
+                    if (X3 == 0) {
+                        if (!tc::mbar_wait(tc::smem_addr(&bars->k_full[ST3]), round_par ^ (J3 >= 3 ? 1u : 0u), abort_flag)) return false;
+                        tc::fence_after_sync();
+                    }
+                    issue_qk(t_buf, dq0 + X3 * kStageStep, dk0 + ST3 * kStageStep, tc::smem_addr(&bars->s_full[B]));
+                    if (X3 == 1) tc::mma_commit(tc::smem_addr(&bars->k_empty[ST3]));
                 }
                 return true;
             };
+            static_assert(KV_STAGES == 3, "the issue loop is unrolled over 6 = lcm(3 score buffers, 2 query tiles, 3 ring stages) / ... score tiles");
             bool ok = tc::mbar_wait(tc::smem_addr(&bars->q_full), 0, abort_flag) &&
                       tc::mbar_wait(tc::smem_addr(&bars->k_full[0]), 0, abort_flag);
-            if (ok) {
+            if (ok) {   // prologue: S(0), S(1) from key tile 0, S(2) from key tile 1
                 tc::fence_after_sync();
-                issue_qk(t_s0, dq0, dk0, b_sfull0);
-                issue_qk(t_s1, dq1, dk0, b_sfull1);
+                issue_qk(tmem, dq0, dk0, tc::smem_addr(&bars->s_full[0]));
+                issue_qk(tmem + BN, dq0 + kStageStep, dk0, tc::smem_addr(&bars->s_full[1]));
                 tc::mma_commit(tc::smem_addr(&bars->k_empty[0]));
+                if (n_score > 2) {
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->k_full[1]), 0, abort_flag);
+                    if (ok) {
+                        tc::fence_after_sync();
+                        issue_qk(tmem + 2 * BN, dq0, dk0 + kStageStep, tc::smem_addr(&bars->s_full[2]));
+                    }
+                }
             }
-            static_assert(KV_STAGES == 3, "the issue loop is unrolled over three ring stages");
-            uint32_t ph = 0;
-            for (int j = 0; ok && j < n_tiles; ph ^= 1u) {
-                ok = step(std::integral_constant<int, 0>{}, j++, ph);
-                if (ok && j < n_tiles) ok = step(std::integral_constant<int, 1>{}, j++, ph);
-                if (ok && j < n_tiles) ok = step(std::integral_constant<int, 2>{}, j++, ph);
+            uint32_t round_par = 0;
+            for (int k0 = 0; ok && k0 < n_score; k0 += 6, round_par ^= 1u) {
+                ok = step(std::integral_constant<int, 0>{}, k0, round_par);
+                if (ok) ok = step(std::integral_constant<int, 1>{}, k0, round_par);          // n_score is even
+                if (ok && k0 + 2 < n_score) ok = step(std::integral_constant<int, 2>{}, k0, round_par);
+                if (ok && k0 + 2 < n_score) ok = step(std::integral_constant<int, 3>{}, k0, round_par);
+                if (ok && k0 + 4 < n_score) ok = step(std::integral_constant<int, 4>{}, k0, round_par);
+                if (ok && k0 + 4 < n_score) ok = step(std::integral_constant<int, 5>{}, k0, round_par);
             }
             if (ok) tc::mma_commit(tc::smem_addr(&bars->o_final));
         }
@@ -200,9 +213,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const int x = (warp - 2) >> 2;                 // 0: tile A (warps 2-5), 1: tile B (warps 6-9)
         const int row = (warp & 3) * 32 + lane;        // row inside the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + x * BN + lane_addr;
-        const uint32_t t_o = tmem + 2 * BN + x * kHeadDim + lane_addr;
-        const uint32_t sbar = tc::smem_addr(&bars->s_full[x]), pbar = tc::smem_addr(&bars->p_full[x]);
+        const uint32_t t_o = tmem + 3 * BN + x * kHeadDim + lane_addr;
+        const uint32_t obar = tc::smem_addr(&bars->o_done[x]);
         const float c = p.scale_log2;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
@@ -214,7 +226,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             tc::tmem_st32(t_o + 32, z);
         }
         for (int j = 0; j < n_tiles; ++j) {
-            if (!(ok = tc::mbar_wait(sbar, j & 1, abort_flag))) break;
+            const int k = 2 * j + x, buf = k % 3;                      // score tile and its buffer
+            const uint32_t kpar = (uint32_t)(k / 3) & 1u;
+            const uint32_t t_s = tmem + buf * BN + lane_addr;
+            const uint32_t sbar = tc::smem_addr(&bars->s_full[buf]), pbar = tc::smem_addr(&bars->p_full[buf]);
+            if (!(ok = tc::mbar_wait(sbar, kpar, abort_flag))) break;
             tc::fence_after_sync();
             uint32_t s[BN];   // fp32 bit patterns of this row of S
 #pragma unroll
@@ -240,8 +256,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             if (j == 0) {
                 m = m_new;
             } else if (__any_sync(0xffffffffu, m_new - m > kRescaleThreshold)) {
-                // raise the running maximum: rescale the row sum and the accumulator O in place
-                // (s_full(j) was committed after PV(j-1), so O is quiescent here)
+                // raise the running maximum: rescale the row sum and the accumulator O in place, once the
+                // previous P V of this query tile has completed (the next one is issued after this tile's P)
+                if (!(ok = tc::mbar_wait(obar, (uint32_t)(j - 1) & 1u, abort_flag))) break;
+                tc::fence_after_sync();
                 const float f = exp2f(m - m_new);
                 l *= f;
                 m = m_new;
