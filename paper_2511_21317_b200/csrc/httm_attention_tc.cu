@@ -63,6 +63,28 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// 2^t for two values without the special-function unit: round-to-nearest range reduction
+// t = n + f, f in [-0.5, 0.5] (the integer lands in the low mantissa bits of t + 1.5 * 2^23), a cubic
+// minimax polynomial for 2^f (relative error < 1e-4, far below the bf16 rounding of P) evaluated with
+// packed fp32 FMAs, and n added to the exponent field.  Arguments below -125 give 2^-125.
+__device__ __forceinline__ float2 exp2_poly2(float2 t) {
+    const float kMagic = 12582912.0f;
+    t.x = fmaxf(t.x, -125.0f);
+    t.y = fmaxf(t.y, -125.0f);
+    const float2 tt = tc::fadd2(t, make_float2(kMagic, kMagic));
+    const float2 n = tc::fadd2(tt, make_float2(-kMagic, -kMagic));
+    const float2 f = tc::ffma2(n, make_float2(-1.0f, -1.0f), t);
+    float2 q = tc::ffma2(make_float2(0.055171460f, 0.055171460f), f, make_float2(0.24261086f, 0.24261086f));
+    q = tc::ffma2(q, f, make_float2(0.69326097f, 0.69326097f));
+    q = tc::ffma2(q, f, make_float2(0.99992812f, 0.99992812f));
+    return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(tt.x) << 23)),
+                       __int_as_float(__float_as_int(q.y) + (__float_as_int(tt.y) << 23)));
+}
+// Of every eight pairs of scores, the pairs whose bit is set here take the polynomial (FMA pipe), the
+// others ex2.approx (special-function unit, 16 results per clock per SM): with every exponential on
+// that unit the softmax of two query tiles alone takes twice as long as their tensor-core work.
+constexpr uint32_t kPolyPairs = 0x52;   // pairs 1, 4, 6 of 8
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const TcParams p) {
@@ -112,7 +134,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // reaches the 32 TMEM lanes 32 * (warp % 4) ..: any four consecutive warps cover a 128-row tile.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (tc::elect_one()) {
             const uint32_t qb = tc::smem_addr(&bars->q_full);
             tc::mbar_expect_tx(qb, 2 * TILE_BYTES);
             tc::tma_load_3d(s_q, &map_q, qb, 0, q0, head);
@@ -136,7 +158,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // Every operand of a tcgen05.mma below is a loop-invariant base plus a compile-time offset (the
         // ring stage is a template constant, the loop is unrolled over the three stages): operands that
         // are recomputed per instruction at run time make the issue itself cost more than the MMA.
-        if (lane == 0) {
+        if (tc::elect_one()) {
             constexpr uint32_t idesc_qk = tc::idesc_bf16(BM, BN, false, false);
             constexpr uint32_t idesc_pv = tc::idesc_bf16(BM, kHeadDim, false, true);
             const uint64_t dq0 = tc::smem_desc_sw128(s_q);
@@ -281,7 +303,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const float2 t = tc::ffma2(make_float2(__uint_as_float(s[cc * 16 + 2 * i]), __uint_as_float(s[cc * 16 + 2 * i + 1])), c2, neg_m2);
-                    const float2 e = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+                    const float2 e = ((kPolyPairs >> i) & 1u) ? exp2_poly2(t) : make_float2(fast_exp2(t.x), fast_exp2(t.y));
                     if (i & 1)
                         sum1 = tc::fadd2(sum1, e);
                     else

@@ -19,6 +19,14 @@ __device__ __forceinline__ uint64_t timer_ns() {
     return t;
 }
 
+// One lane of a fully active warp.  Code behind this predicate is known to the assembler to run
+// in a single thread, which keeps the uniform operands of tcgen05.mma / TMA instructions cheap.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
