@@ -81,9 +81,12 @@ __device__ __forceinline__ float2 exp2_poly2(float2 t) {
                        __int_as_float(__float_as_int(q.y) + (__float_as_int(tt.y) << 23)));
 }
 // Of every eight pairs of scores, the pairs whose bit is set here take the polynomial (FMA pipe), the
-// others ex2.approx (special-function unit, 16 results per clock per SM): with every exponential on
-// that unit the softmax of two query tiles alone takes twice as long as their tensor-core work.
-constexpr uint32_t kPolyPairs = 0x52;   // pairs 1, 4, 6 of 8
+// others ex2.approx (special-function unit, 16 results per clock per SM: with every exponential there,
+// the softmax of two query tiles needs 2048 cycles against 1056 of tensor-core work).  The polynomial
+// costs about ten issue slots per pair against two, and the softmax warps are as short of issue slots as
+// of special-function throughput: measured at 10500 x 10500 x 16 heads, one pair in eight is the best
+// split (0/8: 574 us, 1/8: 540 us, 2/8: 557 us, 3/8: 587 us).
+constexpr uint32_t kPolyPairs = 0x10;   // pair 4 of 8
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
