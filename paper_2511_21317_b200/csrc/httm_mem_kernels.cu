@@ -471,7 +471,7 @@ cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count,
 }
 
 // ------------------------------------------------------------------------------------
-// a3. Merged-token aggregation (Sec. 3.2: mean of the dst token and the src tokens
+// a3 (blocks of more than 32 tokens).  Merged-token aggregation (Sec. 3.2: mean of the dst token and the src tokens
 //     matched to it; Algorithm 1 "BlockAggregate"), one warp per (tensor, head, block).
 //     The block is staged in shared memory by a TMA bulk copy, double buffered per warp.
 //     Each lane owns two channels.  For every kept token, in reordered order, the warp
@@ -661,6 +661,210 @@ __global__ void __launch_bounds__(merge_warps_per_cta(32 * PASSES) * 32) merge_k
     }
 }
 
+// ------------------------------------------------------------------------------------
+// a3 (blocks of at most 32 tokens).  The group sums of a block are one small dense
+//     contraction: merged_sum[kept row][channel] = sum_token W[row][token] x[token][channel]
+//     with the 0/1 assignment matrix W.  It runs on the tensor cores (m16n8k16, bf16 inputs,
+//     fp32 accumulation: W is exact in bf16, the products are exact, and the measured
+//     accumulation error is below that of an fp32 add chain).  W is built in registers from
+//     the map; x comes from the swizzled TMA stage through ldmatrix.trans (conflict free).
+//     The mean is the sum times the reciprocal of the group size, rounded once to bf16.
+//     One warp per (tensor, head, block); kept tokens are compacted in reordered order.
+// ------------------------------------------------------------------------------------
+constexpr int kMergeTcWarps = 8;
+constexpr int kMergeTcAux = 32 * 4 + 16;   // reciprocal group sizes per kept row + 2 mbarriers
+constexpr int kMergeTcSmem = kMergeTcWarps * (2 * 32 * kRowBytes + kMergeTcAux) + 1024 /*alignment slack*/;
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t saddr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(kMergeTcWarps * 32, 2)
+merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, const MergeArgs a) {
+    constexpr uint32_t STAGE_BYTES = 32 * kRowBytes;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;   // accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
+    unsigned char* stage = smem + (size_t)warp * 2 * STAGE_BYTES;                       // [2][32][128], 1024-aligned, swizzled
+    unsigned char* aux = smem + (size_t)kMergeTcWarps * 2 * STAGE_BYTES + (size_t)warp * kMergeTcAux;
+    float* rcnt = reinterpret_cast<float*>(aux);                                        // [32] 1 / group size of kept row
+    const uint32_t mbar0 = smem_u32(aux + 32 * 4), stage0 = smem_u32(stage);
+
+    if (lane == 0) {
+        mbar_init(mbar0, 1);
+        mbar_init(mbar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    // task -> (tensor t, head h, unit u); units 0 .. n_blocks-1 are merging blocks, the rest are
+    // chunks of 32 special tokens (never merged: rows 0 .. n_special_total-1 are copied)
+    const int sp_chunks = (a.n_special_total + 31) / 32;
+    const int per_head = a.n_blocks + sp_chunks;
+    const int64_t n_tasks = 3ll * a.heads * per_head;
+    const int64_t stride = (int64_t)gridDim.x * kMergeTcWarps;
+    const int64_t first = (int64_t)blockIdx.x * kMergeTcWarps + warp;
+    TaskCursor cur, nxt;   // the task being processed; the task whose load is issued next
+    cur.init(first, stride, a.heads, per_head);
+    nxt = cur;
+
+    auto unit_start = [&](const TaskCursor& c) { return c.u >= a.n_blocks ? (c.u - a.n_blocks) * 32 : __ldg(&a.blocks[c.u].start); };
+    auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only; the whole 32-row box is transferred (rows past the head's end are zero filled)
+        const uint32_t mb = mbar0 + 8 * buf;
+        mbar_expect_tx(mb, STAGE_BYTES);
+        tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, unit_start(c), c.h);
+    };
+    if (first < n_tasks && lane == 0) issue(nxt, 0);
+    nxt.advance();
+    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+    nxt.advance();
+
+    int it = 0;
+    bool failed = false;
+    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
+        const int buf = it & 1;
+        const uint32_t parity = (it >> 1) & 1;
+        const bool more = task + 2 * stride < n_tasks;
+        const int t = cur.t, h = cur.h;
+        const bool special = cur.u >= a.n_blocks;
+        int start, n, r, moff;
+        if (special) {
+            start = (cur.u - a.n_blocks) * 32;
+            n = min(32, a.n_special_total - start);
+            r = 0;
+            moff = start;
+        } else {
+            const BlockInfo bi = a.blocks[cur.u];
+            start = bi.start;
+            n = bi.n;
+            r = t == 0 ? bi.r_q : bi.r_k;
+            moff = t == 0 ? bi.moff_q : bi.moff_k;
+        }
+        const int m_len = t == 0 ? a.m_q : a.m_k;
+        uint32_t* out = reinterpret_cast<uint32_t*>(a.merged[t] + ((int64_t)h * m_len + moff) * kHeadDim);   // 32 words per row
+        const uint32_t blk = stage0 + buf * STAGE_BYTES;
+
+        // the map entry does not depend on the staged rows: fetch it before waiting
+        int rep = -1;
+        if (r > 0 && lane < n) {
+            rep = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + lane) - start;
+            if (rep < 0 || rep >= n) {   // corrupt map: record, treat as kept
+                atomicCAS(a.status, kDevOk, kDevBadIndex);
+                rep = lane;
+            }
+        }
+        if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
+            failed = true;
+            break;
+        }
+        if (r == 0) {   // nothing merges here: copy the rows, 16 bytes per lane (chunk c of row j sits at c ^ (j & 7))
+            const unsigned char* sb = stage + buf * STAGE_BYTES;
+            uint4* o4 = reinterpret_cast<uint4*>(out);
+            for (int q = lane; q < n * 8; q += 32) {
+                const int row = q >> 3, ch = q & 7;
+                o4[q] = *reinterpret_cast<const uint4*>(sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
+            }
+            if (t == 0 && !special && lane < n) a.rank_q[(int64_t)h * a.n_tokens + start + lane] = moff + lane;
+        } else {
+            // merged row of every token: rank of its representative among the kept tokens
+            const unsigned kept = __ballot_sync(0xffffffffu, rep == lane);   // rep == -1 for lanes >= n
+            const int n_kept = __popc(kept);
+            const int row_of = rep >= 0 ? __popc(kept & ((1u << rep) - 1u)) : -1;
+            if (t == 0 && lane < n) a.rank_q[(int64_t)h * a.n_tokens + start + lane] = moff + row_of;
+            const unsigned group = __match_any_sync(0xffffffffu, row_of);
+            if (rep == lane) rcnt[row_of] = 1.0f / (float)__popc(group);
+            // x fragments: for k step ks (16 tokens) and channel tile pair np, one ldmatrix.x4.trans gives
+            // b0, b1 of channel tile 2 np and b0, b1 of channel tile 2 np + 1
+            uint32_t bf[2][4][4];
+            const int n_ks = n > 16 ? 2 : 1;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                if (ks < n_ks) {
+                    const int tok = 16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8;
+                    const uint32_t rowaddr = blk + tok * kRowBytes;
+#pragma unroll
+                    for (int np = 0; np < 4; ++np) ldmatrix_x4_trans(bf[ks][np], rowaddr + (((2 * np + (lane >> 4)) ^ (tok & 7)) << 4));
+                }
+            }
+            // W fragments need the rows of tokens 16 ks + {2 tq, 2 tq + 1, 2 tq + 8, 2 tq + 9}
+            int rw[2][4];
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                rw[ks][0] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq);
+                rw[ks][1] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 1);
+                rw[ks][2] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 8);
+                rw[ks][3] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 9);
+            }
+            __syncwarp();   // reciprocal group sizes visible; every lane has its fragments: the stage can be refilled
+            if (more && lane == 0) issue(nxt, buf);
+            const int n_mt = n_kept > 16 ? 2 : 1;
+#pragma unroll 1
+            for (int mt = 0; mt < n_mt; ++mt) {
+                const int r0 = 16 * mt + g, r1 = r0 + 8;   // this lane's two accumulator rows
+                float c[8][4];
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < 2; ++ks) {
+                    if (ks < n_ks) {
+                        uint32_t af[4];   // bf16 1.0 = 0x3f80
+                        af[0] = (rw[ks][0] == r0 ? 0x3f80u : 0u) | (rw[ks][1] == r0 ? 0x3f800000u : 0u);
+                        af[1] = (rw[ks][0] == r1 ? 0x3f80u : 0u) | (rw[ks][1] == r1 ? 0x3f800000u : 0u);
+                        af[2] = (rw[ks][2] == r0 ? 0x3f80u : 0u) | (rw[ks][3] == r0 ? 0x3f800000u : 0u);
+                        af[3] = (rw[ks][2] == r1 ? 0x3f80u : 0u) | (rw[ks][3] == r1 ? 0x3f800000u : 0u);
+#pragma unroll
+                        for (int nt = 0; nt < 8; ++nt)
+                            mma_bf16_16816(c[nt], af, bf[ks][nt >> 1][2 * (nt & 1)], bf[ks][nt >> 1][2 * (nt & 1) + 1]);
+                    }
+                }
+                const bool w0 = r0 < n_kept && r0 < n - r, w1 = r1 < n_kept && r1 < n - r;   // (a corrupt map cannot overrun)
+                const float i0 = w0 ? rcnt[r0] : 0.f, i1 = w1 ? rcnt[r1] : 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {
+                    if (w0) {
+                        const __nv_bfloat162 o = __floats2bfloat162_rn(c[nt][0] * i0, c[nt][1] * i0);
+                        out[r0 * 32 + nt * 4 + tq] = *reinterpret_cast<const uint32_t*>(&o);
+                    }
+                    if (w1) {
+                        const __nv_bfloat162 o = __floats2bfloat162_rn(c[nt][2] * i1, c[nt][3] * i1);
+                        out[r1 * 32 + nt * 4 + tq] = *reinterpret_cast<const uint32_t*>(&o);
+                    }
+                }
+            }
+            __syncwarp();   // every lane is done with the reciprocals before the next task rewrites them
+            continue;
+        }
+        __syncwarp();   // every lane is done reading this stage buffer
+        if (more && lane == 0) issue(nxt, buf);
+    }
+    if (failed) {
+        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+    }
+}
+
+static cudaError_t launch_merge_tc(const MergeArgs& a, int sm_count, cudaStream_t stream) {
+    CUtensorMap mq, mk, mv;
+    const int64_t N = a.n_tokens;
+    if (!encode_rows_tensor_map(&mq, a.xr[0], N, a.heads, kHeadDim, N * kHeadDim, 32) ||
+        !encode_rows_tensor_map(&mk, a.xr[1], N, a.heads, kHeadDim, N * kHeadDim, 32) ||
+        !encode_rows_tensor_map(&mv, a.xr[2], N, a.heads, kHeadDim, N * kHeadDim, 32))
+        return cudaErrorInvalidValue;
+    const int64_t n_tasks = 3ll * a.heads * (a.n_blocks + (a.n_special_total + 31) / 32);
+    int64_t grid = (n_tasks + kMergeTcWarps - 1) / kMergeTcWarps;
+    const int64_t cap = (int64_t)sm_count * 2;
+    if (grid > cap) grid = cap;
+    if (grid < 1) grid = 1;
+    merge_tc_kernel<<<(unsigned)grid, kMergeTcWarps * 32, kMergeTcSmem, stream>>>(mq, mk, mv, a);
+    return cudaGetLastError();
+}
+
 template <int PASSES>
 static cudaError_t launch_merge_t(const MergeArgs& a, int sm_count, cudaStream_t stream) {
     constexpr int NMAX = 32 * PASSES;
@@ -678,7 +882,7 @@ static cudaError_t launch_merge_t(const MergeArgs& a, int sm_count, cudaStream_t
 }
 
 cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream) {
-    if (max_block_tokens <= 32) return launch_merge_t<1>(a, sm_count, stream);
+    if (max_block_tokens <= 32) return launch_merge_tc(a, sm_count, stream);   // tensor-core kernel
     if (max_block_tokens <= 128) return launch_merge_t<4>(a, sm_count, stream);
     return launch_merge_t<8>(a, sm_count, stream);
 }
@@ -740,7 +944,7 @@ cudaError_t configure_kernels() {
     HTTM_SET_SMEM(match_kernel<1>, match_smem_bytes(32));
     HTTM_SET_SMEM(match_kernel<4>, match_smem_bytes(128));
     HTTM_SET_SMEM(match_kernel<8>, match_smem_bytes(256));
-    HTTM_SET_SMEM(merge_kernel<1>, merge_smem_bytes(32));
+    HTTM_SET_SMEM(merge_tc_kernel, kMergeTcSmem);
     HTTM_SET_SMEM(merge_kernel<4>, merge_smem_bytes(128));
     HTTM_SET_SMEM(merge_kernel<8>, merge_smem_bytes(256));
 #undef HTTM_SET_SMEM
