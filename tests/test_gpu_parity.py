@@ -210,3 +210,31 @@ def test_small_config_full_size_sampled():
     toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 64), np.arange(5), [wl.n_tokens - 1]]))
     stats = run_case(wl, sample=toks)
     assert stats["merged_exactly_rounded"] > 0.99
+
+
+def test_medium_config_full_size_sampled():
+    """The benchmark's workload at full size (33k tokens, 16 heads), in the launch configuration the benchmark
+    times: permutation, reordered tensors, maps, rank and merged tensors in full; attention on sampled tokens;
+    unmerge as a pure copy on every token."""
+    wl = synth.WORKLOADS["medium"]
+    rng = np.random.default_rng(2)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 48), np.arange(5), [wl.n_tokens - 1]]))
+    stats = run_case(wl, sample=toks)
+    assert stats["merged_exactly_rounded"] > 0.99
+
+
+def test_dense_attention_medium_config_sampled():
+    """The dense in-run reference at the benchmark's size, on sampled tokens."""
+    wl = synth.WORKLOADS["medium"]
+    q, k, v = synth.make_qkv(wl)
+    g = orc.Geometry.of(wl)
+    rng = np.random.default_rng(3)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 24), [0, 4, 5, wl.n_tokens - 1, 32768, 32767]]))
+    ref = orc.dense_attention(g, q, k, v, toks)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        out = ctx.dense_attention(*(hb.bf16_from_bits(x, DEV) for x in (q, k, v)))
+        torch.cuda.synchronize()
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        bits = hb.bits_from_bf16(out)
+        assert np.isfinite(parity.bits_to_f64(bits)).all()
+        parity.check_output(bits[toks], ref, what="dense medium")
