@@ -30,7 +30,7 @@ constexpr int KV_STAGES = 3;
 constexpr int TILE_BYTES = BM * kRowBytes;   // 16 KB
 constexpr int NTHREADS = 320;   // producer warp, MMA warp, 2 x 4 softmax warps: registers are granted per four warps, so 168 per thread as with twelve
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row exchange*/;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
 struct Barriers {
@@ -40,6 +40,7 @@ struct Barriers {
     uint64_t s_full[3], p_full[3];   // per score buffer
     uint64_t o_done[2];              // per query tile: one completion per P V
     uint64_t o_final;
+    uint64_t x_full, x_done;         // single pass: tile B's (max, sum) published / tile A done reading O_B
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -50,6 +51,7 @@ struct TcParams {
     int32_t m_q, m_k;
     float scale_log2;
     int32_t* status;
+    int32_t tiles_per_head, total_tiles, chunk;   // query tiles per head, in all heads, per CTA
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -88,6 +90,34 @@ __device__ __forceinline__ float2 exp2_poly2(float2 t) {
 // split (0/8: 574 us, 1/8: 540 us, 2/8: 557 us, 3/8: 587 us).
 constexpr uint32_t kPolyPairs = 0x10;   // pair 4 of 8
 
+// Work decomposition.  The query tiles of all heads form one list (head-major); CTA c of G takes the
+// contiguous chunk [c L, (c + 1) L) of it and walks it in PASSES: two consecutive tiles of the same head as
+// a pair pass (tiles A and B share the K/V stream), a left-over tile as a single pass: the same machinery
+// with ONE query tile whose even key tiles go to softmax group A / accumulator O_A and odd ones to group B /
+// O_B (two partial softmaxes over disjoint keys), combined in the epilogue.  Either way score tile k is
+// handled by group k mod 2 in buffer k mod 3.  With one CTA per SM the SMs finish within one tile of each other,
+// whereas a grid of 672 two-tile CTAs on 148 SMs runs 4.54 waves as 5.
+struct Pass {
+    int head, tile;   // tile = index of query tile A inside the head
+    bool pair;
+};
+struct PassWalker {
+    int t, t_end, tiles_per_head;
+    __device__ PassWalker(int chunk, int total, int tph) : t(blockIdx.x * chunk), t_end(min(total, (int)(blockIdx.x + 1) * chunk)), tiles_per_head(tph) {}
+    __device__ bool next(Pass* ps) {
+        if (t >= t_end) return false;
+        ps->head = t / tiles_per_head;
+        ps->tile = t - ps->head * tiles_per_head;
+        ps->pair = t + 1 < t_end && ps->tile + 1 < tiles_per_head;
+        t += ps->pair ? 2 : 1;
+        return true;
+    }
+};
+// Completions a pass adds to each barrier family, so that every role can carry the phase parities from
+// pass to pass: stage st of the K/V ring completes once per key tile j with j mod 3 == st; score buffer b
+// once per score tile k with k mod 3 == b (2 n tiles in a pair pass, n in a single pass).
+__device__ __forceinline__ int count_mod3(int n, int r) { return (n - r + 2) / 3; }
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const TcParams p) {
@@ -100,9 +130,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     volatile int* abort_flag = &bars->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int head = blockIdx.y;
-    const int q0 = blockIdx.x * (2 * BM);
     const int n_tiles = (p.m_k + BN - 1) / BN;
+    const int kv_cnt[3] = {count_mod3(n_tiles, 0), count_mod3(n_tiles, 1), count_mod3(n_tiles, 2)};   // per pass
 
     if (tid == 0) {
         bars->abort_flag = 0;
@@ -120,6 +149,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc::mbar_init(tc::smem_addr(&bars->o_done[0]), 1);
         tc::mbar_init(tc::smem_addr(&bars->o_done[1]), 1);
         tc::mbar_init(tc::smem_addr(&bars->o_final), 1);
+        tc::mbar_init(tc::smem_addr(&bars->x_full), 128);
+        tc::mbar_init(tc::smem_addr(&bars->x_done), 128);
         tc::fence_barrier_init();
         tc::prefetch_tensormap(&map_q);
         tc::prefetch_tensormap(&map_k);
@@ -131,35 +162,43 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
     // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the first 64 columns of its S
+    PassWalker walker(p.chunk, p.total_tiles, p.tiles_per_head);
+    Pass ps;
 
-    // Register budget: the softmax threads hold a whole 128-wide row of S; with ten warps every thread
-    // has 168 registers from launch, so no register reallocation between the roles is needed.  A warp
-    // reaches the 32 TMEM lanes 32 * (warp % 4) ..: any four consecutive warps cover a 128-row tile.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (tc::elect_one()) {
-            const uint32_t qb = tc::smem_addr(&bars->q_full);
-            tc::mbar_expect_tx(qb, 2 * TILE_BYTES);
-            tc::tma_load_3d(s_q, &map_q, qb, 0, q0, head);
-            tc::tma_load_3d(s_q + TILE_BYTES, &map_q, qb, 0, q0 + BM, head);
-            for (int j = 0; j < n_tiles; ++j) {
-                const int st = j % KV_STAGES;
-                const uint32_t ph = (uint32_t)(j / KV_STAGES) & 1u;
-                if (j >= KV_STAGES && !tc::mbar_wait(tc::smem_addr(&bars->k_empty[st]), ph ^ 1u, abort_flag)) break;
-                const uint32_t kb = tc::smem_addr(&bars->k_full[st]);
-                tc::mbar_expect_tx(kb, TILE_BYTES);
-                tc::tma_load_3d(s_k + st * TILE_BYTES, &map_k, kb, 0, j * BN, head);
-                if (j >= KV_STAGES && !tc::mbar_wait(tc::smem_addr(&bars->v_empty[st]), ph ^ 1u, abort_flag)) break;
-                const uint32_t vb = tc::smem_addr(&bars->v_full[st]);
-                tc::mbar_expect_tx(vb, TILE_BYTES);
-                tc::tma_load_3d(s_v + st * TILE_BYTES, &map_v, vb, 0, j * BN, head);
+            uint32_t kv_base[3] = {0, 0, 0};   // completions of each ring stage before this pass (parity bit)
+            for (int pass = 0; walker.next(&ps); ++pass) {
+                // the previous pass's MMAs read Q and the ring: all of them are complete at o_final
+                if (pass > 0 && !tc::mbar_wait(tc::smem_addr(&bars->o_final), (uint32_t)(pass - 1) & 1u, abort_flag)) break;
+                const uint32_t qb = tc::smem_addr(&bars->q_full);
+                tc::mbar_expect_tx(qb, ps.pair ? 2 * TILE_BYTES : TILE_BYTES);
+                tc::tma_load_3d(s_q, &map_q, qb, 0, ps.tile * BM, ps.head);
+                if (ps.pair) tc::tma_load_3d(s_q + TILE_BYTES, &map_q, qb, 0, (ps.tile + 1) * BM, ps.head);
+                bool ok = true;
+                for (int j = 0; j < n_tiles; ++j) {
+                    const int st = j % KV_STAGES;
+                    const uint32_t par = (kv_base[st] + (uint32_t)(j / KV_STAGES)) & 1u;   // completion index of tile j in stage st
+                    if (j >= KV_STAGES && !(ok = tc::mbar_wait(tc::smem_addr(&bars->k_empty[st]), par ^ 1u, abort_flag))) break;
+                    const uint32_t kb = tc::smem_addr(&bars->k_full[st]);
+                    tc::mbar_expect_tx(kb, TILE_BYTES);
+                    tc::tma_load_3d(s_k + st * TILE_BYTES, &map_k, kb, 0, j * BN, ps.head);
+                    if (j >= KV_STAGES && !(ok = tc::mbar_wait(tc::smem_addr(&bars->v_empty[st]), par ^ 1u, abort_flag))) break;
+                    const uint32_t vb = tc::smem_addr(&bars->v_full[st]);
+                    tc::mbar_expect_tx(vb, TILE_BYTES);
+                    tc::tma_load_3d(s_v + st * TILE_BYTES, &map_v, vb, 0, j * BN, ps.head);
+                }
+                if (!ok) break;
+#pragma unroll
+                for (int st = 0; st < 3; ++st) kv_base[st] += (uint32_t)kv_cnt[st];
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // Every operand of a tcgen05.mma below is a loop-invariant base plus a compile-time offset (the
-        // ring stage is a template constant, the loop is unrolled over the three stages): operands that
+        // Every operand of a tcgen05.mma below is a loop-invariant base plus a compile-time offset (score
+        // buffer, query tile and ring stage are template constants of the unrolled steps): operands that
         // are recomputed per instruction at run time make the issue itself cost more than the MMA.
         if (tc::elect_one()) {
             constexpr uint32_t idesc_qk = tc::idesc_bf16(BM, BN, false, false);
@@ -167,7 +206,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const uint64_t dq0 = tc::smem_desc_sw128(s_q);
             const uint64_t dk0 = tc::smem_desc_sw128(s_k), dv0 = tc::smem_desc_sw128(s_v);
             constexpr uint64_t kStageStep = TILE_BYTES >> 4;   // descriptor address field counts 16-byte units
-            const int n_score = 2 * n_tiles;                   // score tiles k = 2 j + x
             // S(buffer) = Q_x K(stage)^T: four K=16 steps, 32 bytes apart inside the 128-byte rows
             auto issue_qk = [&](uint32_t t_s, uint64_t dq, uint64_t dk, uint32_t bar) {
                 tc::mma_ss_c<false>(t_s, dq, dk, idesc_qk);
@@ -182,22 +220,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
                 for (int k = 0; k < 8; ++k) tc::mma_ts_c<true>(t_o, t_p + 8 * k, dv + (uint64_t)(k * 128), idesc_pv);
             };
-            // Score tile k = k0 + C with k0 a multiple of 6: buffer, query tile and ring stages are compile-time.
-            // round_par = parity of k0 / 6.  Returns false when a wait gave up.
-            auto step = [&](auto c_c, int k0, uint32_t round_par) -> bool {
+            uint32_t kv_base[3] = {0, 0, 0}, sp_base[3] = {0, 0, 0};   // completions before this pass: ring stages, score buffers
+            // PAIR pass, score tile k = k0 + C with k0 a multiple of 6 (round_par = parity of k0 / 6).
+            auto step_pair = [&](auto c_c, int k0, uint32_t round_par, int n_score) -> bool {
                 constexpr int C = decltype(c_c)::value;
                 constexpr int B = C % 3, X = C % 2, ST = (C >> 1) % KV_STAGES;                 // this tile: P(k) V
                 constexpr int X3 = 1 - X, J3 = (C + 3) >> 1, ST3 = J3 % KV_STAGES;            // tile k + 3: next S in the same buffer
                 const uint32_t t_buf = tmem + B * BN, t_o = tmem + 3 * BN + X * kHeadDim;
-                if (X == 0 && !tc::mbar_wait(tc::smem_addr(&bars->v_full[ST]), round_par, abort_flag)) return false;
-                if (!tc::mbar_wait(tc::smem_addr(&bars->p_full[B]), (C / 3) & 1, abort_flag)) return false;
+                if (X == 0 && !tc::mbar_wait(tc::smem_addr(&bars->v_full[ST]), (kv_base[ST] + round_par) & 1u, abort_flag)) return false;
+                if (!tc::mbar_wait(tc::smem_addr(&bars->p_full[B]), (sp_base[B] + (C / 3)) & 1u, abort_flag)) return false;
                 tc::fence_after_sync();
                 issue_pv(t_o, t_buf, dv0 + ST * kStageStep);
                 tc::mma_commit(tc::smem_addr(&bars->o_done[X]));
                 if (X == 1) tc::mma_commit(tc::smem_addr(&bars->v_empty[ST]));
                 if (k0 + C + 3 < n_score) {
                     if (X3 == 0) {
-                        if (!tc::mbar_wait(tc::smem_addr(&bars->k_full[ST3]), round_par ^ (J3 >= 3 ? 1u : 0u), abort_flag)) return false;
+                        if (!tc::mbar_wait(tc::smem_addr(&bars->k_full[ST3]), (kv_base[ST3] + round_par + (J3 >= 3 ? 1u : 0u)) & 1u, abort_flag)) return false;
                         tc::fence_after_sync();
                     }
                     issue_qk(t_buf, dq0 + X3 * kStageStep, dk0 + ST3 * kStageStep, tc::smem_addr(&bars->s_full[B]));
@@ -205,32 +243,87 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
                 return true;
             };
-            static_assert(KV_STAGES == 3, "the issue loop is unrolled over 6 = lcm(3 score buffers, 2 query tiles, 3 ring stages) / ... score tiles");
-            bool ok = tc::mbar_wait(tc::smem_addr(&bars->q_full), 0, abort_flag) &&
-                      tc::mbar_wait(tc::smem_addr(&bars->k_full[0]), 0, abort_flag);
-            if (ok) {   // prologue: S(0), S(1) from key tile 0, S(2) from key tile 1
+            // SINGLE pass, score tile k = key tile k = k0 + C with k0 a multiple of 6: buffer and ring stage k mod 3,
+            // softmax group and accumulator k mod 2.
+            auto step_single = [&](auto c_c, int k0) -> bool {
+                constexpr int C = decltype(c_c)::value;
+                constexpr int B = C % 3, X = C % 2;
+                constexpr uint32_t IDX = C / 3;   // completion index of this tile in its buffer / stage, modulo 2 (k0 / 3 is even)
+                const uint32_t t_buf = tmem + B * BN, t_o = tmem + 3 * BN + X * kHeadDim;
+                if (!tc::mbar_wait(tc::smem_addr(&bars->v_full[B]), (kv_base[B] + IDX) & 1u, abort_flag)) return false;
+                if (!tc::mbar_wait(tc::smem_addr(&bars->p_full[B]), (sp_base[B] + IDX) & 1u, abort_flag)) return false;
                 tc::fence_after_sync();
-                issue_qk(tmem, dq0, dk0, tc::smem_addr(&bars->s_full[0]));
-                issue_qk(tmem + BN, dq0 + kStageStep, dk0, tc::smem_addr(&bars->s_full[1]));
-                tc::mma_commit(tc::smem_addr(&bars->k_empty[0]));
-                if (n_score > 2) {
-                    ok = tc::mbar_wait(tc::smem_addr(&bars->k_full[1]), 0, abort_flag);
-                    if (ok) {
+                issue_pv(t_o, t_buf, dv0 + B * kStageStep);
+                tc::mma_commit(tc::smem_addr(&bars->o_done[X]));
+                tc::mma_commit(tc::smem_addr(&bars->v_empty[B]));
+                if (k0 + C + 3 < n_tiles) {
+                    if (!tc::mbar_wait(tc::smem_addr(&bars->k_full[B]), (kv_base[B] + IDX + 1u) & 1u, abort_flag)) return false;
+                    tc::fence_after_sync();
+                    issue_qk(t_buf, dq0, dk0 + B * kStageStep, tc::smem_addr(&bars->s_full[B]));
+                    tc::mma_commit(tc::smem_addr(&bars->k_empty[B]));
+                }
+                return true;
+            };
+            static_assert(KV_STAGES == 3, "the issue loops are unrolled over three ring stages and three score buffers");
+            bool ok = true;
+            for (int pass = 0; ok && walker.next(&ps); ++pass) {
+                ok = tc::mbar_wait(tc::smem_addr(&bars->q_full), (uint32_t)pass & 1u, abort_flag) &&
+                     tc::mbar_wait(tc::smem_addr(&bars->k_full[0]), kv_base[0] & 1u, abort_flag);
+                if (!ok) break;
+                tc::fence_after_sync();
+                if (ps.pair) {
+                    const int n_score = 2 * n_tiles;   // score tiles k = 2 j + x
+                    // prologue: S(0), S(1) from key tile 0, S(2) from key tile 1
+                    issue_qk(tmem, dq0, dk0, tc::smem_addr(&bars->s_full[0]));
+                    issue_qk(tmem + BN, dq0 + kStageStep, dk0, tc::smem_addr(&bars->s_full[1]));
+                    tc::mma_commit(tc::smem_addr(&bars->k_empty[0]));
+                    if (n_score > 2) {
+                        if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->k_full[1]), kv_base[1] & 1u, abort_flag))) break;
                         tc::fence_after_sync();
                         issue_qk(tmem + 2 * BN, dq0, dk0 + kStageStep, tc::smem_addr(&bars->s_full[2]));
                     }
+                    uint32_t round_par = 0;
+                    for (int k0 = 0; ok && k0 < n_score; k0 += 6, round_par ^= 1u) {
+                        ok = step_pair(std::integral_constant<int, 0>{}, k0, round_par, n_score);
+                        if (ok) ok = step_pair(std::integral_constant<int, 1>{}, k0, round_par, n_score);   // n_score is even
+                        if (ok && k0 + 2 < n_score) ok = step_pair(std::integral_constant<int, 2>{}, k0, round_par, n_score);
+                        if (ok && k0 + 2 < n_score) ok = step_pair(std::integral_constant<int, 3>{}, k0, round_par, n_score);
+                        if (ok && k0 + 4 < n_score) ok = step_pair(std::integral_constant<int, 4>{}, k0, round_par, n_score);
+                        if (ok && k0 + 4 < n_score) ok = step_pair(std::integral_constant<int, 5>{}, k0, round_par, n_score);
+                    }
+#pragma unroll
+                    for (int b = 0; b < 3; ++b) sp_base[b] += (uint32_t)count_mod3(n_score, b);
+                } else {
+                    // prologue: S(0), S(1), S(2) from key tiles 0, 1, 2
+                    issue_qk(tmem, dq0, dk0, tc::smem_addr(&bars->s_full[0]));
+                    tc::mma_commit(tc::smem_addr(&bars->k_empty[0]));
+                    if (n_tiles > 1) {
+                        if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->k_full[1]), kv_base[1] & 1u, abort_flag))) break;
+                        tc::fence_after_sync();
+                        issue_qk(tmem + BN, dq0, dk0 + kStageStep, tc::smem_addr(&bars->s_full[1]));
+                        tc::mma_commit(tc::smem_addr(&bars->k_empty[1]));
+                    }
+                    if (n_tiles > 2) {
+                        if (!(ok = tc::mbar_wait(tc::smem_addr(&bars->k_full[2]), kv_base[2] & 1u, abort_flag))) break;
+                        tc::fence_after_sync();
+                        issue_qk(tmem + 2 * BN, dq0, dk0 + 2 * kStageStep, tc::smem_addr(&bars->s_full[2]));
+                        tc::mma_commit(tc::smem_addr(&bars->k_empty[2]));
+                    }
+                    for (int k0 = 0; ok && k0 < n_tiles; k0 += 6) {
+                        ok = step_single(std::integral_constant<int, 0>{}, k0);
+                        if (ok && k0 + 1 < n_tiles) ok = step_single(std::integral_constant<int, 1>{}, k0);
+                        if (ok && k0 + 2 < n_tiles) ok = step_single(std::integral_constant<int, 2>{}, k0);
+                        if (ok && k0 + 3 < n_tiles) ok = step_single(std::integral_constant<int, 3>{}, k0);
+                        if (ok && k0 + 4 < n_tiles) ok = step_single(std::integral_constant<int, 4>{}, k0);
+                        if (ok && k0 + 5 < n_tiles) ok = step_single(std::integral_constant<int, 5>{}, k0);
+                    }
+#pragma unroll
+                    for (int b = 0; b < 3; ++b) sp_base[b] += (uint32_t)count_mod3(n_tiles, b);
                 }
+                if (ok) tc::mma_commit(tc::smem_addr(&bars->o_final));
+#pragma unroll
+                for (int st = 0; st < 3; ++st) kv_base[st] += (uint32_t)kv_cnt[st];
             }
-            uint32_t round_par = 0;
-            for (int k0 = 0; ok && k0 < n_score; k0 += 6, round_par ^= 1u) {
-                ok = step(std::integral_constant<int, 0>{}, k0, round_par);
-                if (ok) ok = step(std::integral_constant<int, 1>{}, k0, round_par);          // n_score is even
-                if (ok && k0 + 2 < n_score) ok = step(std::integral_constant<int, 2>{}, k0, round_par);
-                if (ok && k0 + 2 < n_score) ok = step(std::integral_constant<int, 3>{}, k0, round_par);
-                if (ok && k0 + 4 < n_score) ok = step(std::integral_constant<int, 4>{}, k0, round_par);
-                if (ok && k0 + 4 < n_score) ok = step(std::integral_constant<int, 5>{}, k0, round_par);
-            }
-            if (ok) tc::mma_commit(tc::smem_addr(&bars->o_final));
         }
         __syncwarp();
     } else {
@@ -241,108 +334,164 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t t_o = tmem + 3 * BN + x * kHeadDim + lane_addr;
         const uint32_t obar = tc::smem_addr(&bars->o_done[x]);
         const float c = p.scale_log2;
-        float m = -INFINITY, l = 0.f;
+        uint32_t sp_base[3] = {0, 0, 0}, od_base = 0;   // completions before this pass: score buffers, this group's P V
+        uint32_t n_single = 0;                          // single passes so far (phase of x_full / x_done)
+        float2* xch = reinterpret_cast<float2*>(smem + (2 + 2 * KV_STAGES) * TILE_BYTES + 256);   // [128 rows] (max, sum) of group B
         bool ok = true;
-        {   // the accumulator O starts at zero: every PV step accumulates (ordered before the first p_full arrival)
-            uint32_t z[32];
+        for (int pass = 0; ok && walker.next(&ps); ++pass) {
+            const int n_score = ps.pair ? 2 * n_tiles : n_tiles;
+            // this group's score tiles are k = 2 i + x; in a pair pass they come from key tile i, in a single pass from key tile k
+            const int n_own = ps.pair ? n_tiles : (n_tiles - x + 1) / 2;
+            {
+                float m = -INFINITY, l = 0.f;
+                {   // the accumulator O starts at zero: every PV step accumulates (ordered before the first p_full arrival)
+                    uint32_t z[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) z[i] = 0u;
-            tc::tmem_st32(t_o, z);
-            tc::tmem_st32(t_o + 32, z);
-        }
-        for (int j = 0; j < n_tiles; ++j) {
-            const int k = 2 * j + x, buf = k % 3;                      // score tile and its buffer
-            const uint32_t kpar = (uint32_t)(k / 3) & 1u;
-            const uint32_t t_s = tmem + buf * BN + lane_addr;
-            const uint32_t sbar = tc::smem_addr(&bars->s_full[buf]), pbar = tc::smem_addr(&bars->p_full[buf]);
-            if (!(ok = tc::mbar_wait(sbar, kpar, abort_flag))) break;
-            tc::fence_after_sync();
-            uint32_t s[BN];   // fp32 bit patterns of this row of S
+                    for (int i = 0; i < 32; ++i) z[i] = 0u;
+                    tc::tmem_st32(t_o, z);
+                    tc::tmem_st32(t_o + 32, z);
+                    if (n_own == 0) tc::tmem_wait_st();
+                }
+                for (int j = 0; j < n_own; ++j) {
+                    const int k = 2 * j + x, buf = k % 3;                      // score tile and its buffer
+                    const int key_tile = ps.pair ? j : k;
+                    const uint32_t kpar = (sp_base[buf] + (uint32_t)(k / 3)) & 1u;
+                    const uint32_t t_s = tmem + buf * BN + lane_addr;
+                    const uint32_t sbar = tc::smem_addr(&bars->s_full[buf]), pbar = tc::smem_addr(&bars->p_full[buf]);
+                    if (!(ok = tc::mbar_wait(sbar, kpar, abort_flag))) break;
+                    tc::fence_after_sync();
+                    uint32_t s[BN];   // fp32 bit patterns of this row of S
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(t_s + cc * 32, s + cc * 32);
-            tc::tmem_wait_ld();
-            const int valid = p.m_k - j * BN;
-            if (valid < BN) {
-#pragma unroll
-                for (int i = 0; i < BN; ++i)
-                    if (i >= valid) s[i] = 0xff800000u;   // -inf: keys past the end
-            }
-            // row maximum: four independent chains of three-input maxima
-            float mx4[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                mx4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
-#pragma unroll
-                for (int i = 2; i < 32; i += 2)
-                    mx4[q] = tc::fmax3(mx4[q], __uint_as_float(s[32 * q + i]), __uint_as_float(s[32 * q + i + 1]));
-            }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            const float m_new = fmaxf(m, mx * c);
-            if (j == 0) {
-                m = m_new;
-            } else if (__any_sync(0xffffffffu, m_new - m > kRescaleThreshold)) {
-                // raise the running maximum: rescale the row sum and the accumulator O in place, once the
-                // previous P V of this query tile has completed (the next one is issued after this tile's P)
-                if (!(ok = tc::mbar_wait(obar, (uint32_t)(j - 1) & 1u, abort_flag))) break;
-                tc::fence_after_sync();
-                const float f = exp2f(m - m_new);
-                l *= f;
-                m = m_new;
-#pragma unroll 1
-                for (int cc = 0; cc < 8; ++cc) {   // eight columns at a time: this rare path must not cost registers
-                    uint32_t o[8];
-                    tc::tmem_ld8(t_o + cc * 8, o);
+                    for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(t_s + cc * 32, s + cc * 32);
                     tc::tmem_wait_ld();
+                    const int valid = p.m_k - key_tile * BN;
+                    if (valid < BN) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                    tc::tmem_st8(t_o + cc * 8, o);
+                        for (int i = 0; i < BN; ++i)
+                            if (i >= valid) s[i] = 0xff800000u;   // -inf: keys past the end
+                    }
+                    // row maximum: four independent chains of three-input maxima
+                    float mx4[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        mx4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
+#pragma unroll
+                        for (int i = 2; i < 32; i += 2)
+                            mx4[q] = tc::fmax3(mx4[q], __uint_as_float(s[32 * q + i]), __uint_as_float(s[32 * q + i + 1]));
+                    }
+                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    const float m_new = fmaxf(m, mx * c);
+                    if (j == 0) {
+                        m = m_new;
+                    } else if (__any_sync(0xffffffffu, m_new - m > kRescaleThreshold)) {
+                        // raise the running maximum: rescale the row sum and the accumulator O in place, once the
+                        // previous P V of this query tile has completed (the next one is issued after this tile's P)
+                        if (!(ok = tc::mbar_wait(obar, (od_base + (uint32_t)(j - 1)) & 1u, abort_flag))) break;
+                        tc::fence_after_sync();
+                        const float f = exp2f(m - m_new);
+                        l *= f;
+                        m = m_new;
+#pragma unroll 1
+                        for (int cc = 0; cc < 8; ++cc) {   // eight columns at a time: this rare path must not cost registers
+                            uint32_t o[8];
+                            tc::tmem_ld8(t_o + cc * 8, o);
+                            tc::tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                            tc::tmem_st8(t_o + cc * 8, o);
+                        }
+                    }
+                    const float2 c2 = make_float2(c, c), neg_m2 = make_float2(-m, -m);
+                    float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0;
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float2 t = tc::ffma2(make_float2(__uint_as_float(s[cc * 16 + 2 * i]), __uint_as_float(s[cc * 16 + 2 * i + 1])), c2, neg_m2);
+                            const float2 e = ((kPolyPairs >> i) & 1u) ? exp2_poly2(t) : make_float2(fast_exp2(t.x), fast_exp2(t.y));
+                            if (i & 1)
+                                sum1 = tc::fadd2(sum1, e);
+                            else
+                                sum0 = tc::fadd2(sum0, e);
+                            pk[i] = pack_bf16(e.x, e.y);
+                        }
+                        tc::tmem_st8(t_s + cc * 8, pk);   // P: bf16 pairs over the first 64 columns of S
+                    }
+                    l += (sum0.x + sum0.y) + (sum1.x + sum1.y);
+                    tc::tmem_wait_st();
+                    tc::fence_before_sync();
+                    tc::mbar_arrive(pbar);
                 }
-            }
-            const float2 c2 = make_float2(c, c), neg_m2 = make_float2(-m, -m);
-            float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0;
+                if (ok && ps.pair) {
+                    if ((ok = tc::mbar_wait(tc::smem_addr(&bars->o_final), (uint32_t)pass & 1u, abort_flag))) {
+                        tc::fence_after_sync();
+                        const int grow = (ps.tile + x) * BM + row;
+                        const float inv = 1.0f / l;
+                        uint32_t o[64];
+                        tc::tmem_ld32(t_o, o);
+                        tc::tmem_ld32(t_o + 32, o + 32);
+                        tc::tmem_wait_ld();
+                        if (grow < p.m_q) {
+                            uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)ps.head * p.out_stride_head + (int64_t)grow * p.out_stride_token);
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-                uint32_t pk[8];
+                            for (int i = 0; i < 8; ++i) {
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+                                v.y = pack_bf16(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+                                v.z = pack_bf16(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+                                v.w = pack_bf16(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+                                dst[i] = v;
+                            }
+                        }
+                    }
+                } else if (ok && x == 1) {
+                    // single pass, group B: publish this row's partial (max, sum); O_B stays in tensor memory for group A.
+                    // Do not touch O_B again (next pass's zero fill) before group A has read it.
+                    xch[row] = make_float2(m, l);
+                    tc::mbar_arrive(tc::smem_addr(&bars->x_full));
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->x_done), n_single & 1u, abort_flag);
+                } else if (ok) {
+                    // single pass, group A: combine the two partial softmaxes over disjoint keys
+                    //   out = (O_A 2^(m_A - m) + O_B 2^(m_B - m)) / (l_A 2^(m_A - m) + l_B 2^(m_B - m)),  m = max(m_A, m_B)
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->o_final), (uint32_t)pass & 1u, abort_flag) &&
+                         tc::mbar_wait(tc::smem_addr(&bars->x_full), n_single & 1u, abort_flag);
+                    if (ok) {
+                        tc::fence_after_sync();
+                        const float2 pb = xch[row];
+                        const float mm = fmaxf(m, pb.x);
+                        const float fa = exp2f(m - mm), fb = exp2f(pb.x - mm);   // 2^(-inf) = 0 when group B had no key tile
+                        const float inv = 1.0f / (l * fa + pb.y * fb);
+                        const float wa = fa * inv, wb = fb * inv;
+                        const int grow = ps.tile * BM + row;
+                        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)ps.head * p.out_stride_head + (int64_t)grow * p.out_stride_token);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float2 t = tc::ffma2(make_float2(__uint_as_float(s[cc * 16 + 2 * i]), __uint_as_float(s[cc * 16 + 2 * i + 1])), c2, neg_m2);
-                    const float2 e = ((kPolyPairs >> i) & 1u) ? exp2_poly2(t) : make_float2(fast_exp2(t.x), fast_exp2(t.y));
-                    if (i & 1)
-                        sum1 = tc::fadd2(sum1, e);
-                    else
-                        sum0 = tc::fadd2(sum0, e);
-                    pk[i] = pack_bf16(e.x, e.y);
+                        for (int half = 0; half < 2; ++half) {
+                            uint32_t oa[32], ob[32];
+                            tc::tmem_ld32(t_o + half * 32, oa);
+                            tc::tmem_ld32(t_o + kHeadDim + half * 32, ob);   // O_B sits right behind O_A; same TMEM lanes
+                            tc::tmem_wait_ld();
+                            if (grow < p.m_q) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    uint32_t w[4];
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e)
+                                        w[e] = pack_bf16(fmaf(__uint_as_float(oa[8 * i + 2 * e]), wa, __uint_as_float(ob[8 * i + 2 * e]) * wb),
+                                                         fmaf(__uint_as_float(oa[8 * i + 2 * e + 1]), wa, __uint_as_float(ob[8 * i + 2 * e + 1]) * wb));
+                                    dst[half * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
+                                }
+                            }
+                        }
+                        tc::fence_before_sync();
+                        tc::mbar_arrive(tc::smem_addr(&bars->x_done));
+                    }
                 }
-                asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(t_s + cc * 8),
-                             "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7])
-                             : "memory");
+                od_base += (uint32_t)n_own;
+                if (!ps.pair) ++n_single;
             }
-            const float sum = (sum0.x + sum0.y) + (sum1.x + sum1.y);
-            l += sum;
-            tc::tmem_wait_st();
-            tc::fence_before_sync();
-            tc::mbar_arrive(pbar);
-        }
-        if (ok && (ok = tc::mbar_wait(tc::smem_addr(&bars->o_final), 0, abort_flag))) {
-            tc::fence_after_sync();
-            const int grow = q0 + x * BM + row;
-            const float inv = 1.0f / l;
-            uint32_t o[64];
-            tc::tmem_ld32(t_o, o);
-            tc::tmem_ld32(t_o + 32, o + 32);
-            tc::tmem_wait_ld();
-            if (grow < p.m_q) {
-                uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)head * p.out_stride_head + (int64_t)grow * p.out_stride_token);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    uint4 v;
-                    v.x = pack_bf16(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-                    v.y = pack_bf16(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-                    v.z = pack_bf16(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-                    v.w = pack_bf16(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-                    dst[i] = v;
-                }
-            }
+            for (int b = 0; b < 3; ++b) sp_base[b] += (uint32_t)count_mod3(n_score, b);
         }
     }
     tc::fence_before_sync();
@@ -358,15 +507,20 @@ cudaError_t configure_attention() {
 }
 
 // Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
-cudaError_t launch_attention(const AttentionArgs& a, int /*sm_count*/, cudaStream_t stream) {
+cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream) {
     CUtensorMap mq, mk, mv;
     if (!encode_rows_tensor_map(&mq, a.q.ptr, a.m_q, a.heads, a.q.stride_token, a.q.stride_head, BM) ||
         !encode_rows_tensor_map(&mk, a.k.ptr, a.m_k, a.heads, a.k.stride_token, a.k.stride_head, BN) ||
         !encode_rows_tensor_map(&mv, a.v.ptr, a.m_k, a.heads, a.v.stride_token, a.v.stride_head, BN))
         return cudaErrorInvalidValue;
-    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status};
-    dim3 grid((a.m_q + 2 * BM - 1) / (2 * BM), a.heads);
-    attention_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
+    const int tiles_per_head = (a.m_q + BM - 1) / BM, total = tiles_per_head * a.heads;
+    // one CTA per SM (fewer when there are fewer tiles), each with a contiguous chunk of the query tiles
+    int ctas = sm_count < 1 ? 1 : sm_count;
+    if (ctas > total) ctas = total;
+    const int chunk = (total + ctas - 1) / ctas;
+    ctas = (total + chunk - 1) / chunk;
+    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, chunk};
+    attention_tc_kernel<<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
 
