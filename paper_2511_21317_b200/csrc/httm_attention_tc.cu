@@ -51,7 +51,7 @@ struct TcParams {
     int32_t m_q, m_k;
     float scale_log2;
     int32_t* status;
-    int32_t tiles_per_head, total_tiles, chunk;   // query tiles per head, in all heads, per CTA
+    int32_t tiles_per_head, total_tiles, rounds;  // query tiles per head and in all heads; rounds of pair passes
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -90,26 +90,54 @@ __device__ __forceinline__ float2 exp2_poly2(float2 t) {
 // split (0/8: 574 us, 1/8: 540 us, 2/8: 557 us, 3/8: 587 us).
 constexpr uint32_t kPolyPairs = 0x10;   // pair 4 of 8
 
-// Work decomposition.  The query tiles of all heads form one list (head-major); CTA c of G takes the
-// contiguous chunk [c L, (c + 1) L) of it and walks it in PASSES: two consecutive tiles of the same head as
-// a pair pass (tiles A and B share the K/V stream), a left-over tile as a single pass: the same machinery
-// with ONE query tile whose even key tiles go to softmax group A / accumulator O_A and odd ones to group B /
-// O_B (two partial softmaxes over disjoint keys), combined in the epilogue.  Either way score tile k is
-// handled by group k mod 2 in buffer k mod 3.  With one CTA per SM the SMs finish within one tile of each other,
-// whereas a grid of 672 two-tile CTAs on 148 SMs runs 4.54 waves as 5.
+// Work decomposition.  The query tiles of all heads form one list (head-major, T tiles).  With G CTAs
+// (one per SM), round r < R = T / (2 G) gives CTA c the two tiles 2 (r G + c), +1: a PAIR pass (tiles A and B
+// share the K/V stream) if they belong to the same head, else two single passes.  The remaining
+// T - 2 G R < 2 G tiles are one more partial round of pairs if there are more than G of them, else they are
+// dealt one per CTA as SINGLE passes: the same machinery with ONE query tile whose
+// even key tiles go to softmax group A / accumulator O_A and odd ones to group B / O_B (two partial
+// softmaxes over disjoint keys), combined in the epilogue; a single pass takes about half a pair pass.
+// Either way score tile k is handled by group k mod 2 in buffer k mod 3.  All CTAs work on neighbouring
+// tiles at any time (K/V of one or two heads stay in L2), and the SMs finish within half a pass of each
+// other, whereas a grid of 672 two-tile CTAs on 148 SMs runs 4.54 waves as 5.
 struct Pass {
     int head, tile;   // tile = index of query tile A inside the head
     bool pair;
 };
 struct PassWalker {
-    int t, t_end, tiles_per_head;
-    __device__ PassWalker(int chunk, int total, int tph) : t(blockIdx.x * chunk), t_end(min(total, (int)(blockIdx.x + 1) * chunk)), tiles_per_head(tph) {}
-    __device__ bool next(Pass* ps) {
-        if (t >= t_end) return false;
+    int r = 0, sub = 0;
+    int rounds, total, tiles_per_head;
+    __device__ PassWalker(int rounds_, int total_, int tph) : rounds(rounds_), total(total_), tiles_per_head(tph) {}
+    __device__ void set(Pass* ps, int t, bool pair) {
         ps->head = t / tiles_per_head;
         ps->tile = t - ps->head * tiles_per_head;
-        ps->pair = t + 1 < t_end && ps->tile + 1 < tiles_per_head;
-        t += ps->pair ? 2 : 1;
+        ps->pair = pair;
+    }
+    __device__ bool next(Pass* ps) {
+        const int G = gridDim.x, c = blockIdx.x;
+        const int rem = total - 2 * G * rounds;               // tiles left after the full rounds, < 2 G
+        const int pair_rounds = rounds + (rem > G ? 1 : 0);   // more than G left: one more (partial) round of pairs
+        if (r < pair_rounds) {
+            const int t = 2 * (r * G + c);
+            if (t + 1 < total && t / tiles_per_head == (t + 1) / tiles_per_head) {
+                set(ps, t, true);
+                ++r;
+                return true;
+            }
+            if (t + sub < total) {   // the two tiles straddle a head boundary (two single passes, the cost of one pair pass),
+                set(ps, t + sub, false);   // or only one tile is left
+                if (sub == 1) ++r;
+                sub ^= 1;
+                return true;
+            }
+            r = pair_rounds + 1;
+            return false;
+        }
+        if (r > pair_rounds || rem > G) return false;
+        const int t = 2 * G * rounds + c;                     // at most G left: one single pass each
+        ++r;
+        if (t >= total) return false;
+        set(ps, t, false);
         return true;
     }
 };
@@ -162,7 +190,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
     // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the first 64 columns of its S
-    PassWalker walker(p.chunk, p.total_tiles, p.tiles_per_head);
+    PassWalker walker(p.rounds, p.total_tiles, p.tiles_per_head);
     Pass ps;
 
     if (warp == 0) {
@@ -514,12 +542,11 @@ cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t 
         !encode_rows_tensor_map(&mv, a.v.ptr, a.m_k, a.heads, a.v.stride_token, a.v.stride_head, BN))
         return cudaErrorInvalidValue;
     const int tiles_per_head = (a.m_q + BM - 1) / BM, total = tiles_per_head * a.heads;
-    // one CTA per SM (fewer when there are fewer tiles), each with a contiguous chunk of the query tiles
+    // one CTA per SM (fewer when there are fewer tiles)
     int ctas = sm_count < 1 ? 1 : sm_count;
     if (ctas > total) ctas = total;
-    const int chunk = (total + ctas - 1) / ctas;
-    ctas = (total + chunk - 1) / chunk;
-    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, chunk};
+    const int rounds = total / (2 * ctas);
+    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, rounds};
     attention_tc_kernel<<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
