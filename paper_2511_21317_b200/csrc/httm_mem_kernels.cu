@@ -183,7 +183,7 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 }
 
 template <int PASSES>
-__global__ void __launch_bounds__(match_warps_per_cta(32 * PASSES) * 32, PASSES == 1 ? 3 : 1)
+__global__ void __launch_bounds__(match_warps_per_cta(32 * PASSES) * 32, PASSES == 1 ? 2 : 1)   // 3 CTAs/SM would need 80 registers: spills cost more than the third CTA gains
 match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const MatchArgs a) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = match_warps_per_cta(NMAX);
@@ -455,7 +455,7 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
         return cudaErrorInvalidValue;
     const int64_t n_tasks = 2ll * a.heads * a.n_blocks;
     int ctas_per_sm = (int)((224 * 1024) / (smem + 1024));
-    ctas_per_sm = ctas_per_sm < 1 ? 1 : (ctas_per_sm > 32 / WARPS ? 32 / WARPS : ctas_per_sm);
+    ctas_per_sm = ctas_per_sm < 1 ? 1 : (ctas_per_sm > 16 / WARPS ? (16 / WARPS < 1 ? 1 : 16 / WARPS) : ctas_per_sm);
     int64_t grid = (n_tasks + WARPS - 1) / WARPS;
     const int64_t cap = (int64_t)sm_count * ctas_per_sm;
     if (grid > cap) grid = cap;
