@@ -27,6 +27,9 @@ if ROOT not in sys.path:
 
 from paper_2511_21317_b200 import synth  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (ncu, profiles/ncu_full_medium_five_kernels.txt);
+# None for workloads that were not captured, and to be reset to None whenever the attention kernel changes.
+ATTENTION_DRAM_TRAFFIC = {"medium": None}
 METRIC = "httm_global_attention_layer_throughput"
 UNIT = "tokens/s"
 
@@ -223,19 +226,22 @@ def run_ours(args, wl):
     launches = ctx.launch_count() - l0
     ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
 
-    # ---- per-kernel durations: the same five launches with events between them
-    stage_ms = np.zeros(5)
-    evs = [[ev() for _ in range(6)] for _ in range(args.steps)]
-    for s in range(args.steps):
-        evs[s][0].record(stream)
-        for st in range(5):
+    # ---- per-kernel durations: every kernel of the path launched on its own with events between them.
+    #      Order: reorder, match, merge (the separate kernels), then - where the geometry allows it - match and
+    #      merge reading their blocks straight from Q/K/V (the two that the public call uses), attention, unmerge.
+    direct = ctx.query(hb.Q_MAX_BLOCK_TOKENS) <= 32
+    order = [0, 1, 2] + ([5, 6] if direct else []) + [3, 4]
+    stage_ms = {st: 0.0 for st in order}
+    evs = [[ev() for _ in range(len(order) + 1)] for _ in range(args.steps)]
+    for s_ in range(args.steps):
+        evs[s_][0].record(stream)
+        for i, st in enumerate(order):
             ctx.launch_stage(st, dq, dk, dv, out)
-            evs[s][st + 1].record(stream)
+            evs[s_][i + 1].record(stream)
     torch.cuda.synchronize()
-    for s in range(args.steps):
-        for st in range(5):
-            stage_ms[st] += evs[s][st].elapsed_time(evs[s][st + 1])
-    stage_ms /= args.steps
+    for s_ in range(args.steps):
+        for i, st in enumerate(order):
+            stage_ms[st] += evs[s_][i].elapsed_time(evs[s_][i + 1]) / args.steps
 
     # ---- dense baseline of the same run (same attention kernel on the unmerged tokens)
     dsteps = max(3, min(args.steps, 10))
@@ -279,9 +285,10 @@ def run_ours(args, wl):
             "unmerge": H * Mq * D * b + H * N * 4 + H * N * D * b,
         }
         attn_flops = 4.0 * H * Mq * Mk * D
+        alg["match_direct"], alg["merge_direct"] = alg["match"], alg["merge"]
         kernels = {}
-        for i, name in enumerate(hb.STAGE_NAMES):
-            ms = float(stage_ms[i])
+        for st in order:
+            name, ms = hb.STAGE_NAMES[st], float(stage_ms[st])
             if name == "attention":
                 tf = attn_flops / (ms * 1e-3) / 1e12
                 kernels[name] = {"ms": ms, "tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
@@ -290,12 +297,15 @@ def run_ours(args, wl):
                 gbs = alg[name] / (ms * 1e-3) / 1e9
                 kernels[name] = {"ms": ms, "algorithmic_mb": alg[name] / 1e6, "gbs": gbs,
                                  "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0}
+        used = ([5, 6] if direct else [0, 1, 2]) + [3, 4]
+        path = {"kernels_of_the_public_call": [hb.STAGE_NAMES[st] for st in used],
+                "sum_of_their_stage_times_ms": float(sum(stage_ms[st] for st in used))}
         attn_ms = float(stage_ms[3])
         attn_tf = attn_flops / (attn_ms * 1e-3) / 1e12
         roofline = {"kernel": "attention (merged sets)", "bound": "tensor", "achieved": attn_tf,
                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": attn_tf / peaks["bf16_tflops_sustained"],
                     "peak_source": peaks["source"] + " (sustained bf16 GEMM; kernel timed inside the step)",
-                    "traffic": None}
+                    "traffic": ATTENTION_DRAM_TRAFFIC.get(wl.name)}
         line = {
             "metric": METRIC, "value": world * N / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -307,6 +317,7 @@ def run_ours(args, wl):
             "gpu_launches": int(launches),
             "roofline": roofline,
             "kernels": kernels,
+            "path": path,
             "merged_tokens": {"M_q": Mq, "M_k": Mk},
             "dense": {"ms": dense_ms, "tflops": 4.0 * H * N * N * D / (dense_ms * 1e-3) / 1e12, "steps": dsteps},
             "speedup_vs_dense": dense_ms / ms_step,

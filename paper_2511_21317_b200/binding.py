@@ -20,8 +20,8 @@ LIB_PATH = os.path.join(_HERE, "libhttm.so")
 Q_TOKENS, Q_MERGED_Q, Q_MERGED_K, Q_BLOCKS, Q_WORKSPACE_BYTES, Q_MAX_BLOCK_TOKENS, Q_DEVICE_STATUS = range(7)
 (X_PI, X_PI_INV, X_BLOCK_START, X_ASSIGN_Q, X_ASSIGN_K, X_RANK_Q, X_Q_REORDERED, X_K_REORDERED, X_V_REORDERED,
  X_Q_MERGED, X_K_MERGED, X_V_MERGED, X_O_MERGED) = range(13)
-STAGE_REORDER, STAGE_MATCH, STAGE_MERGE, STAGE_ATTENTION, STAGE_UNMERGE = range(5)
-STAGE_NAMES = ("reorder", "match", "merge", "attention", "unmerge")
+STAGE_REORDER, STAGE_MATCH, STAGE_MERGE, STAGE_ATTENTION, STAGE_UNMERGE, STAGE_MATCH_DIRECT, STAGE_MERGE_DIRECT = range(7)
+STAGE_NAMES = ("reorder", "match", "merge", "attention", "unmerge", "match_direct", "merge_direct")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPORTED", -3: "HTTM_ERR_ALIGNMENT",

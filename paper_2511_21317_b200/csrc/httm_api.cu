@@ -37,6 +37,8 @@ struct httm_ctx {
     int sm_count = 148;
     std::vector<int32_t> pi, pi_inv, blk_start;
     std::vector<BlockInfo> blocks;
+    std::vector<BlockGeom> geom;
+    BlockGeom* d_geom = nullptr;
     // device workspace
     int32_t *d_pi = nullptr, *d_pi_inv = nullptr, *d_assign_q = nullptr, *d_assign_k = nullptr, *d_rank_q = nullptr;
     int32_t* d_status = nullptr;
@@ -72,7 +74,7 @@ struct httm_ctx {
         return HTTM_OK;
     }
     void release() {
-        void* ptrs[] = {d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
+        void* ptrs[] = {d_geom, d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
                         d_vr, d_qm,     d_km,       d_vm,       d_om,     d_hq,     d_hk,     d_hv, d_hout};
         for (void* p : ptrs)
             if (p) cudaFree(p);
@@ -156,8 +158,32 @@ int stage_reorder(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const
     return check_cuda(c, launch_reorder(a, s), "reorder launch");
 }
 
-int stage_match(httm_ctx* c, cudaStream_t s) {
+SourceLayout source_layout(const httm_ctx* c) {
+    SourceLayout L{};
+    L.frames = c->cfg.frames;
+    L.grid_h = c->cfg.grid_h;
+    L.grid_w = c->cfg.grid_w;
+    L.n_special = c->n_special;
+    L.tokens_per_frame = c->tokens_per_frame;
+    L.blk_frames = c->cfg.blk_frames;
+    L.blk_h = c->cfg.blk_h;
+    L.blk_w = c->cfg.blk_w;
+    return L;
+}
+
+// Blocks of at most 32 tokens are read by the match and merge kernels straight from Q/K/V (tiled TMA loads of
+// the block's patch window): the reordered copies are then not needed on the hot path.
+bool direct_mode(const httm_ctx* c) { return c->max_block <= 32 && c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767; }
+
+// src: the original Q, K, V (direct mode) or nullptr (blocks come from the reordered copies)
+int stage_match(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     MatchArgs a{};
+    if (src) {
+        a.geom = c->d_geom;
+        a.src[0] = view(src[0]);
+        a.src[1] = view(src[1]);
+        a.layout = source_layout(c);
+    }
     a.xr[0] = c->d_qr;
     a.xr[1] = c->d_kr;
     a.assign[0] = c->d_assign_q;
@@ -171,8 +197,15 @@ int stage_match(httm_ctx* c, cudaStream_t s) {
     return check_cuda(c, launch_match(a, c->max_block, c->sm_count, s), "match launch");
 }
 
-int stage_merge(httm_ctx* c, cudaStream_t s) {
+int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     MergeArgs a{};
+    if (src) {
+        a.geom = c->d_geom;
+        a.src[0] = view(src[0]);
+        a.src[1] = view(src[1]);
+        a.src[2] = view(src[2]);
+        a.layout = source_layout(c);
+    }
     a.xr[0] = c->d_qr;
     a.xr[1] = c->d_kr;
     a.xr[2] = c->d_vr;
@@ -248,9 +281,15 @@ int dense_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const ht
 int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out,
                 cudaStream_t s) {
     int rc;
-    if ((rc = stage_reorder(c, q, k, v, s))) return rc;
-    if ((rc = stage_match(c, s))) return rc;
-    if ((rc = stage_merge(c, s))) return rc;
+    if (direct_mode(c)) {   // four kernels: the temporal reorder is folded into the block loads of match and merge
+        const httm_tensor src[3] = {q, k, v};
+        if ((rc = stage_match(c, s, src))) return rc;
+        if ((rc = stage_merge(c, s, src))) return rc;
+    } else {
+        if ((rc = stage_reorder(c, q, k, v, s))) return rc;
+        if ((rc = stage_match(c, s))) return rc;
+        if ((rc = stage_merge(c, s))) return rc;
+    }
     if ((rc = stage_attention(c, s))) return rc;
     return stage_unmerge(c, out, s);
 }
@@ -333,6 +372,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
                 c->max_block = std::max(c->max_block, bi.n);
                 c->blk_start.push_back(pos);
                 c->blocks.push_back(bi);
+                c->geom.push_back(BlockGeom{(int16_t)g0, (int16_t)y0, (int16_t)x0, (int16_t)f, (int16_t)hh, (int16_t)ww});
                 for (int tl = 0; tl < f; ++tl)
                     for (int yl = 0; yl < hh; ++yl)
                         for (int xl = 0; xl < ww; ++xl) c->pi[pos++] = (g0 + tl) * P + nsp + (y0 + yl) * w + (x0 + xl);
@@ -366,7 +406,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
     if ((rc = check_cuda(c, configure_kernels(), "cudaFuncSetAttribute"))) return done(rc);
 
     const size_t H = cfg->heads, N = c->n_tokens;
-    if ((rc = c->alloc(&c->d_pi, N)) || (rc = c->alloc(&c->d_pi_inv, N)) || (rc = c->alloc(&c->d_blocks, c->blocks.size())) ||
+    if ((rc = c->alloc(&c->d_pi, N)) || (rc = c->alloc(&c->d_pi_inv, N)) || (rc = c->alloc(&c->d_blocks, c->blocks.size())) || (rc = c->alloc(&c->d_geom, c->geom.size())) ||
         (rc = c->alloc(&c->d_status, 4)) || (rc = c->alloc(&c->d_assign_q, H * N)) || (rc = c->alloc(&c->d_assign_k, H * N)) ||
         (rc = c->alloc(&c->d_rank_q, H * N)) || (rc = c->alloc(&c->d_qr, H * N * kHeadDim)) ||
         (rc = c->alloc(&c->d_kr, H * N * kHeadDim)) || (rc = c->alloc(&c->d_vr, H * N * kHeadDim)) ||
@@ -385,6 +425,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
     up(c->d_pi, c->pi.data(), N * 4);
     up(c->d_pi_inv, c->pi_inv.data(), N * 4);
     up(c->d_blocks, c->blocks.data(), c->blocks.size() * sizeof(BlockInfo));
+    up(c->d_geom, c->geom.data(), c->geom.size() * sizeof(BlockGeom));
     up(c->d_assign_q, ident.data(), H * N * 4);
     up(c->d_assign_k, ident.data(), H * N * 4);
     up(c->d_rank_q, ident.data(), H * N * 4);
@@ -456,6 +497,13 @@ int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm
         case HTTM_STAGE_UNMERGE:
             if ((rc = check_tensor(c, out, "out"))) return rc;
             return stage_unmerge(c, out, s);
+        case HTTM_STAGE_MATCH_DIRECT:
+        case HTTM_STAGE_MERGE_DIRECT: {
+            if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "direct stages need merging blocks of at most 32 tokens");
+            if ((rc = check_tensor(c, q, "q")) || (rc = check_tensor(c, k, "k")) || (rc = check_tensor(c, v, "v"))) return rc;
+            const httm_tensor src[3] = {q, k, v};
+            return stage == HTTM_STAGE_MATCH_DIRECT ? stage_match(c, s, src) : stage_merge(c, s, src);
+        }
         default:
             return c->fail(HTTM_ERR_INVALID_ARG, "unknown stage %d", stage);
     }

@@ -29,6 +29,19 @@ struct BlockInfo {
     int32_t r_k, nd_k, moff_k;
 };
 
+// Where a merging block sits in the original layout (used when the kernels read the blocks straight from
+// Q/K/V with tiled TMA loads instead of from the reordered copies): first frame, first patch row and
+// column, and the clipped extents.
+struct BlockGeom {
+    int16_t s0, y0, x0, frames, rows, cols;   // rows x cols patches over `frames` frames; 12 bytes
+};
+// Geometry of the original token layout: token (frame s, in-frame index p) is row s * tokens_per_frame + p;
+// patch (y, x) has p = n_special + y * grid_w + x.
+struct SourceLayout {
+    int32_t frames, grid_h, grid_w, n_special, tokens_per_frame;
+    int32_t blk_frames, blk_h, blk_w;
+};
+
 struct TensorView {          // bf16, element strides
     const __nv_bfloat16* ptr;
     int64_t stride_head, stride_token;
@@ -42,6 +55,10 @@ struct ReorderArgs {
 };
 
 struct MatchArgs {
+    // direct mode (geom != nullptr): blocks are read from the original tensors src[0..1]; else from xr
+    const BlockGeom* geom;
+    TensorView src[2];
+    SourceLayout layout;
     const __nv_bfloat16* xr[2];   // reordered Q, K  [H][N][64]
     int32_t* assign[2];           // A_q, A_k        [H][N]
     const BlockInfo* blocks;
@@ -50,6 +67,10 @@ struct MatchArgs {
 };
 
 struct MergeArgs {
+    // direct mode (geom != nullptr): blocks and special tokens are read from the original tensors src[0..2]
+    const BlockGeom* geom;
+    TensorView src[3];
+    SourceLayout layout;
     const __nv_bfloat16* xr[3];   // reordered Q, K, V
     const int32_t* assign[2];     // A_q, A_k (V uses A_k)
     __nv_bfloat16* merged[3];     // Q_m [H][M_q][64], K_m, V_m [H][M_k][64]

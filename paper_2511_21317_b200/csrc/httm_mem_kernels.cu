@@ -176,13 +176,47 @@ __device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// tiled TMA load of one merging block straight from an original tensor: {64 channels, x, y, frame, head}
+__device__ __forceinline__ void tma_block_load(uint32_t dst_smem, const CUtensorMap* map, uint32_t mbar, int x0, int y0, int s0, int head) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(dst_smem),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(mbar), "r"(0), "r"(x0), "r"(y0), "r"(s0), "r"(head)
+        : "memory");
+}
+// Direct mode: a block arrives as the box [box_frames][box_h][box_w] of 128-byte rows (zero rows where the block
+// is clipped by the grid edge or the last frame); its tokens are numbered in the same (frame, row, column)
+// order without the holes.  For a block that is not clipped both numberings coincide.
+struct BoxMap {
+    int box_h, box_w;          // rows and columns of the box
+    int rows, cols;            // of this block
+    uint32_t m_plane, m_cols;  // multipliers for floor(j / (rows * cols)) and floor(j / cols), j < 256
+    bool clipped;
+    __device__ void set(int box_frames, int bh, int bw, int frames, int r, int c) {
+        box_h = bh;
+        box_w = bw;
+        rows = r;
+        cols = c;
+        clipped = frames != box_frames || r != bh || c != bw;
+        if (clipped) {
+            m_plane = 65536u / (uint32_t)(r * c) + 1u;
+            m_cols = 65536u / (uint32_t)c + 1u;
+        }
+    }
+    // token number -> box row
+    __device__ __forceinline__ int row_of_token(int j) const {
+        if (!clipped) return j;
+        const int t = (int)(((uint32_t)j * m_plane) >> 16), rem = j - t * rows * cols;
+        const int y = (int)(((uint32_t)rem * m_cols) >> 16), x = rem - y * cols;
+        return (t * box_h + y) * box_w + x;
+    }
+};
 // monotone map float -> uint32 (larger float <-> larger key); every real score maps to a key >= 1
 __device__ __forceinline__ uint32_t score_key(float s) {
     const uint32_t b = __float_as_uint(s);
     return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
 }
 
-template <int PASSES>
+template <int PASSES, bool DIRECT>
 __global__ void __launch_bounds__(match_warps_per_cta(32 * PASSES) * 32, PASSES == 1 ? 2 : 1)   // 3 CTAs/SM would need 80 registers: spills cost more than the third CTA gains
 match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const MatchArgs a) {
     constexpr int NMAX = 32 * PASSES;
@@ -215,11 +249,32 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     cur.init(first, stride, a.heads, a.n_blocks);
     nxt = cur;
 
+    // direct mode: box extents (clipped to the scene once) and the box coordinates of the rows this lane owns
+    const int box_f = DIRECT ? min(a.layout.blk_frames, a.layout.frames) : 1, box_h = DIRECT ? min(a.layout.blk_h, a.layout.grid_h) : 1,
+              box_w = DIRECT ? min(a.layout.blk_w, a.layout.grid_w) : 1;
+    const int box_rows = box_f * box_h * box_w;
+    const uint32_t box_bytes = (uint32_t)box_rows * kRowBytes;
+    int own_t[MT], own_y[MT], own_x[MT];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const int rho = mt * 16 + (tq & 1) * 8 + g;
+        own_t[mt] = DIRECT ? rho / (box_h * box_w) : 0;
+        own_y[mt] = DIRECT ? (rho / box_w) % box_h : 0;
+        own_x[mt] = DIRECT ? rho % box_w : 0;
+    }
+    BoxMap bm;
+    bm.clipped = false;
     auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only; the whole box is transferred (rows past the head's end are zero filled)
-        const int start = __ldg(&a.blocks[c.u].start);
         const uint32_t mb = mbar0 + 8 * buf;
-        mbar_expect_tx(mb, STAGE_BYTES);
-        tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : &map_k, mb, start, c.h);
+        if (DIRECT) {
+            const BlockGeom bg = a.geom[c.u];
+            mbar_expect_tx(mb, box_bytes);
+            tma_block_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : &map_k, mb, bg.x0, bg.y0, bg.s0, c.h);
+        } else {
+            const int start = __ldg(&a.blocks[c.u].start);
+            mbar_expect_tx(mb, STAGE_BYTES);
+            tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : &map_k, mb, start, c.h);
+        }
     };
     if (first < n_tasks && lane == 0) issue(nxt, 0);
     nxt.advance();
@@ -259,6 +314,12 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             magic_n = (1u << 23) / (uint32_t)n + 1u;
             magic_nd = (1u << 23) / (uint32_t)nd + 1u;
         }
+        BlockGeom bg{};
+        if (DIRECT) {
+            bg = a.geom[cur.u];
+            bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
+        }
+        const int n_rows = DIRECT ? box_rows : n;   // rows of the stage that may hold tokens
         auto div_n = [&](int x) { return (int)(((uint32_t)x * magic_n) >> 23); };          // x < (n + 1) * n_dst
         auto pos_of = [&](int d) { return (int)(((uint32_t)((d + 1) * n + nd - 1) * magic_nd) >> 23) - 1; };   // position of dst d
         const uint32_t blk = stage0 + buf * STAGE_BYTES;
@@ -275,7 +336,7 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         };
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-            if (mt * 16 < n) {   // warp-uniform
+            if (mt * 16 < n_rows) {   // warp-uniform
                 uint32_t(*fr)[4] = af[KEEP_A ? mt : 0];
                 load_a(mt, fr);
                 float lo[4] = {0.f, 0.f, 0.f, 0.f}, hi[4] = {0.f, 0.f, 0.f, 0.f};
@@ -298,7 +359,7 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         for (int nt = 0; nt < NT; ++nt) {
             if (nt * 8 < nd) {
                 const int d = min(nt * 8 + (lane & 7), nd - 1);
-                const int row = pos_of(d);
+                const int row = DIRECT ? bm.row_of_token(pos_of(d)) : pos_of(d);
 #pragma unroll
                 for (int kp = 0; kp < 2; ++kp) {   // one ldmatrix.x4 = k steps 2 kp and 2 kp + 1
                     uint32_t rr[4];
@@ -322,18 +383,19 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int d = nt * 8 + 2 * tq + e;
-                wd[nt][e] = d < nd ? invn[pos_of(d)] : 0.f;
+                wd[nt][e] = d < nd ? invn[DIRECT ? bm.row_of_token(pos_of(d)) : pos_of(d)] : 0.f;
             }
         uint32_t key[MT];
-        int best[MT];
+        int best[MT], tok[MT];   // tok: number of the owned token in the block, -1 if the row holds none
         bool is_src[MT];
         const int own_half = tq & 1;   // owner of rows g (tq == 0) or g + 8 (tq == 1); lanes with tq >= 2 own nothing
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
             key[mt] = 0;
             best[mt] = 0;
+            tok[mt] = -1;
             is_src[mt] = false;
-            if (mt * 16 < n) {
+            if (mt * 16 < n_rows) {
                 uint32_t(*fr)[4] = af[KEEP_A ? mt : 0];
                 if (!KEEP_A) load_a(mt, fr);
                 float top[2] = {-INFINITY, -INFINITY};   // rows g, g + 8
@@ -375,12 +437,15 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                         }
                     }
                 }
-                const int j = mt * 16 + own_half * 8 + g;
-                if (tq < 2 && j < n) {
+                const int rho = mt * 16 + own_half * 8 + g;   // row of the stage; j: number of the token in the block
+                const bool valid = DIRECT ? (own_t[mt] < bg.frames && own_y[mt] < bg.rows && own_x[mt] < bg.cols) : rho < n;
+                const int j = DIRECT ? (own_t[mt] * bg.rows + own_y[mt]) * bg.cols + own_x[mt] : rho;
+                tok[mt] = valid ? j : -1;
+                if (tq < 2 && valid) {
                     const int dj = div_n(j * nd);
                     if (!(div_n((j + 1) * nd) > dj)) {   // not a dst position: a src token
                         is_src[mt] = true;
-                        key[mt] = score_key((own_half ? top[1] : top[0]) * invn[j]);
+                        key[mt] = score_key((own_half ? top[1] : top[0]) * invn[rho]);
                         best[mt] = pos_of(own_half ? arg[1] : arg[0]);
                     }
                 }
@@ -427,8 +492,7 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
         }
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
-            const int j = mt * 16 + own_half * 8 + g;
-            if (tq < 2 && j < n) A[j] = bi.start + (merged[mt] ? best[mt] : j);
+            if (tq < 2 && tok[mt] >= 0) A[tok[mt]] = bi.start + (merged[mt] ? best[mt] : tok[mt]);
         }
         __syncwarp();   // every lane is done with the inverse norms (and, with several passes, the stage buffer)
         if (!KEEP_A) {
@@ -443,16 +507,28 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     }
 }
 
+// 5-D map of the patch tokens of an original tensor with one merging block as the box
+static bool encode_block_map(CUtensorMap* map, const TensorView& t, const SourceLayout& L, int heads) {
+    const int bw = L.blk_w < L.grid_w ? L.blk_w : L.grid_w, bh = L.blk_h < L.grid_h ? L.blk_h : L.grid_h,
+              bf = L.blk_frames < L.frames ? L.blk_frames : L.frames;
+    return encode_patch_tensor_map(map, t.ptr + (int64_t)L.n_special * t.stride_token, L.grid_w, L.grid_h, L.frames, heads, t.stride_token,
+                                   L.tokens_per_frame, t.stride_head, bw, bh, bf);
+}
+
 template <int PASSES>
 static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t stream) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = match_warps_per_cta(NMAX);
     const size_t smem = match_smem_bytes(NMAX);
+    const bool direct = a.geom != nullptr && PASSES == 1;
     CUtensorMap mq, mk;
     const int64_t N = a.n_tokens;
-    if (!encode_rows_tensor_map(&mq, a.xr[0], N, a.heads, kHeadDim, N * kHeadDim, NMAX) ||
-        !encode_rows_tensor_map(&mk, a.xr[1], N, a.heads, kHeadDim, N * kHeadDim, NMAX))
+    if (direct) {
+        if (!encode_block_map(&mq, a.src[0], a.layout, a.heads) || !encode_block_map(&mk, a.src[1], a.layout, a.heads)) return cudaErrorInvalidValue;
+    } else if (!encode_rows_tensor_map(&mq, a.xr[0], N, a.heads, kHeadDim, N * kHeadDim, NMAX) ||
+               !encode_rows_tensor_map(&mk, a.xr[1], N, a.heads, kHeadDim, N * kHeadDim, NMAX)) {
         return cudaErrorInvalidValue;
+    }
     const int64_t n_tasks = 2ll * a.heads * a.n_blocks;
     int ctas_per_sm = (int)((224 * 1024) / (smem + 1024));
     ctas_per_sm = ctas_per_sm < 1 ? 1 : (ctas_per_sm > 16 / WARPS ? (16 / WARPS < 1 ? 1 : 16 / WARPS) : ctas_per_sm);
@@ -460,7 +536,10 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
     const int64_t cap = (int64_t)sm_count * ctas_per_sm;
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
-    match_kernel<PASSES><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
+    if (direct)
+        match_kernel<1, true><<<(unsigned)grid, match_warps_per_cta(32) * 32, match_smem_bytes(32), stream>>>(mq, mk, a);
+    else
+        match_kernel<PASSES, false><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
     return cudaGetLastError();
 }
 
@@ -682,9 +761,13 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t saddr) {
                  : "memory");
 }
 
+// DIRECT: the blocks come straight from the original tensors (5-D block maps), the special tokens frame by
+// frame (4-D frame maps sq, sk, sv); otherwise from the reordered copies, specials in chunks of 32.
+template <bool DIRECT>
 __global__ void __launch_bounds__(kMergeTcWarps * 32, 2)
 merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const __grid_constant__ CUtensorMap map_v, const MergeArgs a) {
+                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_sq,
+                const __grid_constant__ CUtensorMap map_sk, const __grid_constant__ CUtensorMap map_sv, const MergeArgs a) {
     constexpr uint32_t STAGE_BYTES = 32 * kRowBytes;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -705,8 +788,14 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     // task -> (tensor t, head h, unit u); units 0 .. n_blocks-1 are merging blocks, the rest are
     // chunks of 32 special tokens (never merged: rows 0 .. n_special_total-1 are copied)
-    const int sp_chunks = (a.n_special_total + 31) / 32;
+    const int sp_chunks = DIRECT ? (a.layout.n_special > 0 ? a.layout.frames : 0) : (a.n_special_total + 31) / 32;
     const int per_head = a.n_blocks + sp_chunks;
+    const int box_f = DIRECT ? min(a.layout.blk_frames, a.layout.frames) : 1, box_h = DIRECT ? min(a.layout.blk_h, a.layout.grid_h) : 1,
+              box_w = DIRECT ? min(a.layout.blk_w, a.layout.grid_w) : 1;
+    const int box_rows = box_f * box_h * box_w;
+    const int own_t = DIRECT ? lane / (box_h * box_w) : 0, own_y = DIRECT ? (lane / box_w) % box_h : 0, own_x = DIRECT ? lane % box_w : 0;
+    BoxMap bm;
+    bm.clipped = false;
     const int64_t n_tasks = 3ll * a.heads * per_head;
     const int64_t stride = (int64_t)gridDim.x * kMergeTcWarps;
     const int64_t first = (int64_t)blockIdx.x * kMergeTcWarps + warp;
@@ -717,8 +806,21 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto unit_start = [&](const TaskCursor& c) { return c.u >= a.n_blocks ? (c.u - a.n_blocks) * 32 : __ldg(&a.blocks[c.u].start); };
     auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only; the whole 32-row box is transferred (rows past the head's end are zero filled)
         const uint32_t mb = mbar0 + 8 * buf;
-        mbar_expect_tx(mb, STAGE_BYTES);
-        tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, unit_start(c), c.h);
+        if (!DIRECT) {
+            mbar_expect_tx(mb, STAGE_BYTES);
+            tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, unit_start(c), c.h);
+        } else if (c.u >= a.n_blocks) {   // the special tokens of frame u - n_blocks
+            mbar_expect_tx(mb, (uint32_t)a.layout.n_special * kRowBytes);
+            const CUtensorMap* m = c.t == 0 ? &map_sq : (c.t == 1 ? &map_sk : &map_sv);
+            asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+                             stage0 + buf * STAGE_BYTES),
+                         "l"(reinterpret_cast<uint64_t>(m)), "r"(mb), "r"(0), "r"(0), "r"(c.u - a.n_blocks), "r"(c.h)
+                         : "memory");
+        } else {
+            const BlockGeom bg = a.geom[c.u];
+            mbar_expect_tx(mb, (uint32_t)box_rows * kRowBytes);
+            tma_block_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, bg.x0, bg.y0, bg.s0, c.h);
+        }
     };
     if (first < n_tasks && lane == 0) issue(nxt, 0);
     nxt.advance();
@@ -734,12 +836,18 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int t = cur.t, h = cur.h;
         const bool special = cur.u >= a.n_blocks;
         int start, n, r, moff;
+        BlockGeom bg{};
         if (special) {
-            start = (cur.u - a.n_blocks) * 32;
-            n = min(32, a.n_special_total - start);
+            start = DIRECT ? (cur.u - a.n_blocks) * a.layout.n_special : (cur.u - a.n_blocks) * 32;
+            n = DIRECT ? a.layout.n_special : min(32, a.n_special_total - start);
             r = 0;
             moff = start;
+            bm.clipped = false;
         } else {
+            if (DIRECT) {
+                bg = a.geom[cur.u];
+                bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
+            }
             const BlockInfo bi = a.blocks[cur.u];
             start = bi.start;
             n = bi.n;
@@ -751,13 +859,17 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint32_t blk = stage0 + buf * STAGE_BYTES;
 
         // the map entry does not depend on the staged rows: fetch it before waiting
+        // lane = row of the stage; tok = number of the token it holds (-1: none); rep = ROW of the token it is merged into
+        const int tok = !DIRECT || special ? (lane < n ? lane : -1)
+                                           : ((own_t < bg.frames && own_y < bg.rows && own_x < bg.cols) ? (own_t * bg.rows + own_y) * bg.cols + own_x : -1);
         int rep = -1;
-        if (r > 0 && lane < n) {
-            rep = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + lane) - start;
+        if (r > 0 && tok >= 0) {
+            rep = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + tok) - start;
             if (rep < 0 || rep >= n) {   // corrupt map: record, treat as kept
                 atomicCAS(a.status, kDevOk, kDevBadIndex);
-                rep = lane;
+                rep = tok;
             }
+            if (DIRECT) rep = bm.row_of_token(rep);
         }
         if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
             failed = true;
@@ -767,7 +879,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const unsigned char* sb = stage + buf * STAGE_BYTES;
             uint4* o4 = reinterpret_cast<uint4*>(out);
             for (int q = lane; q < n * 8; q += 32) {
-                const int row = q >> 3, ch = q & 7;
+                const int row = DIRECT ? bm.row_of_token(q >> 3) : q >> 3, ch = q & 7;
                 o4[q] = *reinterpret_cast<const uint4*>(sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
             }
             if (t == 0 && !special && lane < n) a.rank_q[(int64_t)h * a.n_tokens + start + lane] = moff + lane;
@@ -776,13 +888,13 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const unsigned kept = __ballot_sync(0xffffffffu, rep == lane);   // rep == -1 for lanes >= n
             const int n_kept = __popc(kept);
             const int row_of = rep >= 0 ? __popc(kept & ((1u << rep) - 1u)) : -1;
-            if (t == 0 && lane < n) a.rank_q[(int64_t)h * a.n_tokens + start + lane] = moff + row_of;
+            if (t == 0 && tok >= 0) a.rank_q[(int64_t)h * a.n_tokens + start + tok] = moff + row_of;
             const unsigned group = __match_any_sync(0xffffffffu, row_of);
             if (rep == lane) rcnt[row_of] = 1.0f / (float)__popc(group);
             // x fragments: for k step ks (16 tokens) and channel tile pair np, one ldmatrix.x4.trans gives
             // b0, b1 of channel tile 2 np and b0, b1 of channel tile 2 np + 1
             uint32_t bf[2][4][4];
-            const int n_ks = n > 16 ? 2 : 1;
+            const int n_ks = (DIRECT ? box_rows : n) > 16 ? 2 : 1;   // rows of the stage that may hold tokens
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
                 if (ks < n_ks) {
@@ -850,18 +962,32 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 }
 
 static cudaError_t launch_merge_tc(const MergeArgs& a, int sm_count, cudaStream_t stream) {
-    CUtensorMap mq, mk, mv;
+    CUtensorMap m[3], sp[3];
     const int64_t N = a.n_tokens;
-    if (!encode_rows_tensor_map(&mq, a.xr[0], N, a.heads, kHeadDim, N * kHeadDim, 32) ||
-        !encode_rows_tensor_map(&mk, a.xr[1], N, a.heads, kHeadDim, N * kHeadDim, 32) ||
-        !encode_rows_tensor_map(&mv, a.xr[2], N, a.heads, kHeadDim, N * kHeadDim, 32))
-        return cudaErrorInvalidValue;
-    const int64_t n_tasks = 3ll * a.heads * (a.n_blocks + (a.n_special_total + 31) / 32);
+    const bool direct = a.geom != nullptr;
+    const int sp_units = direct ? (a.layout.n_special > 0 ? a.layout.frames : 0) : (a.n_special_total + 31) / 32;
+    for (int t = 0; t < 3; ++t) {
+        if (direct) {
+            if (!encode_block_map(&m[t], a.src[t], a.layout, a.heads)) return cudaErrorInvalidValue;
+            if (a.layout.n_special > 0 &&
+                !encode_frame_tensor_map(&sp[t], a.src[t].ptr, a.layout.tokens_per_frame, a.layout.frames, a.heads, a.src[t].stride_token,
+                                         a.src[t].stride_head, a.layout.n_special))
+                return cudaErrorInvalidValue;
+            if (a.layout.n_special <= 0) sp[t] = m[t];   // never used
+        } else {
+            if (!encode_rows_tensor_map(&m[t], a.xr[t], N, a.heads, kHeadDim, N * kHeadDim, 32)) return cudaErrorInvalidValue;
+            sp[t] = m[t];   // not used
+        }
+    }
+    const int64_t n_tasks = 3ll * a.heads * (a.n_blocks + sp_units);
     int64_t grid = (n_tasks + kMergeTcWarps - 1) / kMergeTcWarps;
     const int64_t cap = (int64_t)sm_count * 2;
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
-    merge_tc_kernel<<<(unsigned)grid, kMergeTcWarps * 32, kMergeTcSmem, stream>>>(mq, mk, mv, a);
+    if (direct)
+        merge_tc_kernel<true><<<(unsigned)grid, kMergeTcWarps * 32, kMergeTcSmem, stream>>>(m[0], m[1], m[2], sp[0], sp[1], sp[2], a);
+    else
+        merge_tc_kernel<false><<<(unsigned)grid, kMergeTcWarps * 32, kMergeTcSmem, stream>>>(m[0], m[1], m[2], sp[0], sp[1], sp[2], a);
     return cudaGetLastError();
 }
 
@@ -941,10 +1067,12 @@ cudaError_t configure_kernels() {
 #define HTTM_SET_SMEM(kern, bytes)                                                                      \
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes));          \
     if (e != cudaSuccess) return e;
-    HTTM_SET_SMEM(match_kernel<1>, match_smem_bytes(32));
-    HTTM_SET_SMEM(match_kernel<4>, match_smem_bytes(128));
-    HTTM_SET_SMEM(match_kernel<8>, match_smem_bytes(256));
-    HTTM_SET_SMEM(merge_tc_kernel, kMergeTcSmem);
+    HTTM_SET_SMEM((match_kernel<1, false>), match_smem_bytes(32));
+    HTTM_SET_SMEM((match_kernel<1, true>), match_smem_bytes(32));
+    HTTM_SET_SMEM((match_kernel<4, false>), match_smem_bytes(128));
+    HTTM_SET_SMEM((match_kernel<8, false>), match_smem_bytes(256));
+    HTTM_SET_SMEM(merge_tc_kernel<false>, kMergeTcSmem);
+    HTTM_SET_SMEM(merge_tc_kernel<true>, kMergeTcSmem);
     HTTM_SET_SMEM(merge_kernel<4>, merge_smem_bytes(128));
     HTTM_SET_SMEM(merge_kernel<8>, merge_smem_bytes(256));
 #undef HTTM_SET_SMEM

@@ -43,6 +43,38 @@ bool encode_rows_tensor_map(CUtensorMap* map, const void* base, int64_t rows, in
     return r == CUDA_SUCCESS;
 }
 
+bool encode_patch_tensor_map(CUtensorMap* map, const void* base, int grid_w, int grid_h, int frames, int64_t heads,
+                             int64_t stride_token, int64_t tokens_per_frame, int64_t stride_head, int box_w, int box_h,
+                             int box_frames) {
+    std::call_once(g_encode_once, resolve_encode);
+    if (!g_encode) return false;
+    const cuuint64_t dims[5] = {64, (cuuint64_t)grid_w, (cuuint64_t)grid_h, (cuuint64_t)frames, (cuuint64_t)heads};
+    const cuuint64_t strides[4] = {(cuuint64_t)stride_token * 2, (cuuint64_t)stride_token * grid_w * 2,
+                                   (cuuint64_t)stride_token * tokens_per_frame * 2,
+                                   (cuuint64_t)(heads > 1 ? stride_head : stride_token * tokens_per_frame * frames) * 2};
+    const cuuint32_t box[5] = {64, (cuuint32_t)box_w, (cuuint32_t)box_h, (cuuint32_t)box_frames, 1};
+    const cuuint32_t elem[5] = {1, 1, 1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, elem,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool encode_frame_tensor_map(CUtensorMap* map, const void* base, int64_t tokens_per_frame, int frames, int64_t heads,
+                             int64_t stride_token, int64_t stride_head, int box_tokens) {
+    std::call_once(g_encode_once, resolve_encode);
+    if (!g_encode) return false;
+    const cuuint64_t dims[4] = {64, (cuuint64_t)tokens_per_frame, (cuuint64_t)frames, (cuuint64_t)heads};
+    const cuuint64_t strides[3] = {(cuuint64_t)stride_token * 2, (cuuint64_t)stride_token * tokens_per_frame * 2,
+                                   (cuuint64_t)(heads > 1 ? stride_head : stride_token * tokens_per_frame * frames) * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)box_tokens, 1, 1};
+    const cuuint32_t elem[4] = {1, 1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 namespace {
 
 __global__ void __launch_bounds__(128) umma_selftest_kernel(const __grid_constant__ CUtensorMap map_q,

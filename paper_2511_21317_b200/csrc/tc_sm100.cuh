@@ -246,4 +246,15 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 bool encode_rows_tensor_map(CUtensorMap* map, const void* base, int64_t rows, int64_t heads, int64_t stride_row,
                             int64_t stride_head, int box_rows);
 
+// Host: 5-D bf16 tensor map over the patch tokens of an original [heads][tokens][64] tensor (any head / token
+// strides): dimensions {64 channels, grid_w, grid_h, frames, heads}, box {64, box_w, box_h, box_frames, 1},
+// 128-byte swizzle; `base` points at patch (0, 0) of frame 0.  A box is one merging block in (frame, row,
+// column) order; parts of it outside the grid or past the last frame are zero filled.
+bool encode_patch_tensor_map(CUtensorMap* map, const void* base, int grid_w, int grid_h, int frames, int64_t heads,
+                             int64_t stride_token, int64_t tokens_per_frame, int64_t stride_head, int box_w, int box_h,
+                             int box_frames);
+// Host: 4-D map {64 channels, tokens_per_frame, frames, heads} with box {64, box_tokens, 1, 1} (the special tokens of one frame).
+bool encode_frame_tensor_map(CUtensorMap* map, const void* base, int64_t tokens_per_frame, int frames, int64_t heads,
+                             int64_t stride_token, int64_t stride_head, int box_tokens);
+
 }  // namespace httm

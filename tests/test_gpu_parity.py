@@ -31,6 +31,8 @@ def run_case(wl, q=None, k=None, v=None, sample=None, peaky=False):
         out = ctx.global_attention(dq, dk, dv)
         torch.cuda.synchronize()
         assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        # the public call reads small blocks straight from Q/K/V; the reorder kernel runs on request
+        ctx.launch_stage(hb.STAGE_REORDER, dq, dk, dv)
         ex = exports(ctx)
         out_bits = hb.bits_from_bf16(out)
         stats = parity.full_check(g, wl.ratio_q, wl.ratio_kv, q, k, v, ex, out_bits, sample, wl.name, peaky)
@@ -38,6 +40,7 @@ def run_case(wl, q=None, k=None, v=None, sample=None, peaky=False):
         out2 = ctx.global_attention(dq, dk, dv)
         torch.cuda.synchronize()
         assert torch.equal(out, out2)
+        ctx.launch_stage(hb.STAGE_REORDER, dq, dk, dv)
         ex2 = exports(ctx)
         for name in ex:
             assert np.array_equal(ex[name], ex2[name]), f"{name} differs between two identical calls"
@@ -238,3 +241,31 @@ def test_dense_attention_medium_config_sampled():
         bits = hb.bits_from_bf16(out)
         assert np.isfinite(parity.bits_to_f64(bits)).all()
         parity.check_output(bits[toks], ref, what="dense medium")
+
+
+def test_direct_block_loads_equal_the_reordered_copies():
+    """Match and merge reading their blocks straight from Q/K/V (what the public call does for blocks of
+    at most 32 tokens) against the same kernels reading the reorder kernel's copies: identical maps and
+    ranks; merged values identical where no block is clipped, within one bf16 step elsewhere (the order
+    in which a clipped block's tokens enter the fp32 sums differs)."""
+    for wl in (synth.WORKLOADS["tiny"].replace(heads=3),
+               synth.Workload("clipped", 5, 9, 10, 2, 4, 4, 0.6, 0.7, heads=3, seed=7)):
+        q, k, v = synth.make_qkv(wl)
+        with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+            dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+            names = {"assign_q": hb.X_ASSIGN_Q, "assign_k": hb.X_ASSIGN_K, "rank_q": hb.X_RANK_Q,
+                     "q_m": hb.X_Q_MERGED, "k_m": hb.X_K_MERGED, "v_m": hb.X_V_MERGED}
+            for st in (hb.STAGE_REORDER, hb.STAGE_MATCH, hb.STAGE_MERGE):
+                ctx.launch_stage(st, dq, dk, dv)
+            sep = {n: ctx.export(w).copy() for n, w in names.items()}
+            for st in (hb.STAGE_MATCH_DIRECT, hb.STAGE_MERGE_DIRECT):
+                ctx.launch_stage(st, dq, dk, dv)
+            direct = {n: ctx.export(w) for n, w in names.items()}
+            for n in ("assign_q", "assign_k", "rank_q"):
+                assert np.array_equal(sep[n], direct[n]), f"{wl.name}: {n} differs between the two ways of loading a block"
+            for n in ("q_m", "k_m", "v_m"):
+                a, b = parity.bits_to_f64(sep[n]), parity.bits_to_f64(direct[n])
+                if wl.name != "clipped":
+                    assert np.array_equal(sep[n], direct[n]), f"{wl.name}: {n} differs"
+                else:
+                    assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(a) + 1e-30).all(), f"{wl.name}: {n} differs by more than a bf16 step"
