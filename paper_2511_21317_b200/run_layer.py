@@ -1,6 +1,6 @@
 """Run a few HTTM global-attention layers of a named synthetic workload and nothing else.
 
-    python -m paper_2511_21317_b200.run_layer --workload medium --calls 2 [--dense 1] [--ratio 0.9] [--block 4x4x4]
+    python -m paper_2511_21317_b200.run_layer --workload medium --calls 2 [--dense 1] [--stages 1] [--ratio 0.9] [--block 4x4x4]
 
 A profiler is pointed at this command: few launches, no timing loops, no CPU work besides
 the input generator.  It prints the merged lengths and the device status word, and exits
@@ -22,6 +22,8 @@ def main() -> int:
     ap.add_argument("--workload", default="medium", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--calls", type=int, default=2, help="httm_global_attention calls")
     ap.add_argument("--dense", type=int, default=0, help="httm_dense_attention calls")
+    ap.add_argument("--stages", type=int, default=0, help="rounds of every kernel launched on its own (reorder, match, merge, "
+                    "match and merge with direct block loads where supported, attention, unmerge)")
     ap.add_argument("--heads", type=int, default=None, help="override the number of heads")
     ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
     ap.add_argument("--block", default=None, help="override the block shape, e.g. 4x4x4")
@@ -44,6 +46,10 @@ def main() -> int:
             ctx.global_attention(dq, dk, dv, out)
         for _ in range(args.dense):
             ctx.dense_attention(dq, dk, dv, out)
+        direct = ctx.query(hb.Q_MAX_BLOCK_TOKENS) <= 32
+        for _ in range(args.stages):
+            for st in [0, 1, 2] + ([5, 6] if direct else []) + [3, 4]:
+                ctx.launch_stage(st, dq, dk, dv, out)
         torch.cuda.synchronize()
         status = ctx.query(hb.Q_DEVICE_STATUS)
         print(f"run_layer: {wl.name} N={wl.n_tokens} M_q={ctx.m_q} M_k={ctx.m_k} calls={args.calls} dense={args.dense} "
