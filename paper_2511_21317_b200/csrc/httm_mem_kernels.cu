@@ -151,7 +151,7 @@ struct TaskCursor {
 //     Token j of a block is owned, for the selection, by lane (j & 7) * 4 + ((j >> 3) & 1),
 //     slot j >> 4: the lane where the MMA accumulator layout leaves row j's results.
 // ------------------------------------------------------------------------------------
-__host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 32 ? 8 : (nmax <= 128 ? 4 : 2); }
+__host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 64 ? 8 : (nmax <= 128 ? 4 : 2); }
 __host__ __device__ constexpr int match_aux_bytes(int nmax) { return nmax * 4 + 16; }   // inverse norms + 2 mbarriers
 __host__ __device__ constexpr int match_smem_bytes(int nmax) {
     return match_warps_per_cta(nmax) * (2 * nmax * kRowBytes + match_aux_bytes(nmax)) + 1024 /*alignment slack*/;
@@ -545,199 +545,9 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
 
 cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream) {
     if (max_block_tokens <= 32) return launch_match_t<1>(a, sm_count, stream);
+    if (max_block_tokens <= 64) return launch_match_t<2>(a, sm_count, stream);
     if (max_block_tokens <= 128) return launch_match_t<4>(a, sm_count, stream);
     return launch_match_t<8>(a, sm_count, stream);
-}
-
-// ------------------------------------------------------------------------------------
-// a3 (blocks of more than 32 tokens).  Merged-token aggregation (Sec. 3.2: mean of the dst token and the src tokens
-//     matched to it; Algorithm 1 "BlockAggregate"), one warp per (tensor, head, block).
-//     The block is staged in shared memory by a TMA bulk copy, double buffered per warp.
-//     Each lane owns two channels.  For every kept token, in reordered order, the warp
-//     finds its group with one ballot over the map, sums the group's rows in token order
-//     in fp32 registers (deterministic), divides once and rounds once to bf16.
-//     Kept tokens are compacted: merged row = moff(block) + local rank.
-//     The Q tasks also write rank_q (merged row of every token) for the unmerge.
-// ------------------------------------------------------------------------------------
-__host__ __device__ constexpr int merge_warps_per_cta(int nmax) { return nmax <= 32 ? 8 : (nmax <= 128 ? 4 : 2); }
-__host__ __device__ constexpr int merge_smem_bytes(int nmax) { return merge_warps_per_cta(nmax) * (2 * nmax * kRowBytes + 16) + 128; }
-
-template <int PASSES>
-__global__ void __launch_bounds__(merge_warps_per_cta(32 * PASSES) * 32) merge_kernel(const __grid_constant__ MergeArgs a) {
-    constexpr int NMAX = 32 * PASSES;
-    constexpr int WARPS = merge_warps_per_cta(NMAX);
-    constexpr uint32_t STAGE_BYTES = NMAX * kRowBytes;
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* stage = smem_raw + (size_t)warp * 2 * STAGE_BYTES;                       // [2][NMAX][128]
-    uint64_t* mbar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)WARPS * 2 * STAGE_BYTES) + 2 * warp;
-    const uint32_t mbar0 = smem_u32(mbar), stage0 = smem_u32(stage);
-
-    if (lane == 0) {
-        mbar_init(mbar0, 1);
-        mbar_init(mbar0 + 8, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncwarp();
-
-    // task -> (tensor t, head h, unit u); units 0 .. n_blocks-1 are merging blocks, the rest are
-    // chunks of 32 special tokens (never merged: rows 0 .. n_special_total-1 are copied)
-    const int sp_chunks = (a.n_special_total + 31) / 32;
-    const int per_head = a.n_blocks + sp_chunks;
-    const int64_t n_tasks = 3ll * a.heads * per_head;
-    const int64_t stride = (int64_t)gridDim.x * WARPS;
-    const int64_t first = (int64_t)blockIdx.x * WARPS + warp;
-    TaskCursor cur, nxt;   // the task being processed; the task whose load is issued next
-    cur.init(first, stride, a.heads, per_head);
-    nxt = cur;
-
-    struct Unit {
-        int t, h, start, n, r, moff;
-        bool special;
-    };
-    auto decode = [&](const TaskCursor& c) {
-        Unit u;
-        u.t = c.t;
-        u.h = c.h;
-        u.special = c.u >= a.n_blocks;
-        if (u.special) {
-            u.start = (c.u - a.n_blocks) * 32;
-            u.n = min(32, a.n_special_total - u.start);
-            u.r = 0;
-            u.moff = u.start;
-        } else {
-            const BlockInfo bi = a.blocks[c.u];
-            u.start = bi.start;
-            u.n = bi.n;
-            u.r = u.t == 0 ? bi.r_q : bi.r_k;
-            u.moff = u.t == 0 ? bi.moff_q : bi.moff_k;
-        }
-        return u;
-    };
-    auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only
-        const Unit u = decode(c);
-        const uint32_t bytes = (uint32_t)u.n * kRowBytes;
-        const uint32_t mb = mbar0 + 8 * buf;
-        mbar_expect_tx(mb, bytes);
-        bulk_load(stage0 + buf * STAGE_BYTES, a.xr[u.t] + ((int64_t)u.h * a.n_tokens + u.start) * kHeadDim, bytes, mb);
-    };
-    if (first < n_tasks && lane == 0) issue(nxt, 0);
-    nxt.advance();
-    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
-    nxt.advance();
-
-    int it = 0;
-    bool failed = false;
-    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
-        const int buf = it & 1;
-        const uint32_t parity = (it >> 1) & 1;
-        const Unit u = decode(cur);
-        const int n = u.n;
-        const int m_len = u.t == 0 ? a.m_q : a.m_k;
-        uint32_t* out = reinterpret_cast<uint32_t*>(a.merged[u.t] + ((int64_t)u.h * m_len + u.moff) * kHeadDim);
-        const uint32_t* xs = reinterpret_cast<const uint32_t*>(stage + buf * STAGE_BYTES);   // [n][32] bf16 pairs
-
-        // the map entries do not depend on the staged rows: fetch them before waiting
-        int rep[PASSES];
-        if (u.r > 0) {
-            const int32_t* A = a.assign[u.t == 0 ? 0 : 1] + (int64_t)u.h * a.n_tokens + u.start;
-#pragma unroll
-            for (int p = 0; p < PASSES; ++p) {
-                const int j = lane + 32 * p;
-                rep[p] = j < n ? __ldg(A + j) - u.start : -1;
-                if (j < n && (rep[p] < 0 || rep[p] >= n)) {   // corrupt map: record, treat as kept
-                    atomicCAS(a.status, kDevOk, kDevBadIndex);
-                    rep[p] = j;
-                }
-            }
-        }
-        if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
-            failed = true;
-            break;
-        }
-        if (u.r == 0) {   // nothing merges here: copy the rows, 16 bytes per lane
-            const uint4* s4 = reinterpret_cast<const uint4*>(xs);
-            uint4* o4 = reinterpret_cast<uint4*>(out);
-            for (int q = lane; q < n * 8; q += 32) o4[q] = s4[q];
-            if (u.t == 0 && !u.special)
-                for (int j = lane; j < n; j += 32) a.rank_q[(int64_t)u.h * a.n_tokens + u.start + j] = u.moff + j;
-        } else {
-            unsigned kept[PASSES];
-            int kept_before[PASSES];   // kept tokens in earlier passes
-            int running = 0;
-#pragma unroll
-            for (int p = 0; p < PASSES; ++p) {
-                const int j = lane + 32 * p;
-                kept[p] = __ballot_sync(0xffffffffu, j < n && rep[p] == j);
-                kept_before[p] = running;
-                running += __popc(kept[p]);
-            }
-            if (u.t == 0) {   // merged row of every token of the block
-#pragma unroll
-                for (int p = 0; p < PASSES; ++p) {
-                    const int j = lane + 32 * p;
-                    if (j < n) {
-                        int row = 0;
-#pragma unroll
-                        for (int pp = 0; pp < PASSES; ++pp)
-                            if ((rep[p] >> 5) == pp) row = kept_before[pp] + __popc(kept[pp] & ((1u << (rep[p] & 31)) - 1u));
-                        a.rank_q[(int64_t)u.h * a.n_tokens + u.start + j] = u.moff + row;
-                    }
-                }
-            }
-            int row = 0;
-#pragma unroll
-            for (int p = 0; p < PASSES; ++p) {
-                unsigned km = kept[p];
-                while (km) {
-                    const int j = __ffs(km) - 1 + 32 * p;   // next kept token; its group = every token mapped to it
-                    km &= km - 1;
-                    float2 acc = make_float2(0.f, 0.f);
-                    int cnt = 0;
-#pragma unroll
-                    for (int pp = 0; pp < PASSES; ++pp) {
-                        unsigned mm = __ballot_sync(0xffffffffu, rep[pp] == j);
-                        cnt += __popc(mm);
-                        const uint32_t* xp = xs + (pp * 32) * 32 + lane;
-                        while (mm) {
-                            const int i0 = __ffs(mm) - 1;
-                            mm &= mm - 1;
-                            const uint32_t w0 = xp[i0 * 32];
-                            if (mm) {
-                                const int i1 = __ffs(mm) - 1;
-                                mm &= mm - 1;
-                                const uint32_t w1 = xp[i1 * 32];
-                                acc.x += __uint_as_float(w0 << 16);
-                                acc.y += __uint_as_float(w0 & 0xffff0000u);
-                                acc.x += __uint_as_float(w1 << 16);
-                                acc.y += __uint_as_float(w1 & 0xffff0000u);
-                            } else {
-                                acc.x += __uint_as_float(w0 << 16);
-                                acc.y += __uint_as_float(w0 & 0xffff0000u);
-                            }
-                        }
-                    }
-                    if (cnt > 1) {   // mean: quotient by reciprocal with one correction step
-                        const float c = (float)cnt, rc = 1.0f / c;
-                        float qx = acc.x * rc, qy = acc.y * rc;
-                        qx = fmaf(fmaf(-qx, c, acc.x), rc, qx);
-                        qy = fmaf(fmaf(-qy, c, acc.y), rc, qy);
-                        acc = make_float2(qx, qy);
-                    }
-                    const __nv_bfloat162 o = __floats2bfloat162_rn(acc.x, acc.y);
-                    if (row < n - u.r) out[row * 32 + lane] = *reinterpret_cast<const uint32_t*>(&o);   // (a corrupt map cannot overrun)
-                    ++row;
-                }
-            }
-        }
-        __syncwarp();   // every lane is done reading this stage buffer
-        if (lane == 0 && task + 2 * stride < n_tasks) issue(nxt, buf);
-    }
-    if (failed) {
-        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
-        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
-    }
 }
 
 // ------------------------------------------------------------------------------------
@@ -991,26 +801,226 @@ static cudaError_t launch_merge_tc(const MergeArgs& a, int sm_count, cudaStream_
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------
+// a3 (blocks of 33 to 256 tokens).  The same contraction as above, merged_sum = W x, for blocks that
+//     take several 32-token passes: lane l holds the map entries of tokens l, l + 32, ...; the kept rows
+//     are walked in tiles of 16, the tokens in steps of 16, and the x fragments are fetched per
+//     (row tile, token step) with ldmatrix.trans from the swizzled TMA stage (blocks come from the
+//     reordered copies).  Group sizes are counted with shared-memory atomics.
+// ------------------------------------------------------------------------------------
+__host__ __device__ constexpr int merge_multi_warps(int nmax) { return nmax <= 64 ? 8 : (nmax <= 128 ? 4 : 2); }
+__host__ __device__ constexpr int merge_multi_aux(int nmax) { return nmax * 8 + 16; }   // counts, reciprocals, 2 mbarriers
+__host__ __device__ constexpr int merge_multi_smem(int nmax) {
+    return merge_multi_warps(nmax) * (2 * nmax * kRowBytes + merge_multi_aux(nmax)) + 1024 /*alignment slack*/;
+}
+
 template <int PASSES>
-static cudaError_t launch_merge_t(const MergeArgs& a, int sm_count, cudaStream_t stream) {
+__global__ void __launch_bounds__(merge_multi_warps(32 * PASSES) * 32, 1)
+merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const MergeArgs a) {
     constexpr int NMAX = 32 * PASSES;
-    constexpr int WARPS = merge_warps_per_cta(NMAX);
-    const size_t smem = merge_smem_bytes(NMAX);
+    constexpr int WARPS = merge_multi_warps(NMAX);
+    constexpr int KS = NMAX / 16;   // token steps
+    constexpr uint32_t STAGE_BYTES = NMAX * kRowBytes;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;   // accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
+    unsigned char* stage = smem + (size_t)warp * 2 * STAGE_BYTES;                       // [2][NMAX][128], 1024-aligned, swizzled
+    unsigned char* aux = smem + (size_t)WARPS * 2 * STAGE_BYTES + (size_t)warp * merge_multi_aux(NMAX);
+    int* cnt = reinterpret_cast<int*>(aux);                                             // [NMAX] group size of kept row
+    float* rcnt = reinterpret_cast<float*>(aux + NMAX * 4);                             // [NMAX] its reciprocal
+    const uint32_t mbar0 = smem_u32(aux + NMAX * 8), stage0 = smem_u32(stage);
+
+    if (lane == 0) {
+        mbar_init(mbar0, 1);
+        mbar_init(mbar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    // task -> (tensor t, head h, unit u); units 0 .. n_blocks-1 are merging blocks, the rest are
+    // chunks of 32 special tokens (never merged: rows 0 .. n_special_total-1 are copied)
+    const int sp_chunks = (a.n_special_total + 31) / 32;
+    const int per_head = a.n_blocks + sp_chunks;
+    const int64_t n_tasks = 3ll * a.heads * per_head;
+    const int64_t stride = (int64_t)gridDim.x * WARPS;
+    const int64_t first = (int64_t)blockIdx.x * WARPS + warp;
+    TaskCursor cur, nxt;   // the task being processed; the task whose load is issued next
+    cur.init(first, stride, a.heads, per_head);
+    nxt = cur;
+
+    auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only; the whole NMAX-row box is transferred (rows past the head's end are zero filled)
+        const int start = c.u >= a.n_blocks ? (c.u - a.n_blocks) * 32 : __ldg(&a.blocks[c.u].start);
+        const uint32_t mb = mbar0 + 8 * buf;
+        mbar_expect_tx(mb, STAGE_BYTES);
+        tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, start, c.h);
+    };
+    if (first < n_tasks && lane == 0) issue(nxt, 0);
+    nxt.advance();
+    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+    nxt.advance();
+
+    int it = 0;
+    bool failed = false;
+    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
+        const int buf = it & 1;
+        const uint32_t parity = (it >> 1) & 1;
+        const bool more = task + 2 * stride < n_tasks;
+        const int t = cur.t, h = cur.h;
+        const bool special = cur.u >= a.n_blocks;
+        int start, n, r, moff;
+        if (special) {
+            start = (cur.u - a.n_blocks) * 32;
+            n = min(32, a.n_special_total - start);
+            r = 0;
+            moff = start;
+        } else {
+            const BlockInfo bi = a.blocks[cur.u];
+            start = bi.start;
+            n = bi.n;
+            r = t == 0 ? bi.r_q : bi.r_k;
+            moff = t == 0 ? bi.moff_q : bi.moff_k;
+        }
+        const int m_len = t == 0 ? a.m_q : a.m_k;
+        uint32_t* out = reinterpret_cast<uint32_t*>(a.merged[t] + ((int64_t)h * m_len + moff) * kHeadDim);   // 32 words per row
+        const uint32_t blk = stage0 + buf * STAGE_BYTES;
+
+        // the map entries do not depend on the staged rows: fetch them before waiting
+        int rep[PASSES];
+#pragma unroll
+        for (int p = 0; p < PASSES; ++p) {
+            const int j = lane + 32 * p;
+            rep[p] = -1;
+            if (r > 0 && j < n) {
+                rep[p] = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + j) - start;
+                if (rep[p] < 0 || rep[p] >= n) {   // corrupt map: record, treat as kept
+                    atomicCAS(a.status, kDevOk, kDevBadIndex);
+                    rep[p] = j;
+                }
+            }
+        }
+        if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
+            failed = true;
+            break;
+        }
+        if (r == 0) {   // nothing merges here: copy the rows, 16 bytes per lane (chunk c of row j sits at c ^ (j & 7))
+            const unsigned char* sb = stage + buf * STAGE_BYTES;
+            uint4* o4 = reinterpret_cast<uint4*>(out);
+            for (int q = lane; q < n * 8; q += 32) {
+                const int row = q >> 3, ch = q & 7;
+                o4[q] = *reinterpret_cast<const uint4*>(sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
+            }
+            if (t == 0 && !special)
+                for (int j = lane; j < n; j += 32) a.rank_q[(int64_t)h * a.n_tokens + start + j] = moff + j;
+        } else {
+            // merged row of every token: rank of its representative among the kept tokens
+            unsigned kept[PASSES];
+            int kept_before[PASSES], n_kept = 0;
+#pragma unroll
+            for (int p = 0; p < PASSES; ++p) {
+                kept[p] = __ballot_sync(0xffffffffu, rep[p] == lane + 32 * p);   // rep == -1 for positions >= n
+                kept_before[p] = n_kept;
+                n_kept += __popc(kept[p]);
+                cnt[lane + 32 * p] = 0;
+            }
+            __syncwarp();
+            int row_of[PASSES];
+#pragma unroll
+            for (int p = 0; p < PASSES; ++p) {
+                row_of[p] = -1;
+                if (rep[p] >= 0) {
+#pragma unroll
+                    for (int pp = 0; pp < PASSES; ++pp)
+                        if ((rep[p] >> 5) == pp) row_of[p] = kept_before[pp] + __popc(kept[pp] & ((1u << (rep[p] & 31)) - 1u));
+                    atomicAdd(&cnt[row_of[p]], 1);
+                    if (t == 0) a.rank_q[(int64_t)h * a.n_tokens + start + lane + 32 * p] = moff + row_of[p];
+                }
+            }
+            __syncwarp();
+#pragma unroll
+            for (int p = 0; p < PASSES; ++p)
+                if (lane + 32 * p < n_kept) rcnt[lane + 32 * p] = 1.0f / (float)cnt[lane + 32 * p];
+            __syncwarp();
+            const int n_ks = (n + 15) >> 4, n_mt = (n_kept + 15) >> 4;
+            const int n_out = min(n_kept, n - r);   // (a corrupt map cannot overrun)
+#pragma unroll 1
+            for (int mt = 0; mt < n_mt; ++mt) {
+                const int r0 = 16 * mt + g, r1 = r0 + 8;   // this lane's two accumulator rows
+                float c[8][4];
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    if (ks < n_ks) {   // warp-uniform
+                        // W fragment: rows of tokens 16 ks + {2 tq, 2 tq + 1, 2 tq + 8, 2 tq + 9} (held by pass ks / 2, lane 16 (ks & 1) + ..)
+                        const int src = 16 * (ks & 1) + 2 * tq;
+                        const int w0 = __shfl_sync(0xffffffffu, row_of[ks >> 1], src), w1 = __shfl_sync(0xffffffffu, row_of[ks >> 1], src + 1);
+                        const int w2 = __shfl_sync(0xffffffffu, row_of[ks >> 1], src + 8), w3 = __shfl_sync(0xffffffffu, row_of[ks >> 1], src + 9);
+                        uint32_t af[4];   // bf16 1.0 = 0x3f80
+                        af[0] = (w0 == r0 ? 0x3f80u : 0u) | (w1 == r0 ? 0x3f800000u : 0u);
+                        af[1] = (w0 == r1 ? 0x3f80u : 0u) | (w1 == r1 ? 0x3f800000u : 0u);
+                        af[2] = (w2 == r0 ? 0x3f80u : 0u) | (w3 == r0 ? 0x3f800000u : 0u);
+                        af[3] = (w2 == r1 ? 0x3f80u : 0u) | (w3 == r1 ? 0x3f800000u : 0u);
+                        if (__any_sync(0xffffffffu, (af[0] | af[1] | af[2] | af[3]) != 0u)) {   // no token of this step belongs to this row tile: skip
+                            const int tok = 16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8;
+                            const uint32_t rowaddr = blk + tok * kRowBytes;
+#pragma unroll
+                            for (int np = 0; np < 4; ++np) {
+                                uint32_t bf[4];
+                                ldmatrix_x4_trans(bf, rowaddr + (((2 * np + (lane >> 4)) ^ (tok & 7)) << 4));
+                                mma_bf16_16816(c[2 * np], af, bf[0], bf[1]);
+                                mma_bf16_16816(c[2 * np + 1], af, bf[2], bf[3]);
+                            }
+                        }
+                    }
+                }
+                const bool s0 = r0 < n_out, s1 = r1 < n_out;
+                const float i0 = s0 ? rcnt[r0] : 0.f, i1 = s1 ? rcnt[r1] : 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {
+                    if (s0) {
+                        const __nv_bfloat162 o = __floats2bfloat162_rn(c[nt][0] * i0, c[nt][1] * i0);
+                        out[r0 * 32 + nt * 4 + tq] = *reinterpret_cast<const uint32_t*>(&o);
+                    }
+                    if (s1) {
+                        const __nv_bfloat162 o = __floats2bfloat162_rn(c[nt][2] * i1, c[nt][3] * i1);
+                        out[r1 * 32 + nt * 4 + tq] = *reinterpret_cast<const uint32_t*>(&o);
+                    }
+                }
+            }
+        }
+        __syncwarp();   // every lane is done reading this stage buffer and the per-row tables
+        if (more && lane == 0) issue(nxt, buf);
+    }
+    if (failed) {
+        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+    }
+}
+
+template <int PASSES>
+static cudaError_t launch_merge_multi(const MergeArgs& a, int sm_count, cudaStream_t stream) {
+    constexpr int NMAX = 32 * PASSES;
+    constexpr int WARPS = merge_multi_warps(NMAX);
+    CUtensorMap m[3];
+    const int64_t N = a.n_tokens;
+    for (int t = 0; t < 3; ++t)
+        if (!encode_rows_tensor_map(&m[t], a.xr[t], N, a.heads, kHeadDim, N * kHeadDim, NMAX)) return cudaErrorInvalidValue;
     const int64_t n_tasks = 3ll * a.heads * (a.n_blocks + (a.n_special_total + 31) / 32);
-    int ctas_per_sm = (int)((224 * 1024) / (smem + 1024));
-    ctas_per_sm = ctas_per_sm < 1 ? 1 : (ctas_per_sm > 64 / WARPS ? 64 / WARPS : ctas_per_sm);
     int64_t grid = (n_tasks + WARPS - 1) / WARPS;
-    const int64_t cap = (int64_t)sm_count * ctas_per_sm;
-    if (grid > cap) grid = cap;
+    if (grid > sm_count) grid = sm_count;
     if (grid < 1) grid = 1;
-    merge_kernel<PASSES><<<(unsigned)grid, WARPS * 32, smem, stream>>>(a);
+    merge_multi_kernel<PASSES><<<(unsigned)grid, WARPS * 32, merge_multi_smem(NMAX), stream>>>(m[0], m[1], m[2], a);
     return cudaGetLastError();
 }
 
 cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream) {
-    if (max_block_tokens <= 32) return launch_merge_tc(a, sm_count, stream);   // tensor-core kernel
-    if (max_block_tokens <= 128) return launch_merge_t<4>(a, sm_count, stream);
-    return launch_merge_t<8>(a, sm_count, stream);
+    if (max_block_tokens <= 32) return launch_merge_tc(a, sm_count, stream);
+    if (max_block_tokens <= 64) return launch_merge_multi<2>(a, sm_count, stream);
+    if (max_block_tokens <= 128) return launch_merge_multi<4>(a, sm_count, stream);
+    return launch_merge_multi<8>(a, sm_count, stream);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1069,12 +1079,14 @@ cudaError_t configure_kernels() {
     if (e != cudaSuccess) return e;
     HTTM_SET_SMEM((match_kernel<1, false>), match_smem_bytes(32));
     HTTM_SET_SMEM((match_kernel<1, true>), match_smem_bytes(32));
+    HTTM_SET_SMEM((match_kernel<2, false>), match_smem_bytes(64));
     HTTM_SET_SMEM((match_kernel<4, false>), match_smem_bytes(128));
     HTTM_SET_SMEM((match_kernel<8, false>), match_smem_bytes(256));
     HTTM_SET_SMEM(merge_tc_kernel<false>, kMergeTcSmem);
     HTTM_SET_SMEM(merge_tc_kernel<true>, kMergeTcSmem);
-    HTTM_SET_SMEM(merge_kernel<4>, merge_smem_bytes(128));
-    HTTM_SET_SMEM(merge_kernel<8>, merge_smem_bytes(256));
+    HTTM_SET_SMEM(merge_multi_kernel<2>, merge_multi_smem(64));
+    HTTM_SET_SMEM(merge_multi_kernel<4>, merge_multi_smem(128));
+    HTTM_SET_SMEM(merge_multi_kernel<8>, merge_multi_smem(256));
 #undef HTTM_SET_SMEM
     return configure_attention();
 }
