@@ -173,6 +173,29 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def rank_barrier(world):
+    """All replicas meet here (nothing else is exchanged: the path has no collective)."""
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def rank_max(x, world, device="cpu"):
+    """The slowest replica's time: the figure a multi-replica run reports."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(tokens_per_replica, world, ms_step):
+    """Whole-job tokens/s of `world` independent replicas timed at `ms_step` (the maximum over the replicas)."""
+    return world * tokens_per_replica / (ms_step * 1e-3)
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
@@ -189,16 +212,11 @@ def run_ours(args, wl):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        rank_barrier(world)
         torch.cuda.synchronize()
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return rank_max(x, world, dev)
 
     q, k, v = synth.make_qkv(wl)
     ctx = hb.Httm(hb.HttmConfig.of(wl, device=local))
@@ -307,11 +325,11 @@ def run_ours(args, wl):
                     "peak_source": peaks["source"] + " (sustained bf16 GEMM; kernel timed inside the step)",
                     "traffic": ATTENTION_DRAM_TRAFFIC.get(wl.name)}
         line = {
-            "metric": METRIC, "value": world * N / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": replica_throughput(N, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(wl),
             "clocks": clocks,
-            "e2e": {"value": world * N / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": replica_throughput(N, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 3 * H * N * D * b, "d2h_bytes_per_step": H * N * D * b, "steps": esteps,
                     "matches_device_path": same},
             "gpu_launches": int(launches),
