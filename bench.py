@@ -135,7 +135,7 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile(prefix="clocks_", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -398,7 +398,7 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args, wl)
     else:
-        args.steps = 50 if args.steps is None else args.steps
+        args.steps = 400 if args.steps is None else args.steps   # ~0.3 s timed: several clock samples fall inside
         args.warmup = 5 if args.warmup is None else args.warmup
         run_ours(args, wl)
 

@@ -269,3 +269,13 @@ def test_direct_block_loads_equal_the_reordered_copies():
                     assert np.array_equal(sep[n], direct[n]), f"{wl.name}: {n} differs"
                 else:
                     assert (np.abs(a - b) <= 2.0 ** -7 * np.abs(a) + 1e-30).all(), f"{wl.name}: {n} differs by more than a bf16 step"
+
+
+def test_large_config_full_size_sampled():
+    """S=100 frames (137k tokens), 64-token blocks, weaker redundancy: the kernels for blocks of more than 32 tokens at
+    full size - maps, ranks and merged tensors in full, attention on sampled tokens."""
+    wl = synth.WORKLOADS["large"]
+    rng = np.random.default_rng(4)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 16), np.arange(5), [wl.n_tokens - 1]]))
+    stats = run_case(wl, sample=toks)
+    assert stats["merged_exactly_rounded"] > 0.99
