@@ -637,49 +637,79 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
     nxt.advance();
 
+    // Everything a task needs besides the staged rows: its place in the tables, and this lane's map entry.
+    // Both are fetched one task ahead (table entry at the start of the previous task, map entry behind its
+    // MMAs), so that their global-memory latency is not paid between waiting for a stage and using it.
+    struct Meta {
+        int t, h, start, n, r, moff;
+        bool special;
+        BlockGeom bg;
+    };
+    auto load_meta = [&](const TaskCursor& c) {
+        Meta m{};
+        m.t = c.t;
+        m.h = c.h;
+        m.special = c.u >= a.n_blocks;
+        if (m.special) {
+            m.start = DIRECT ? (c.u - a.n_blocks) * a.layout.n_special : (c.u - a.n_blocks) * 32;
+            m.n = DIRECT ? a.layout.n_special : min(32, a.n_special_total - m.start);
+            m.r = 0;
+            m.moff = m.start;
+        } else {
+            if (DIRECT) m.bg = a.geom[c.u];
+            const BlockInfo bi = a.blocks[c.u];
+            m.start = bi.start;
+            m.n = bi.n;
+            m.r = c.t == 0 ? bi.r_q : bi.r_k;
+            m.moff = c.t == 0 ? bi.moff_q : bi.moff_k;
+        }
+        return m;
+    };
+    // lane = row of the stage; number of the token it holds in the block (-1: none)
+    auto token_of_lane = [&](const Meta& m) {
+        return !DIRECT || m.special ? (lane < m.n ? lane : -1)
+                                    : ((own_t < m.bg.frames && own_y < m.bg.rows && own_x < m.bg.cols) ? (own_t * m.bg.rows + own_y) * m.bg.cols + own_x : -1);
+    };
+    auto load_target = [&](const Meta& m) {   // token this lane's token is merged into (number in the block), -1 if the lane holds none
+        const int tok = token_of_lane(m);
+        return m.r > 0 && tok >= 0 ? __ldg(a.assign[m.t == 0 ? 0 : 1] + (int64_t)m.h * a.n_tokens + m.start + tok) - m.start : -1;
+    };
+    Meta meta_next{};
+    int target_next = -1;
+    if (first < n_tasks) {
+        meta_next = load_meta(cur);
+        target_next = load_target(meta_next);
+    }
+    TaskCursor ahead = cur;   // the task after the current one
+    ahead.advance();
+
     int it = 0;
     bool failed = false;
-    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
+    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance(), ahead.advance()) {
         const int buf = it & 1;
         const uint32_t parity = (it >> 1) & 1;
-        const bool more = task + 2 * stride < n_tasks;
-        const int t = cur.t, h = cur.h;
-        const bool special = cur.u >= a.n_blocks;
-        int start, n, r, moff;
-        BlockGeom bg{};
-        if (special) {
-            start = DIRECT ? (cur.u - a.n_blocks) * a.layout.n_special : (cur.u - a.n_blocks) * 32;
-            n = DIRECT ? a.layout.n_special : min(32, a.n_special_total - start);
-            r = 0;
-            moff = start;
-            bm.clipped = false;
-        } else {
-            if (DIRECT) {
-                bg = a.geom[cur.u];
-                bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
-            }
-            const BlockInfo bi = a.blocks[cur.u];
-            start = bi.start;
-            n = bi.n;
-            r = t == 0 ? bi.r_q : bi.r_k;
-            moff = t == 0 ? bi.moff_q : bi.moff_k;
-        }
+        const bool more = task + 2 * stride < n_tasks, has_next = task + stride < n_tasks;
+        const Meta meta = meta_next;
+        int rep = target_next;
+        if (has_next) meta_next = load_meta(ahead);   // in flight while this task is processed
+        const int t = meta.t, h = meta.h, start = meta.start, n = meta.n, r = meta.r, moff = meta.moff;
+        const bool special = meta.special;
+        const BlockGeom bg = meta.bg;
+        if (DIRECT && !special) bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
+        if (special) bm.clipped = false;
         const int m_len = t == 0 ? a.m_q : a.m_k;
         uint32_t* out = reinterpret_cast<uint32_t*>(a.merged[t] + ((int64_t)h * m_len + moff) * kHeadDim);   // 32 words per row
         const uint32_t blk = stage0 + buf * STAGE_BYTES;
-
-        // the map entry does not depend on the staged rows: fetch it before waiting
-        // lane = row of the stage; tok = number of the token it holds (-1: none); rep = ROW of the token it is merged into
-        const int tok = !DIRECT || special ? (lane < n ? lane : -1)
-                                           : ((own_t < bg.frames && own_y < bg.rows && own_x < bg.cols) ? (own_t * bg.rows + own_y) * bg.cols + own_x : -1);
-        int rep = -1;
+        const int tok = token_of_lane(meta);
+        // rep = ROW of the stage holding the token this lane's token is merged into
         if (r > 0 && tok >= 0) {
-            rep = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + tok) - start;
             if (rep < 0 || rep >= n) {   // corrupt map: record, treat as kept
                 atomicCAS(a.status, kDevOk, kDevBadIndex);
                 rep = tok;
             }
             if (DIRECT) rep = bm.row_of_token(rep);
+        } else {
+            rep = -1;
         }
         if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
             failed = true;
@@ -693,6 +723,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 o4[q] = *reinterpret_cast<const uint4*>(sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
             }
             if (t == 0 && !special && lane < n) a.rank_q[(int64_t)h * a.n_tokens + start + lane] = moff + lane;
+            if (has_next) target_next = load_target(meta_next);
         } else {
             // merged row of every token: rank of its representative among the kept tokens
             const unsigned kept = __ballot_sync(0xffffffffu, rep == lane);   // rep == -1 for lanes >= n
@@ -745,6 +776,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                             mma_bf16_16816(c[nt], af, bf[ks][nt >> 1][2 * (nt & 1)], bf[ks][nt >> 1][2 * (nt & 1) + 1]);
                     }
                 }
+                if (mt == 0 && has_next) target_next = load_target(meta_next);   // behind this task's MMAs
                 const bool w0 = r0 < n_kept && r0 < n - r, w1 = r1 < n_kept && r1 < n - r;   // (a corrupt map cannot overrun)
                 const float i0 = w0 ? rcnt[r0] : 0.f, i1 = w1 ? rcnt[r1] : 0.f;
 #pragma unroll
