@@ -258,6 +258,9 @@ def test_direct_block_loads_equal_the_reordered_copies():
             for st in (hb.STAGE_REORDER, hb.STAGE_MATCH, hb.STAGE_MERGE):
                 ctx.launch_stage(st, dq, dk, dv)
             sep = {n: ctx.export(w).copy() for n, w in names.items()}
+            # other inputs through the separate kernels: nothing of the first run is left in the buffers
+            for st in (hb.STAGE_REORDER, hb.STAGE_MATCH, hb.STAGE_MERGE):
+                ctx.launch_stage(st, dv, dq, dk)
             for st in (hb.STAGE_MATCH_DIRECT, hb.STAGE_MERGE_DIRECT):
                 ctx.launch_stage(st, dq, dk, dv)
             direct = {n: ctx.export(w) for n, w in names.items()}
