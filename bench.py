@@ -247,7 +247,7 @@ def run_ours(args, wl):
     # ---- per-kernel durations: every kernel of the path launched on its own with events between them.
     #      Order: reorder, match, merge (the separate kernels), then - where the geometry allows it - match and
     #      merge reading their blocks straight from Q/K/V (the two that the public call uses), attention, unmerge.
-    direct = ctx.query(hb.Q_MAX_BLOCK_TOKENS) <= 32
+    direct = True   # every supported geometry has the direct kernels
     order = [0, 1, 2] + ([5, 6] if direct else []) + [3, 4]
     stage_ms = {st: 0.0 for st in order}
     evs = [[ev() for _ in range(len(order) + 1)] for _ in range(args.steps)]

@@ -171,9 +171,9 @@ SourceLayout source_layout(const httm_ctx* c) {
     return L;
 }
 
-// Blocks of at most 32 tokens are read by the match and merge kernels straight from Q/K/V (tiled TMA loads of
-// the block's patch window): the reordered copies are then not needed on the hot path.
-bool direct_mode(const httm_ctx* c) { return c->max_block <= 32 && c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767; }
+// The match and merge kernels read every block straight from Q/K/V (tiled TMA loads of the block's patch window):
+// the reordered copies are not needed on the hot path (the 16-bit block coordinates bound the scene size).
+bool direct_mode(const httm_ctx* c) { return c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767; }
 
 // src: the original Q, K, V (direct mode) or nullptr (blocks come from the reordered copies)
 int stage_match(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
@@ -499,7 +499,7 @@ int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm
             return stage_unmerge(c, out, s);
         case HTTM_STAGE_MATCH_DIRECT:
         case HTTM_STAGE_MERGE_DIRECT: {
-            if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "direct stages need merging blocks of at most 32 tokens");
+            if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "direct stages need a scene of at most 32767 frames / patch rows / patch columns");
             if ((rc = check_tensor(c, q, "q")) || (rc = check_tensor(c, k, "k")) || (rc = check_tensor(c, v, "v"))) return rc;
             const httm_tensor src[3] = {q, k, v};
             return stage == HTTM_STAGE_MATCH_DIRECT ? stage_match(c, s, src) : stage_merge(c, s, src);

@@ -520,7 +520,7 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = match_warps_per_cta(NMAX);
     const size_t smem = match_smem_bytes(NMAX);
-    const bool direct = a.geom != nullptr && PASSES == 1;
+    const bool direct = a.geom != nullptr;
     CUtensorMap mq, mk;
     const int64_t N = a.n_tokens;
     if (direct) {
@@ -537,7 +537,7 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
     if (grid > cap) grid = cap;
     if (grid < 1) grid = 1;
     if (direct)
-        match_kernel<1, true><<<(unsigned)grid, match_warps_per_cta(32) * 32, match_smem_bytes(32), stream>>>(mq, mk, a);
+        match_kernel<PASSES, true><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
     else
         match_kernel<PASSES, false><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
     return cudaGetLastError();
@@ -846,10 +846,11 @@ __host__ __device__ constexpr int merge_multi_smem(int nmax) {
     return merge_multi_warps(nmax) * (2 * nmax * kRowBytes + merge_multi_aux(nmax)) + 1024 /*alignment slack*/;
 }
 
-template <int PASSES>
+template <int PASSES, bool DIRECT>
 __global__ void __launch_bounds__(merge_multi_warps(32 * PASSES) * 32, 1)
 merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                   const __grid_constant__ CUtensorMap map_v, const MergeArgs a) {
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_sq,
+                   const __grid_constant__ CUtensorMap map_sk, const __grid_constant__ CUtensorMap map_sv, const MergeArgs a) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = merge_multi_warps(NMAX);
     constexpr int KS = NMAX / 16;   // token steps
@@ -874,8 +875,22 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     // task -> (tensor t, head h, unit u); units 0 .. n_blocks-1 are merging blocks, the rest are
     // chunks of 32 special tokens (never merged: rows 0 .. n_special_total-1 are copied)
-    const int sp_chunks = (a.n_special_total + 31) / 32;
+    const int sp_chunks = DIRECT ? (a.layout.n_special > 0 ? a.layout.frames : 0) : (a.n_special_total + 31) / 32;
     const int per_head = a.n_blocks + sp_chunks;
+    // direct mode: box extents and the box coordinates of the stage rows lane + 32 p
+    const int box_f = DIRECT ? min(a.layout.blk_frames, a.layout.frames) : 1, box_h = DIRECT ? min(a.layout.blk_h, a.layout.grid_h) : 1,
+              box_w = DIRECT ? min(a.layout.blk_w, a.layout.grid_w) : 1;
+    const int box_rows = box_f * box_h * box_w;
+    int own_t[PASSES], own_y[PASSES], own_x[PASSES];
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) {
+        const int rho = lane + 32 * p;
+        own_t[p] = DIRECT ? rho / (box_h * box_w) : 0;
+        own_y[p] = DIRECT ? (rho / box_w) % box_h : 0;
+        own_x[p] = DIRECT ? rho % box_w : 0;
+    }
+    BoxMap bm;
+    bm.clipped = false;
     const int64_t n_tasks = 3ll * a.heads * per_head;
     const int64_t stride = (int64_t)gridDim.x * WARPS;
     const int64_t first = (int64_t)blockIdx.x * WARPS + warp;
@@ -884,10 +899,23 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     nxt = cur;
 
     auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only; the whole NMAX-row box is transferred (rows past the head's end are zero filled)
-        const int start = c.u >= a.n_blocks ? (c.u - a.n_blocks) * 32 : __ldg(&a.blocks[c.u].start);
         const uint32_t mb = mbar0 + 8 * buf;
-        mbar_expect_tx(mb, STAGE_BYTES);
-        tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, start, c.h);
+        if (!DIRECT) {
+            const int start = c.u >= a.n_blocks ? (c.u - a.n_blocks) * 32 : __ldg(&a.blocks[c.u].start);
+            mbar_expect_tx(mb, STAGE_BYTES);
+            tma_rows_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, start, c.h);
+        } else if (c.u >= a.n_blocks) {   // the special tokens of frame u - n_blocks
+            mbar_expect_tx(mb, (uint32_t)a.layout.n_special * kRowBytes);
+            const CUtensorMap* m = c.t == 0 ? &map_sq : (c.t == 1 ? &map_sk : &map_sv);
+            asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+                             stage0 + buf * STAGE_BYTES),
+                         "l"(reinterpret_cast<uint64_t>(m)), "r"(mb), "r"(0), "r"(0), "r"(c.u - a.n_blocks), "r"(c.h)
+                         : "memory");
+        } else {
+            const BlockGeom bg = a.geom[c.u];
+            mbar_expect_tx(mb, (uint32_t)box_rows * kRowBytes);
+            tma_block_load(stage0 + buf * STAGE_BYTES, c.t == 0 ? &map_q : (c.t == 1 ? &map_k : &map_v), mb, bg.x0, bg.y0, bg.s0, c.h);
+        }
     };
     if (first < n_tasks && lane == 0) issue(nxt, 0);
     nxt.advance();
@@ -903,12 +931,18 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int t = cur.t, h = cur.h;
         const bool special = cur.u >= a.n_blocks;
         int start, n, r, moff;
+        BlockGeom bg{};
+        bm.clipped = false;
         if (special) {
-            start = (cur.u - a.n_blocks) * 32;
-            n = min(32, a.n_special_total - start);
+            start = DIRECT ? (cur.u - a.n_blocks) * a.layout.n_special : (cur.u - a.n_blocks) * 32;
+            n = DIRECT ? a.layout.n_special : min(32, a.n_special_total - start);
             r = 0;
             moff = start;
         } else {
+            if (DIRECT) {
+                bg = a.geom[cur.u];
+                bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
+            }
             const BlockInfo bi = a.blocks[cur.u];
             start = bi.start;
             n = bi.n;
@@ -920,17 +954,21 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t blk = stage0 + buf * STAGE_BYTES;
 
         // the map entries do not depend on the staged rows: fetch them before waiting
-        int rep[PASSES];
+        // stage row lane + 32 p holds token tok[p] of the block (-1: none), merged into the token in stage ROW rep[p]
+        int rep[PASSES], tok[PASSES];
 #pragma unroll
         for (int p = 0; p < PASSES; ++p) {
-            const int j = lane + 32 * p;
+            const int rho = lane + 32 * p;
+            tok[p] = !DIRECT || special ? (rho < n ? rho : -1)
+                                        : ((own_t[p] < bg.frames && own_y[p] < bg.rows && own_x[p] < bg.cols) ? (own_t[p] * bg.rows + own_y[p]) * bg.cols + own_x[p] : -1);
             rep[p] = -1;
-            if (r > 0 && j < n) {
-                rep[p] = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + j) - start;
+            if (r > 0 && tok[p] >= 0) {
+                rep[p] = __ldg(a.assign[t == 0 ? 0 : 1] + (int64_t)h * a.n_tokens + start + tok[p]) - start;
                 if (rep[p] < 0 || rep[p] >= n) {   // corrupt map: record, treat as kept
                     atomicCAS(a.status, kDevOk, kDevBadIndex);
-                    rep[p] = j;
+                    rep[p] = tok[p];
                 }
+                if (DIRECT) rep[p] = bm.row_of_token(rep[p]);
             }
         }
         if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
@@ -941,7 +979,7 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const unsigned char* sb = stage + buf * STAGE_BYTES;
             uint4* o4 = reinterpret_cast<uint4*>(out);
             for (int q = lane; q < n * 8; q += 32) {
-                const int row = q >> 3, ch = q & 7;
+                const int row = DIRECT ? bm.row_of_token(q >> 3) : q >> 3, ch = q & 7;
                 o4[q] = *reinterpret_cast<const uint4*>(sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
             }
             if (t == 0 && !special)
@@ -967,7 +1005,7 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     for (int pp = 0; pp < PASSES; ++pp)
                         if ((rep[p] >> 5) == pp) row_of[p] = kept_before[pp] + __popc(kept[pp] & ((1u << (rep[p] & 31)) - 1u));
                     atomicAdd(&cnt[row_of[p]], 1);
-                    if (t == 0) a.rank_q[(int64_t)h * a.n_tokens + start + lane + 32 * p] = moff + row_of[p];
+                    if (t == 0) a.rank_q[(int64_t)h * a.n_tokens + start + tok[p]] = moff + row_of[p];
                 }
             }
             __syncwarp();
@@ -975,7 +1013,7 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int p = 0; p < PASSES; ++p)
                 if (lane + 32 * p < n_kept) rcnt[lane + 32 * p] = 1.0f / (float)cnt[lane + 32 * p];
             __syncwarp();
-            const int n_ks = (n + 15) >> 4, n_mt = (n_kept + 15) >> 4;
+            const int n_ks = ((DIRECT ? box_rows : n) + 15) >> 4, n_mt = (n_kept + 15) >> 4;   // stage rows that may hold tokens
             const int n_out = min(n_kept, n - r);   // (a corrupt map cannot overrun)
 #pragma unroll 1
             for (int mt = 0; mt < n_mt; ++mt) {
@@ -1036,15 +1074,31 @@ template <int PASSES>
 static cudaError_t launch_merge_multi(const MergeArgs& a, int sm_count, cudaStream_t stream) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = merge_multi_warps(NMAX);
-    CUtensorMap m[3];
+    CUtensorMap m[3], sp[3];
     const int64_t N = a.n_tokens;
-    for (int t = 0; t < 3; ++t)
-        if (!encode_rows_tensor_map(&m[t], a.xr[t], N, a.heads, kHeadDim, N * kHeadDim, NMAX)) return cudaErrorInvalidValue;
-    const int64_t n_tasks = 3ll * a.heads * (a.n_blocks + (a.n_special_total + 31) / 32);
+    const bool direct = a.geom != nullptr;
+    for (int t = 0; t < 3; ++t) {
+        if (direct) {
+            if (!encode_block_map(&m[t], a.src[t], a.layout, a.heads)) return cudaErrorInvalidValue;
+            if (a.layout.n_special > 0 &&
+                !encode_frame_tensor_map(&sp[t], a.src[t].ptr, a.layout.tokens_per_frame, a.layout.frames, a.heads, a.src[t].stride_token,
+                                         a.src[t].stride_head, a.layout.n_special))
+                return cudaErrorInvalidValue;
+            if (a.layout.n_special <= 0) sp[t] = m[t];   // never used
+        } else {
+            if (!encode_rows_tensor_map(&m[t], a.xr[t], N, a.heads, kHeadDim, N * kHeadDim, NMAX)) return cudaErrorInvalidValue;
+            sp[t] = m[t];   // not used
+        }
+    }
+    const int sp_units = direct ? (a.layout.n_special > 0 ? a.layout.frames : 0) : (a.n_special_total + 31) / 32;
+    const int64_t n_tasks = 3ll * a.heads * (a.n_blocks + sp_units);
     int64_t grid = (n_tasks + WARPS - 1) / WARPS;
     if (grid > sm_count) grid = sm_count;
     if (grid < 1) grid = 1;
-    merge_multi_kernel<PASSES><<<(unsigned)grid, WARPS * 32, merge_multi_smem(NMAX), stream>>>(m[0], m[1], m[2], a);
+    if (direct)
+        merge_multi_kernel<PASSES, true><<<(unsigned)grid, WARPS * 32, merge_multi_smem(NMAX), stream>>>(m[0], m[1], m[2], sp[0], sp[1], sp[2], a);
+    else
+        merge_multi_kernel<PASSES, false><<<(unsigned)grid, WARPS * 32, merge_multi_smem(NMAX), stream>>>(m[0], m[1], m[2], sp[0], sp[1], sp[2], a);
     return cudaGetLastError();
 }
 
@@ -1112,13 +1166,19 @@ cudaError_t configure_kernels() {
     HTTM_SET_SMEM((match_kernel<1, false>), match_smem_bytes(32));
     HTTM_SET_SMEM((match_kernel<1, true>), match_smem_bytes(32));
     HTTM_SET_SMEM((match_kernel<2, false>), match_smem_bytes(64));
+    HTTM_SET_SMEM((match_kernel<2, true>), match_smem_bytes(64));
+    HTTM_SET_SMEM((match_kernel<4, true>), match_smem_bytes(128));
+    HTTM_SET_SMEM((match_kernel<8, true>), match_smem_bytes(256));
     HTTM_SET_SMEM((match_kernel<4, false>), match_smem_bytes(128));
     HTTM_SET_SMEM((match_kernel<8, false>), match_smem_bytes(256));
     HTTM_SET_SMEM(merge_tc_kernel<false>, kMergeTcSmem);
     HTTM_SET_SMEM(merge_tc_kernel<true>, kMergeTcSmem);
-    HTTM_SET_SMEM(merge_multi_kernel<2>, merge_multi_smem(64));
-    HTTM_SET_SMEM(merge_multi_kernel<4>, merge_multi_smem(128));
-    HTTM_SET_SMEM(merge_multi_kernel<8>, merge_multi_smem(256));
+    HTTM_SET_SMEM((merge_multi_kernel<2, false>), merge_multi_smem(64));
+    HTTM_SET_SMEM((merge_multi_kernel<4, false>), merge_multi_smem(128));
+    HTTM_SET_SMEM((merge_multi_kernel<8, false>), merge_multi_smem(256));
+    HTTM_SET_SMEM((merge_multi_kernel<2, true>), merge_multi_smem(64));
+    HTTM_SET_SMEM((merge_multi_kernel<4, true>), merge_multi_smem(128));
+    HTTM_SET_SMEM((merge_multi_kernel<8, true>), merge_multi_smem(256));
 #undef HTTM_SET_SMEM
     return configure_attention();
 }

@@ -244,12 +244,14 @@ def test_dense_attention_medium_config_sampled():
 
 
 def test_direct_block_loads_equal_the_reordered_copies():
-    """Match and merge reading their blocks straight from Q/K/V (what the public call does for blocks of
-    at most 32 tokens) against the same kernels reading the reorder kernel's copies: identical maps and
+    """Match and merge reading their blocks straight from Q/K/V (what the public call does) against the same kernels reading the reorder kernel's copies: identical maps and
     ranks; merged values identical where no block is clipped, within one bf16 step elsewhere (the order
     in which a clipped block's tokens enter the fp32 sums differs)."""
     for wl in (synth.WORKLOADS["tiny"].replace(heads=3),
-               synth.Workload("clipped", 5, 9, 10, 2, 4, 4, 0.6, 0.7, heads=3, seed=7)):
+               synth.Workload("clipped", 5, 9, 10, 2, 4, 4, 0.6, 0.7, heads=3, seed=7),
+               synth.Workload("clipped", 9, 10, 11, 4, 4, 4, 0.5, 0.8, heads=2, seed=8),     # 64-token blocks
+               synth.Workload("clipped", 5, 17, 19, 2, 8, 8, 0.7, 0.9, heads=2, seed=9),     # 128
+               synth.Workload("clipped", 5, 9, 11, 4, 8, 8, 0.8, 0.3, heads=1, seed=10)):    # 256
         q, k, v = synth.make_qkv(wl)
         with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
             dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
