@@ -149,9 +149,14 @@ int httm_dense_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tenso
  * The same two operations for callers whose tensors live in HOST memory (pinned memory
  * makes the copies asynchronous).  q, k, v: bf16 [heads][N][head_dim] contiguous;
  * out: bf16 [N][heads*head_dim] contiguous.  Each call copies the inputs to
- * context-owned device buffers (allocated at the first such call), runs the path and
- * copies the result back, all on `stream`; the caller synchronises the stream before
- * reading `out`.  dense != 0 selects httm_dense_attention.
+ * context-owned device buffers, runs the path on `stream` and copies the result back;
+ * the caller synchronises `stream` before reading `out`.  The copies run on two streams
+ * of the context's own over two sets of buffers (all created at the first such call),
+ * so that consecutive calls overlap: one call's host-to-device copy runs during the
+ * previous call's kernels and device-to-host copy.  Consequences: the input buffers
+ * must hold their data when the call is made (their copy does not wait for earlier
+ * work on `stream`) and must stay unchanged, like `out` unread, until `stream` has
+ * been synchronised.  dense != 0 selects httm_dense_attention.
  * Errors: INVALID_ARG, NOMEM, CUDA.
  */
 int httm_attention_host(httm_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,

@@ -46,7 +46,15 @@ struct httm_ctx {
     __nv_bfloat16 *d_qr = nullptr, *d_kr = nullptr, *d_vr = nullptr;
     __nv_bfloat16 *d_qm = nullptr, *d_km = nullptr, *d_vm = nullptr, *d_om = nullptr;
     // staging for the host-buffer entry point (allocated on first use)
-    __nv_bfloat16 *d_hq = nullptr, *d_hk = nullptr, *d_hv = nullptr, *d_hout = nullptr;
+    // Two sets of device buffers, two copy streams and events, so that one call's host-to-device copy overlaps the
+    // previous call's kernels and device-to-host copy (PCIe is full duplex; the copies are 6x the kernel time).
+    struct HostSet {
+        __nv_bfloat16 *q = nullptr, *k = nullptr, *v = nullptr, *out = nullptr;
+        cudaEvent_t loaded = nullptr, consumed = nullptr, computed = nullptr, returned = nullptr;
+        bool used = false;
+    } hs[2];
+    cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+    int64_t host_calls = 0;
     int64_t workspace_bytes = 0;
     int64_t launches = 0;
     std::string error;
@@ -75,9 +83,14 @@ struct httm_ctx {
     }
     void release() {
         void* ptrs[] = {d_geom, d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
-                        d_vr, d_qm,     d_km,       d_vm,       d_om,     d_hq,     d_hk,     d_hv, d_hout};
+                        d_vr, d_qm,     d_km,       d_vm,       d_om,     hs[0].q,  hs[0].k,  hs[0].v, hs[0].out, hs[1].q, hs[1].k, hs[1].v, hs[1].out};
         for (void* p : ptrs)
             if (p) cudaFree(p);
+        for (HostSet& h : hs)
+            for (cudaEvent_t e : {h.loaded, h.consumed, h.computed, h.returned})
+                if (e) cudaEventDestroy(e);
+        if (s_h2d) cudaStreamDestroy(s_h2d);
+        if (s_d2h) cudaStreamDestroy(s_d2h);
     }
 };
 
@@ -460,22 +473,48 @@ int httm_attention_host(httm_ctx* c, const void* q_host, const void* k_host, con
     if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
     const size_t elems = (size_t)c->cfg.heads * c->n_tokens * kHeadDim;
     int rc;
-    if (!c->d_hq) {
-        if ((rc = c->alloc(&c->d_hq, elems)) || (rc = c->alloc(&c->d_hk, elems)) || (rc = c->alloc(&c->d_hv, elems)) ||
-            (rc = c->alloc(&c->d_hout, elems)))
-            return rc;
+    if (!c->s_h2d) {   // first call: buffers, streams, events
+        for (httm_ctx::HostSet& h : c->hs)
+            if ((rc = c->alloc(&h.q, elems)) || (rc = c->alloc(&h.k, elems)) || (rc = c->alloc(&h.v, elems)) || (rc = c->alloc(&h.out, elems)))
+                return rc;
+        cudaError_t e = cudaStreamCreateWithFlags(&c->s_h2d, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->s_d2h, cudaStreamNonBlocking);
+        for (httm_ctx::HostSet& h : c->hs)
+            for (cudaEvent_t* ev : {&h.loaded, &h.consumed, &h.computed, &h.returned})
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+        if ((rc = check_cuda(c, e, "copy streams and events"))) return rc;
     }
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = cudaMemcpyAsync(c->d_hq, q_host, elems * 2, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_hk, k_host, elems * 2, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c->d_hv, v_host, elems * 2, cudaMemcpyHostToDevice, s);
+    httm_ctx::HostSet& h = c->hs[c->host_calls & 1];
+    ++c->host_calls;
+    // host -> device on the copy stream, once the call that used this set two calls ago has read its inputs.  The
+    // copy does NOT wait for earlier work on `stream`: the host buffers must hold their data when the call is made.
+    cudaError_t e = cudaSuccess;
+    if (h.used) e = cudaStreamWaitEvent(c->s_h2d, h.consumed, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h.q, q_host, elems * 2, cudaMemcpyHostToDevice, c->s_h2d);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h.k, k_host, elems * 2, cudaMemcpyHostToDevice, c->s_h2d);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h.v, v_host, elems * 2, cudaMemcpyHostToDevice, c->s_h2d);
+    if (e == cudaSuccess) e = cudaEventRecord(h.loaded, c->s_h2d);
+    // kernels on the caller's stream, after the inputs have landed and after this set's previous result has left
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, h.loaded, 0);
+    if (e == cudaSuccess && h.used) e = cudaStreamWaitEvent(s, h.returned, 0);
     if ((rc = check_cuda(c, e, "host to device copy"))) return rc;
     const int64_t N = c->n_tokens, H = c->cfg.heads;
-    httm_tensor q{c->d_hq, N * kHeadDim, kHeadDim}, k{c->d_hk, N * kHeadDim, kHeadDim}, v{c->d_hv, N * kHeadDim, kHeadDim};
-    httm_tensor o{c->d_hout, kHeadDim, H * kHeadDim};
+    httm_tensor q{h.q, N * kHeadDim, kHeadDim}, k{h.k, N * kHeadDim, kHeadDim}, v{h.v, N * kHeadDim, kHeadDim};
+    httm_tensor o{h.out, kHeadDim, H * kHeadDim};
     rc = dense ? dense_impl(c, q, k, v, o, s) : global_impl(c, q, k, v, o, s);
     if (rc) return rc;
-    return check_cuda(c, cudaMemcpyAsync(out_host, c->d_hout, elems * 2, cudaMemcpyDeviceToHost, s), "device to host copy");
+    // (the workspace between the kernels is shared by consecutive calls: they run in order on the caller's stream)
+    e = cudaEventRecord(h.computed, s);
+    if (e == cudaSuccess) e = cudaEventRecord(h.consumed, s);
+    // device -> host on the second copy stream; the caller's stream waits for it, so that synchronising `stream`
+    // (or anything enqueued on it later) sees the result
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->s_d2h, h.computed, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, h.out, elems * 2, cudaMemcpyDeviceToHost, c->s_d2h);
+    if (e == cudaSuccess) e = cudaEventRecord(h.returned, c->s_d2h);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, h.returned, 0);
+    h.used = true;
+    return check_cuda(c, e, "device to host copy");
 }
 
 int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out, void* cuda_stream) {
