@@ -73,7 +73,11 @@ enum {
     HTTM_Q_BLOCKS = 3,          /* merging blocks per head                             */
     HTTM_Q_WORKSPACE_BYTES = 4, /* device bytes owned by the context                   */
     HTTM_Q_MAX_BLOCK_TOKENS = 5,
-    HTTM_Q_DEVICE_STATUS = 6    /* syncs the device; 0 or the first device-side error   */
+    HTTM_Q_DEVICE_STATUS = 6,   /* syncs the device; 0 or the first device-side error   */
+    HTTM_Q_MERGED_Q_ROWS = 7,   /* rows per head of HTTM_X_Q_MERGED / HTTM_X_O_MERGED: M_q, or N while query
+                                   outlier filtering is on (the merged length then differs per head)    */
+    HTTM_Q_OUTLIERS = 8         /* syncs the device; query tokens (of the merging blocks, all heads) that the
+                                   last call's filtering took out of their groups                      */
 };
 
 /* httm_export selectors: intermediates of the LAST httm_global_attention call.
@@ -91,7 +95,13 @@ enum {
     HTTM_X_Q_MERGED = 9,   /* [H][M_q][D]                                                */
     HTTM_X_K_MERGED = 10,  /* [H][M_k][D]                                                */
     HTTM_X_V_MERGED = 11,
-    HTTM_X_O_MERGED = 12   /* [H][M_q][D] attention output before unmerge               */
+    HTTM_X_O_MERGED = 12,  /* [H][M_q][D] attention output before unmerge               */
+    /* query outlier filtering (Sec. 3.4); with it on, items 9 and 12 are [H][N][D] and head h's first
+     * HTTM_X_MERGED_Q_HEAD[h] rows are valid */
+    HTTM_X_DEVIATION = 13,     /* [H][N] float: distance of each reordered query token to its group's mean */
+    HTTM_X_THRESHOLD = 14,     /* [1]    float: tau, the (K+1)-th largest deviation (+inf: K = 0)           */
+    HTTM_X_MERGED_Q_HEAD = 15, /* [H]    int32: merged query length of every head                         */
+    HTTM_X_ASSIGN_Q_INITIAL = 16 /* [H][N] int32: the query map before the outliers left (3 holds the map after) */
 };
 
 /* httm_launch_stage selectors.  0-4: the five separate kernels of the path (match and merge read the
@@ -106,7 +116,8 @@ enum {
     HTTM_STAGE_ATTENTION = 3,
     HTTM_STAGE_UNMERGE = 4,
     HTTM_STAGE_MATCH_DIRECT = 5,
-    HTTM_STAGE_MERGE_DIRECT = 6
+    HTTM_STAGE_MERGE_DIRECT = 6,
+    HTTM_STAGE_OUTLIER_FILTER = 7 /* between 5 and 6, only after httm_set_outlier_fraction(> 0): five small kernels */
 };
 
 /*
@@ -136,6 +147,20 @@ int httm_create(const httm_config* cfg, httm_ctx** out);
  */
 int httm_global_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out,
                           void* cuda_stream);
+
+/*
+ * Adaptive outlier filtering for the query tokens (Sec. 3.4, Algorithm 2); off (fraction 0) after httm_create.
+ * With 0 < fraction <= 1 every later httm_global_attention / httm_attention_host call inserts, between match and
+ * merge: the deviation of every query token from the mean of the group it was merged into (0 for a token on its
+ * own), the threshold tau = the (K+1)-th largest deviation over ALL heads with K = floor(fraction * heads * N + 1e-9),
+ * and the map update: tokens with deviation > tau leave their groups and stay unmerged; a group that loses its
+ * destination token continues under its remaining member with the lowest reordered position.  Only queries are
+ * filtered; K and V are untouched.  The merged query length then differs from head to head (HTTM_X_MERGED_Q_HEAD).
+ * The first call with fraction > 0 allocates the extra workspace (device allocation: call it outside timed regions).
+ * Supported for merging blocks of at most 32 tokens and scenes of at most 32767 frames / patch rows / columns.
+ * Errors: INVALID_ARG (fraction outside [0, 1]), UNSUPPORTED, NOMEM, CUDA.
+ */
+int httm_set_outlier_fraction(httm_ctx* ctx, double fraction);
 
 /*
  * Exact multi-head softmax attention over all N tokens (the unmerged baseline the

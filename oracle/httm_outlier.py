@@ -119,14 +119,17 @@ def merge_heads(g: orc.Geometry, assign_q: np.ndarray, qr_bits: np.ndarray):
 
 
 def global_attention_filtered(g: orc.Geometry, ratio_q: float, ratio_kv: float, gamma: float, q, k, v,
-                              attend: bool = True, assign_q_filtered=None) -> FilteredResult:
+                              attend: bool = True, assign_q_filtered=None, assign_q_initial=None,
+                              assign_k=None) -> FilteredResult:
     """Algorithm 1 with the query outlier filtering of Sec. 3.4 / Algorithm 2 (no projections).
     assign_q_filtered: continue from a given filtered map (used when a map under test differs from the
-    oracle's only by tokens whose deviation is within the comparison margin of tau)."""
+    oracle's only by tokens whose deviation is within the comparison margin of tau).
+    assign_q_initial, assign_k: continue from given maps of the matching step (used when a map under test
+    differs from the oracle's only inside the similarity margin)."""
     pi, bs = orc.temporal_reorder(g)
     qr, kr, vr = orc.reorder(g, pi, q), orc.reorder(g, pi, k), orc.reorder(g, pi, v)
-    aq0 = orc.match(g, bs, ratio_q, qr, margins=False)
-    ak = orc.match(g, bs, ratio_kv, kr, margins=False)
+    aq0 = orc.match(g, bs, ratio_q, qr, margins=False) if assign_q_initial is None else np.asarray(assign_q_initial, dtype=np.int64)
+    ak = orc.match(g, bs, ratio_kv, kr, margins=False) if assign_k is None else np.asarray(assign_k, dtype=np.int64)
     eps = deviations(aq0, qr)
     tau = outlier_threshold(eps, gamma)
     outlier = eps > tau

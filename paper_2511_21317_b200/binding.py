@@ -17,11 +17,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhttm.so")
 
 # selectors (mirror include/httm.h)
-Q_TOKENS, Q_MERGED_Q, Q_MERGED_K, Q_BLOCKS, Q_WORKSPACE_BYTES, Q_MAX_BLOCK_TOKENS, Q_DEVICE_STATUS = range(7)
+(Q_TOKENS, Q_MERGED_Q, Q_MERGED_K, Q_BLOCKS, Q_WORKSPACE_BYTES, Q_MAX_BLOCK_TOKENS, Q_DEVICE_STATUS, Q_MERGED_Q_ROWS,
+ Q_OUTLIERS) = range(9)
 (X_PI, X_PI_INV, X_BLOCK_START, X_ASSIGN_Q, X_ASSIGN_K, X_RANK_Q, X_Q_REORDERED, X_K_REORDERED, X_V_REORDERED,
- X_Q_MERGED, X_K_MERGED, X_V_MERGED, X_O_MERGED) = range(13)
-STAGE_REORDER, STAGE_MATCH, STAGE_MERGE, STAGE_ATTENTION, STAGE_UNMERGE, STAGE_MATCH_DIRECT, STAGE_MERGE_DIRECT = range(7)
-STAGE_NAMES = ("reorder", "match", "merge", "attention", "unmerge", "match_direct", "merge_direct")
+ X_Q_MERGED, X_K_MERGED, X_V_MERGED, X_O_MERGED, X_DEVIATION, X_THRESHOLD, X_MERGED_Q_HEAD, X_ASSIGN_Q_INITIAL) = range(17)
+(STAGE_REORDER, STAGE_MATCH, STAGE_MERGE, STAGE_ATTENTION, STAGE_UNMERGE, STAGE_MATCH_DIRECT, STAGE_MERGE_DIRECT,
+ STAGE_OUTLIER_FILTER) = range(8)
+STAGE_NAMES = ("reorder", "match", "merge", "attention", "unmerge", "match_direct", "merge_direct", "outlier_filter")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPORTED", -3: "HTTM_ERR_ALIGNMENT",
@@ -30,7 +32,7 @@ _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPO
 EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
-    "httm_global_attention_static", "httm_selftest_tensor_core",
+    "httm_global_attention_static", "httm_selftest_tensor_core", "httm_set_outlier_fraction",
 )
 
 
@@ -66,6 +68,7 @@ def load_library() -> ctypes.CDLL:
     L.httm_create.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(vp)]
     L.httm_global_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_dense_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
+    L.httm_set_outlier_fraction.argtypes = [vp, ctypes.c_double]
     L.httm_attention_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
     L.httm_launch_stage.argtypes = [vp, ctypes.c_int, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_query.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64)]
@@ -202,6 +205,10 @@ class Httm:
                                                   int(dense), self._stream(stream)))
         return out
 
+    def set_outlier_fraction(self, fraction: float):
+        """Query outlier filtering (Sec. 3.4) for the later calls; 0 switches it off."""
+        self._check(self._lib.httm_set_outlier_fraction(self._h, float(fraction)))
+
     def launch_stage(self, stage: int, q=None, k=None, v=None, out=None, stream=None):
         tq = self._tensor(q, "q") if q is not None else _null_tensor()
         tk = self._tensor(k, "k") if k is not None else _null_tensor()
@@ -220,13 +227,15 @@ class Httm:
     def export(self, what: int, stream=None) -> np.ndarray:
         """Intermediate of the last call as a numpy array (int32 indices or uint16 bf16 bits)."""
         H, N, D = self.cfg.heads, self.n_tokens, self.cfg.head_dim
+        q_rows = self.query(Q_MERGED_Q_ROWS)
         shapes = {
             X_PI: ((N,), np.int32), X_PI_INV: ((N,), np.int32), X_BLOCK_START: ((self.n_blocks + 1,), np.int32),
             X_ASSIGN_Q: ((H, N), np.int32), X_ASSIGN_K: ((H, N), np.int32), X_RANK_Q: ((H, N), np.int32),
             X_Q_REORDERED: ((H, N, D), np.uint16), X_K_REORDERED: ((H, N, D), np.uint16),
-            X_V_REORDERED: ((H, N, D), np.uint16), X_Q_MERGED: ((H, self.m_q, D), np.uint16),
+            X_V_REORDERED: ((H, N, D), np.uint16), X_Q_MERGED: ((H, q_rows, D), np.uint16),
             X_K_MERGED: ((H, self.m_k, D), np.uint16), X_V_MERGED: ((H, self.m_k, D), np.uint16),
-            X_O_MERGED: ((H, self.m_q, D), np.uint16),
+            X_O_MERGED: ((H, q_rows, D), np.uint16), X_DEVIATION: ((H, N), np.float32), X_THRESHOLD: ((1,), np.float32),
+            X_MERGED_Q_HEAD: ((H,), np.int32), X_ASSIGN_Q_INITIAL: ((H, N), np.int32),
         }
         shape, dt = shapes[what]
         arr = np.empty(shape, dtype=dt)

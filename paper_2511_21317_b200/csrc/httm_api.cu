@@ -45,6 +45,15 @@ struct httm_ctx {
     BlockInfo* d_blocks = nullptr;
     __nv_bfloat16 *d_qr = nullptr, *d_kr = nullptr, *d_vr = nullptr;
     __nv_bfloat16 *d_qm = nullptr, *d_km = nullptr, *d_vm = nullptr, *d_om = nullptr;
+    // query outlier filtering (Sec. 3.4): off while fraction == 0; its workspace is allocated when it is first switched on.
+    // The merged query length then differs per head: Q_m and O_m get N rows per head.
+    double outlier_fraction = 0.0;
+    int32_t *d_assign_qf = nullptr, *d_kept_cnt = nullptr, *d_moff_var = nullptr, *d_mq_head = nullptr, *d_tile_prefix = nullptr;
+    int32_t* d_sel = nullptr;   // state of the threshold selection, first word = outlier counter
+    float *d_eps = nullptr, *d_tau = nullptr;
+    __nv_bfloat16 *d_qm_var = nullptr, *d_om_var = nullptr;
+    bool filtering() const { return outlier_fraction > 0.0; }
+    int32_t q_rows() const { return filtering() ? n_tokens : m_q; }   // rows per head of Q_m and O_m
     // staging for the host-buffer entry point (allocated on first use)
     // Two sets of device buffers, two copy streams and events, so that one call's host-to-device copy overlaps the
     // previous call's kernels and device-to-host copy (PCIe is full duplex; the copies are 6x the kernel time).
@@ -83,7 +92,8 @@ struct httm_ctx {
     }
     void release() {
         void* ptrs[] = {d_geom, d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
-                        d_vr, d_qm,     d_km,       d_vm,       d_om,     hs[0].q,  hs[0].k,  hs[0].v, hs[0].out, hs[1].q, hs[1].k, hs[1].v, hs[1].out};
+                        d_vr, d_qm,     d_km,       d_vm,       d_om,     hs[0].q,  hs[0].k,  hs[0].v, hs[0].out, hs[1].q, hs[1].k, hs[1].v, hs[1].out,
+                        d_assign_qf, d_kept_cnt, d_moff_var, d_mq_head, d_tile_prefix, d_sel, d_eps, d_tau, d_qm_var, d_om_var};
         for (void* p : ptrs)
             if (p) cudaFree(p);
         for (HostSet& h : hs)
@@ -222,9 +232,10 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.xr[0] = c->d_qr;
     a.xr[1] = c->d_kr;
     a.xr[2] = c->d_vr;
-    a.assign[0] = c->d_assign_q;
+    a.assign[0] = c->filtering() ? c->d_assign_qf : c->d_assign_q;
     a.assign[1] = c->d_assign_k;
-    a.merged[0] = c->d_qm;
+    a.merged[0] = c->filtering() ? c->d_qm_var : c->d_qm;
+    a.moff_q_var = c->filtering() ? c->d_moff_var : nullptr;
     a.merged[1] = c->d_km;
     a.merged[2] = c->d_vm;
     a.rank_q = c->d_rank_q;
@@ -233,7 +244,7 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.n_tokens = c->n_tokens;
     a.heads = c->cfg.heads;
     a.n_special_total = c->cfg.frames * c->n_special;
-    a.m_q = c->m_q;
+    a.m_q = c->q_rows();
     a.m_k = c->m_k;
     a.status = c->d_status;
     c->launches++;
@@ -242,13 +253,17 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
 
 int stage_attention(httm_ctx* c, cudaStream_t s) {
     AttentionArgs a{};
-    a.q = view(c->d_qm, c->m_q);
+    a.q = view(c->filtering() ? c->d_qm_var : c->d_qm, c->q_rows());
     a.k = view(c->d_km, c->m_k);
     a.v = view(c->d_vm, c->m_k);
-    a.out = c->d_om;
-    a.out_stride_head = (int64_t)c->m_q * kHeadDim;
+    a.out = c->filtering() ? c->d_om_var : c->d_om;
+    a.out_stride_head = (int64_t)c->q_rows() * kHeadDim;
     a.out_stride_token = kHeadDim;
-    a.m_q = c->m_q;
+    a.m_q = c->q_rows();
+    if (c->filtering()) {
+        a.mq_head = c->d_mq_head;
+        a.tile_prefix = c->d_tile_prefix;
+    }
     a.m_k = c->m_k;
     a.heads = c->cfg.heads;
     a.scale_log2 = scale_log2();
@@ -259,7 +274,7 @@ int stage_attention(httm_ctx* c, cudaStream_t s) {
 
 int stage_unmerge(httm_ctx* c, const httm_tensor& out, cudaStream_t s) {
     UnmergeArgs a{};
-    a.o_m = c->d_om;
+    a.o_m = c->filtering() ? c->d_om_var : c->d_om;
     a.rank_q = c->d_rank_q;
     a.pi_inv = c->d_pi_inv;
     a.out = reinterpret_cast<__nv_bfloat16*>(out.ptr);
@@ -267,10 +282,40 @@ int stage_unmerge(httm_ctx* c, const httm_tensor& out, cudaStream_t s) {
     a.out_stride_token = out.stride_token;
     a.n_tokens = c->n_tokens;
     a.heads = c->cfg.heads;
-    a.m_q = c->m_q;
+    a.m_q = c->q_rows();
     a.status = c->d_status;
     c->launches++;
     return check_cuda(c, launch_unmerge(a, s), "unmerge launch");
+}
+
+// Sec. 3.4 / Algorithm 2 between match and merge: deviations, global threshold, map update, per-head offsets
+int stage_outlier(httm_ctx* c, const httm_tensor& q, cudaStream_t s) {
+    OutlierArgs a{};
+    a.geom = c->d_geom;
+    a.blocks = c->d_blocks;
+    a.src_q = view(q);
+    a.layout = source_layout(c);
+    a.assign_q = c->d_assign_q;
+    a.assign_q_out = c->d_assign_qf;
+    a.eps = c->d_eps;
+    a.tau = c->d_tau;
+    a.kept_cnt = c->d_kept_cnt;
+    a.moff_var = c->d_moff_var;
+    a.mq_head = c->d_mq_head;
+    a.tile_prefix = c->d_tile_prefix;
+    a.sel = c->d_sel;
+    a.budget = (int64_t)std::floor(c->outlier_fraction * (double)c->cfg.heads * (double)c->n_tokens + 1e-9);
+    a.n_blocks = c->n_blocks;
+    a.n_tokens = c->n_tokens;
+    a.heads = c->cfg.heads;
+    a.n_special_total = c->cfg.frames * c->n_special;
+    a.status = c->d_status;
+    int rc;
+    if ((rc = check_cuda(c, cudaMemsetAsync(c->d_sel, 0, kSelWords * sizeof(int32_t), s), "selection state reset"))) return rc;
+    if ((rc = check_cuda(c, launch_deviation(a, c->sm_count, s), "deviation launch"))) return rc;
+    if ((rc = check_cuda(c, launch_threshold(a, c->sm_count, s), "threshold launch"))) return rc;
+    c->launches += 5;
+    return check_cuda(c, launch_filter(a, s), "filter launch");
 }
 
 int dense_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out,
@@ -297,6 +342,7 @@ int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const h
     if (direct_mode(c)) {   // four kernels: the temporal reorder is folded into the block loads of match and merge
         const httm_tensor src[3] = {q, k, v};
         if ((rc = stage_match(c, s, src))) return rc;
+        if (c->filtering() && (rc = stage_outlier(c, q, s))) return rc;
         if ((rc = stage_merge(c, s, src))) return rc;
     } else {
         if ((rc = stage_reorder(c, q, k, v, s))) return rc;
@@ -456,6 +502,40 @@ int httm_global_attention(httm_ctx* c, httm_tensor q, httm_tensor k, httm_tensor
     return global_impl(c, q, k, v, out, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (!(fraction >= 0.0 && fraction <= 1.0)) return c->fail(HTTM_ERR_INVALID_ARG, "outlier fraction must lie in [0, 1]");
+    if (fraction == 0.0) {
+        c->outlier_fraction = 0.0;
+        return HTTM_OK;
+    }
+    if (c->max_block > 32) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering supports merging blocks of at most 32 tokens");
+    if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering needs a scene of at most 32767 frames / patch rows / patch columns");
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    if (!c->d_eps) {
+        const size_t H = c->cfg.heads, N = c->n_tokens, B = c->n_blocks;
+        int rc;
+        if ((rc = c->alloc(&c->d_assign_qf, H * N)) || (rc = c->alloc(&c->d_kept_cnt, H * B)) || (rc = c->alloc(&c->d_moff_var, H * B)) ||
+            (rc = c->alloc(&c->d_mq_head, H)) || (rc = c->alloc(&c->d_tile_prefix, H + 1)) || (rc = c->alloc(&c->d_sel, kSelWords)) ||
+            (rc = c->alloc(&c->d_tau, 1)) || (rc = c->alloc(&c->d_qm_var, H * N * kHeadDim)) || (rc = c->alloc(&c->d_om_var, H * N * kHeadDim)) ||
+            (rc = c->alloc(&c->d_eps, H * N)))
+            return rc;
+        // special tokens: never merged (identity map entries, deviation 0), written here once; rows of Q_m past a head's
+        // merged length are read by the last query tile of the head (their results are discarded): give them a value
+        std::vector<int32_t> ident(H * N);
+        for (size_t hd = 0; hd < H; ++hd)
+            for (size_t p = 0; p < N; ++p) ident[hd * N + p] = (int32_t)p;
+        cudaError_t e = cudaMemcpy(c->d_assign_qf, ident.data(), H * N * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemset(c->d_eps, 0, H * N * 4);
+        if (e == cudaSuccess) e = cudaMemset(c->d_qm_var, 0, H * N * kRowBytes);
+        if (e == cudaSuccess) e = cudaMemset(c->d_sel, 0, kSelWords * sizeof(int32_t));
+        if ((rc = check_cuda(c, e, "outlier workspace setup"))) return rc;
+    }
+    c->outlier_fraction = fraction;
+    return HTTM_OK;
+}
+
 int httm_dense_attention(httm_ctx* c, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out, void* cuda_stream) {
     if (!c) return HTTM_ERR_INVALID_ARG;
     int rc = check_io(c, q, k, v, out);
@@ -536,6 +616,10 @@ int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm
         case HTTM_STAGE_UNMERGE:
             if ((rc = check_tensor(c, out, "out"))) return rc;
             return stage_unmerge(c, out, s);
+        case HTTM_STAGE_OUTLIER_FILTER:
+            if (!c->filtering()) return c->fail(HTTM_ERR_INVALID_ARG, "outlier filtering is off: call httm_set_outlier_fraction first");
+            if ((rc = check_tensor(c, q, "q"))) return rc;
+            return stage_outlier(c, q, s);
         case HTTM_STAGE_MATCH_DIRECT:
         case HTTM_STAGE_MERGE_DIRECT: {
             if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "direct stages need a scene of at most 32767 frames / patch rows / patch columns");
@@ -558,6 +642,16 @@ int httm_query(httm_ctx* c, int what, int64_t* value) {
         case HTTM_Q_BLOCKS: *value = c->n_blocks; return HTTM_OK;
         case HTTM_Q_WORKSPACE_BYTES: *value = c->workspace_bytes; return HTTM_OK;
         case HTTM_Q_MAX_BLOCK_TOKENS: *value = c->max_block; return HTTM_OK;
+        case HTTM_Q_MERGED_Q_ROWS: *value = c->q_rows(); return HTTM_OK;
+        case HTTM_Q_OUTLIERS: {
+            *value = 0;
+            if (!c->filtering()) return HTTM_OK;
+            DeviceGuard guard(c->cfg.device);
+            int32_t cnt = 0;
+            int rc = check_cuda(c, cudaMemcpy(&cnt, c->d_sel + kSelOutliers, sizeof cnt, cudaMemcpyDeviceToHost), "read outlier count");
+            *value = cnt;
+            return rc;
+        }
         case HTTM_Q_DEVICE_STATUS: {
             DeviceGuard guard(c->cfg.device);
             int32_t st = 0;
@@ -583,18 +677,23 @@ int httm_export(httm_ctx* c, int what, void* host_dst, size_t bytes, void* cuda_
         case HTTM_X_PI: src = c->pi.data(); need = N * 4; host_src = true; break;
         case HTTM_X_PI_INV: src = c->pi_inv.data(); need = N * 4; host_src = true; break;
         case HTTM_X_BLOCK_START: src = c->blk_start.data(); need = c->blk_start.size() * 4; host_src = true; break;
-        case HTTM_X_ASSIGN_Q: src = c->d_assign_q; need = H * N * 4; break;
+        case HTTM_X_ASSIGN_Q: src = c->filtering() ? c->d_assign_qf : c->d_assign_q; need = H * N * 4; break;
+        case HTTM_X_ASSIGN_Q_INITIAL: src = c->d_assign_q; need = H * N * 4; break;
+        case HTTM_X_DEVIATION: src = c->d_eps; need = H * N * 4; break;
+        case HTTM_X_THRESHOLD: src = c->d_tau; need = 4; break;
+        case HTTM_X_MERGED_Q_HEAD: src = c->d_mq_head; need = H * 4; break;
         case HTTM_X_ASSIGN_K: src = c->d_assign_k; need = H * N * 4; break;
         case HTTM_X_RANK_Q: src = c->d_rank_q; need = H * N * 4; break;
         case HTTM_X_Q_REORDERED: src = c->d_qr; need = H * N * kRowBytes; break;
         case HTTM_X_K_REORDERED: src = c->d_kr; need = H * N * kRowBytes; break;
         case HTTM_X_V_REORDERED: src = c->d_vr; need = H * N * kRowBytes; break;
-        case HTTM_X_Q_MERGED: src = c->d_qm; need = H * (size_t)c->m_q * kRowBytes; break;
+        case HTTM_X_Q_MERGED: src = c->filtering() ? c->d_qm_var : c->d_qm; need = H * (size_t)c->q_rows() * kRowBytes; break;
         case HTTM_X_K_MERGED: src = c->d_km; need = H * (size_t)c->m_k * kRowBytes; break;
         case HTTM_X_V_MERGED: src = c->d_vm; need = H * (size_t)c->m_k * kRowBytes; break;
-        case HTTM_X_O_MERGED: src = c->d_om; need = H * (size_t)c->m_q * kRowBytes; break;
+        case HTTM_X_O_MERGED: src = c->filtering() ? c->d_om_var : c->d_om; need = H * (size_t)c->q_rows() * kRowBytes; break;
         default: return c->fail(HTTM_ERR_INVALID_ARG, "unknown export %d", what);
     }
+    if (!src) return c->fail(HTTM_ERR_INVALID_ARG, "export %d needs outlier filtering switched on", what);
     if (bytes != need) return c->fail(HTTM_ERR_INVALID_ARG, "export %d needs %zu bytes, got %zu", what, need, bytes);
     if (host_src) {
         memcpy(host_dst, src, need);

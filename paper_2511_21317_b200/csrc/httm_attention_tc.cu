@@ -52,6 +52,9 @@ struct TcParams {
     float scale_log2;
     int32_t* status;
     int32_t tiles_per_head, total_tiles, rounds;  // query tiles per head and in all heads; rounds of pair passes
+    const int32_t* mq_head;      // optional: per-head query length (then m_q is the row stride and tile_prefix the tile table)
+    const int32_t* tile_prefix;
+    int32_t heads;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -104,14 +107,39 @@ struct Pass {
     int head, tile;   // tile = index of query tile A inside the head
     bool pair;
 };
+template <bool VAR>   // VAR: the heads differ in query length (tile table in device memory)
 struct PassWalker {
     int r = 0, sub = 0;
     int rounds, total, tiles_per_head;
-    __device__ PassWalker(int rounds_, int total_, int tph) : rounds(rounds_), total(total_), tiles_per_head(tph) {}
+    const int32_t* prefix;   // optional: first tile of every head (heads + 1 entries) when the heads differ in length
+    int heads;
+    __device__ PassWalker(int rounds_, int total_, int tph, const int32_t* prefix_, int heads_)
+        : rounds(rounds_), total(total_), tiles_per_head(tph), prefix(prefix_), heads(heads_) {
+        if (VAR) {
+            total = prefix[heads];
+            rounds = total / (2 * (int)gridDim.x);
+        }
+    }
+    __device__ int head_of(int t) const {
+        if (!VAR) return t / tiles_per_head;
+        int lo = 0, hi = heads - 1;   // largest h with prefix[h] <= t
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (prefix[mid] <= t)
+                lo = mid;
+            else
+                hi = mid - 1;
+        }
+        return lo;
+    }
     __device__ void set(Pass* ps, int t, bool pair) {
-        ps->head = t / tiles_per_head;
-        ps->tile = t - ps->head * tiles_per_head;
+        ps->head = head_of(t);
+        ps->tile = t - (VAR ? prefix[ps->head] : ps->head * tiles_per_head);
         ps->pair = pair;
+    }
+    __device__ bool same_head(int t) const {   // tiles t and t + 1
+        if (!VAR) return t / tiles_per_head == (t + 1) / tiles_per_head;
+        return t + 1 < prefix[head_of(t) + 1];
     }
     __device__ bool next(Pass* ps) {
         const int G = gridDim.x, c = blockIdx.x;
@@ -119,7 +147,7 @@ struct PassWalker {
         const int pair_rounds = rounds + (rem > G ? 1 : 0);   // more than G left: one more (partial) round of pairs
         if (r < pair_rounds) {
             const int t = 2 * (r * G + c);
-            if (t + 1 < total && t / tiles_per_head == (t + 1) / tiles_per_head) {
+            if (t + 1 < total && same_head(t)) {
                 set(ps, t, true);
                 ++r;
                 return true;
@@ -146,6 +174,7 @@ struct PassWalker {
 // once per score tile k with k mod 3 == b (2 n tiles in a pair pass, n in a single pass).
 __device__ __forceinline__ int count_mod3(int n, int r) { return (n - r + 2) / 3; }
 
+template <bool VAR>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const TcParams p) {
@@ -190,7 +219,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
     // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the first 64 columns of its S
-    PassWalker walker(p.rounds, p.total_tiles, p.tiles_per_head);
+    PassWalker<VAR> walker(p.rounds, p.total_tiles, p.tiles_per_head, p.tile_prefix, p.heads);
     Pass ps;
 
     if (warp == 0) {
@@ -368,6 +397,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         bool ok = true;
         for (int pass = 0; ok && walker.next(&ps); ++pass) {
             const int n_score = ps.pair ? 2 * n_tiles : n_tiles;
+            const int mq_rows = VAR ? p.mq_head[ps.head] : p.m_q;   // valid query rows of this head
             // this group's score tiles are k = 2 i + x; in a pair pass they come from key tile i, in a single pass from key tile k
             const int n_own = ps.pair ? n_tiles : (n_tiles - x + 1) / 2;
             {
@@ -460,7 +490,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         tc::tmem_ld32(t_o, o);
                         tc::tmem_ld32(t_o + 32, o + 32);
                         tc::tmem_wait_ld();
-                        if (grow < p.m_q) {
+                        if (grow < mq_rows) {
                             uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)ps.head * p.out_stride_head + (int64_t)grow * p.out_stride_token);
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
@@ -499,7 +529,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             tc::tmem_ld32(t_o + half * 32, oa);
                             tc::tmem_ld32(t_o + kHeadDim + half * 32, ob);   // O_B sits right behind O_A; same TMEM lanes
                             tc::tmem_wait_ld();
-                            if (grow < p.m_q) {
+                            if (grow < mq_rows) {
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
                                     uint32_t w[4];
@@ -531,7 +561,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 }  // namespace
 
 cudaError_t configure_attention() {
-    return cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
 }
 
 // Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
@@ -546,8 +578,12 @@ cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t 
     int ctas = sm_count < 1 ? 1 : sm_count;
     if (ctas > total) ctas = total;
     const int rounds = total / (2 * ctas);
-    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, rounds};
-    attention_tc_kernel<<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
+    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, rounds, a.mq_head, a.tile_prefix, a.heads};
+    if (a.mq_head) {   // the tile table lives in device memory: full grid, CTAs without tiles leave at once
+        attention_tc_kernel<true><<<sm_count < 1 ? 1 : sm_count, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
+        return cudaGetLastError();
+    }
+    attention_tc_kernel<false><<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
 

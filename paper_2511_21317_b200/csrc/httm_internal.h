@@ -75,8 +75,39 @@ struct MergeArgs {
     const int32_t* assign[2];     // A_q, A_k (V uses A_k)
     __nv_bfloat16* merged[3];     // Q_m [H][M_q][64], K_m, V_m [H][M_k][64]
     int32_t* rank_q;              // [H][N] merged row of every reordered token (written for Q)
+    const int32_t* moff_q_var;    // optional [H][blocks]: per-head merged offsets of Q (outlier filtering); then m_q is the row stride of merged[0]
     const BlockInfo* blocks;
     int32_t n_blocks, n_tokens, heads, n_special_total, m_q, m_k;
+    int32_t* status;
+};
+
+// Query outlier filtering (Sec. 3.4): deviations, global threshold, map rewrite, per-head merged offsets.
+// layout of OutlierArgs::sel (int32 words)
+constexpr int kSelOutliers = 0;    // tokens the filter took out of their groups
+constexpr int kSelDone = 1;        // [3] CTAs that have finished level 0, 1, 2
+constexpr int kSelPrefix = 4;      // [2] bits of tau fixed after level 0, 1
+constexpr int kSelRank = 6;        // [2] rank (counted from the largest) still to be skipped inside that prefix
+constexpr int kSelFinished = 8;    // tau is final (budget 0 or everything): the refinement kernels return at once
+constexpr int kSelHist = 16;       // [3][2048] histograms of bits 31-21, 20-10, 9-0
+constexpr int kSelWords = kSelHist + 3 * 2048;
+
+struct OutlierArgs {
+    const BlockGeom* geom;
+    const BlockInfo* blocks;
+    TensorView src_q;             // original Q
+    SourceLayout layout;
+    const int32_t* assign_q;      // [H][N] map of the initial merging
+    int32_t* assign_q_out;        // [H][N] map after the outliers left (special tokens: identity, written once at creation)
+    float* eps;                   // [H][N] deviations (special tokens: 0, written once at creation)
+    float* tau;                   // [1] threshold
+    int32_t* kept_cnt;            // [H][blocks] kept tokens per block after filtering
+    int32_t* moff_var;            // [H][blocks] merged row of each block's first kept token
+    int32_t* mq_head;             // [H] merged query length
+    int32_t* tile_prefix;         // [H + 1] index of each head's first 128-row query tile
+    int32_t* sel;                 // [kSelWords] selection state, zeroed before every call: outlier counter, per-level
+                                  // CTA counters, prefixes, remaining ranks, then the three radix histograms
+    int64_t budget;               // K: number of tokens, over all heads, that may be outliers
+    int32_t n_blocks, n_tokens, heads, n_special_total;
     int32_t* status;
 };
 
@@ -97,6 +128,10 @@ struct AttentionArgs {
     int32_t m_q, m_k, heads;
     float scale_log2;             // log2(e) / sqrt(head_dim)
     int32_t* status;
+    // optional (outlier filtering): per-head query lengths [H] and first-tile indices [H + 1] in device memory;
+    // then m_q is the row stride of q / out and an upper bound of every head's length
+    const int32_t* mq_head;
+    const int32_t* tile_prefix;
 };
 
 // Launchers (each enqueues exactly one kernel on `stream`; returns the CUDA error).
@@ -104,6 +139,9 @@ cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream);
 cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
 cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
 cudaError_t launch_unmerge(const UnmergeArgs& a, cudaStream_t stream);
+cudaError_t launch_deviation(const OutlierArgs& a, int sm_count, cudaStream_t stream);
+cudaError_t launch_threshold(const OutlierArgs& a, int sm_count, cudaStream_t stream);
+cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream);   // map rewrite + per-head offsets (two kernels)
 cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 / TMEM kernel
 cudaError_t configure_attention();
 cudaError_t configure_kernels();   // one-time function attributes (dynamic shared memory sizes)

@@ -604,6 +604,14 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               box_w = DIRECT ? min(a.layout.blk_w, a.layout.grid_w) : 1;
     const int box_rows = box_f * box_h * box_w;
     const int own_t = DIRECT ? lane / (box_h * box_w) : 0, own_y = DIRECT ? (lane / box_w) % box_h : 0, own_x = DIRECT ? lane % box_w : 0;
+    if (DIRECT) {   // stage rows that no block load writes enter the MMAs with weight 0: they must hold finite values
+        for (int q = box_rows * 8 + lane; q < 32 * 8; q += 32) {   // (a load of special tokens may overwrite some of them later)
+            *reinterpret_cast<uint4*>(stage + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(stage + STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+    }
     BoxMap bm;
     bm.clipped = false;
     const int64_t n_tasks = 3ll * a.heads * per_head;
@@ -661,7 +669,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             m.start = bi.start;
             m.n = bi.n;
             m.r = c.t == 0 ? bi.r_q : bi.r_k;
-            m.moff = c.t == 0 ? bi.moff_q : bi.moff_k;
+            m.moff = c.t == 0 ? (a.moff_q_var ? __ldg(a.moff_q_var + (int64_t)c.h * a.n_blocks + c.u) : bi.moff_q) : bi.moff_k;
         }
         return m;
     };
@@ -777,7 +785,8 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 }
                 if (mt == 0 && has_next) target_next = load_target(meta_next);   // behind this task's MMAs
-                const bool w0 = r0 < n_kept && r0 < n - r, w1 = r1 < n_kept && r1 < n - r;   // (a corrupt map cannot overrun)
+                const int cap = t == 0 && a.moff_q_var ? n : n - r;   // (a corrupt map cannot overrun; after outlier filtering more than n - r may be kept)
+                const bool w0 = r0 < n_kept && r0 < cap, w1 = r1 < n_kept && r1 < cap;
                 const float i0 = w0 ? rcnt[r0] : 0.f, i1 = w1 ? rcnt[r1] : 0.f;
 #pragma unroll
                 for (int nt = 0; nt < 8; ++nt) {
@@ -888,6 +897,14 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         own_t[p] = DIRECT ? rho / (box_h * box_w) : 0;
         own_y[p] = DIRECT ? (rho / box_w) % box_h : 0;
         own_x[p] = DIRECT ? rho % box_w : 0;
+    }
+    if (DIRECT) {   // stage rows that no block load writes enter the MMAs with weight 0: they must hold finite values
+        for (int q = box_rows * 8 + lane; q < NMAX * 8; q += 32) {   // (a load of special tokens may overwrite some of them later)
+            *reinterpret_cast<uint4*>(stage + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(stage + STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
     }
     BoxMap bm;
     bm.clipped = false;
@@ -1110,6 +1127,409 @@ cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count,
 }
 
 // ------------------------------------------------------------------------------------
+// Adaptive outlier filtering for the query tokens (Sec. 3.4, Algorithm 2), blocks of at most 32 tokens.
+//   deviation_kernel   eps[h][p] = || q_p - mean of the group p was merged into ||_2 (0 for a group of one)
+//   threshold_kernel   tau = the (K+1)-th largest eps over all heads (K = the global budget): radix select
+//   filter_kernel      outliers (eps > tau) leave their groups; the map is rewritten, the kept tokens of
+//                      every (head, block) are counted
+//   offsets_kernel     per head: merged row of every block's first kept token (prefix sum over the blocks),
+//                      merged length, and the head's first 128-row query tile (for the attention kernel)
+// ------------------------------------------------------------------------------------
+__device__ void finish_level(const OutlierArgs& a, int level, int* hist);   // (threshold selection, below)
+constexpr int kDevWarps = 6;   // 6 x 16.3 KB of shared memory: two CTAs per SM
+constexpr int kCentStride = 65;                                        // floats per centroid row: odd, so that row-wise reads spread over the banks
+constexpr int kDevAux = 32 * kCentStride * 4 + 32 * 4 + 16;           // centroids, reciprocal group sizes, 2 mbarriers
+constexpr int kDevSmem = kDevWarps * (2 * 32 * kRowBytes + kDevAux) + 2048 * 4 /*histogram*/ + 1024 /*alignment slack*/;
+
+__global__ void __launch_bounds__(kDevWarps * 32, 2)
+deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a) {
+    constexpr uint32_t STAGE_BYTES = 32 * kRowBytes;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;   // MMA accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
+    unsigned char* stage = smem + (size_t)warp * 2 * STAGE_BYTES;
+    unsigned char* aux = smem + (size_t)kDevWarps * 2 * STAGE_BYTES + (size_t)warp * kDevAux;
+    float* cent = reinterpret_cast<float*>(aux);                  // [32][65] group means
+    float* rcnt = cent + 32 * kCentStride;                         // [32] 1 / group size
+    int* hist = reinterpret_cast<int*>(smem + (size_t)kDevWarps * (2 * STAGE_BYTES + kDevAux));   // [2048] bits 31-21 of this CTA's deviations
+    for (int i = threadIdx.x; i < 2048; i += kDevWarps * 32) hist[i] = 0;
+    __syncthreads();
+    const uint32_t mbar0 = smem_u32(aux + 32 * kCentStride * 4 + 32 * 4), stage0 = smem_u32(stage);
+    if (lane == 0) {
+        mbar_init(mbar0, 1);
+        mbar_init(mbar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    const SourceLayout& L = a.layout;
+    const int box_f = min(L.blk_frames, L.frames), box_h = min(L.blk_h, L.grid_h), box_w = min(L.blk_w, L.grid_w);
+    const int box_rows = box_f * box_h * box_w;
+    const int own_t = lane / (box_h * box_w), own_y = (lane / box_w) % box_h, own_x = lane % box_w;
+    for (int q = box_rows * 8 + lane; q < 32 * 8; q += 32) {   // rows no load ever writes enter the MMAs with weight 0: keep them finite
+        *reinterpret_cast<uint4*>(stage + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(stage + STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncwarp();
+    BoxMap bm;
+    bm.clipped = false;
+
+    const int64_t n_tasks = (int64_t)a.heads * a.n_blocks;   // (head, block), queries only
+    const int64_t stride = (int64_t)gridDim.x * kDevWarps;
+    const int64_t first = (int64_t)blockIdx.x * kDevWarps + warp;
+    TaskCursor cur, nxt;
+    cur.init(first, stride, a.heads, a.n_blocks);   // one "tensor": t stays 0 while the task index is in range
+    nxt = cur;
+    auto issue = [&](const TaskCursor& c, int buf) {   // lane 0 only
+        const BlockGeom bg = a.geom[c.u];
+        const uint32_t mb = mbar0 + 8 * buf;
+        mbar_expect_tx(mb, (uint32_t)box_rows * kRowBytes);
+        tma_block_load(stage0 + buf * STAGE_BYTES, &map_q, mb, bg.x0, bg.y0, bg.s0, c.h);
+    };
+    if (first < n_tasks && lane == 0) issue(nxt, 0);
+    nxt.advance();
+    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+    nxt.advance();
+
+    int it = 0;
+    bool failed = false;
+    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
+        const int buf = it & 1;
+        const uint32_t parity = (it >> 1) & 1;
+        const bool more = task + 2 * stride < n_tasks;
+        const int h = cur.h;
+        const BlockInfo bi = a.blocks[cur.u];
+        const BlockGeom bg = a.geom[cur.u];
+        bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
+        const int n = bi.n, r = bi.r_q;
+        const int tok = (own_t < bg.frames && own_y < bg.rows && own_x < bg.cols) ? (own_t * bg.rows + own_y) * bg.cols + own_x : -1;
+        float* eps = a.eps + (int64_t)h * a.n_tokens + bi.start;
+        int rep = -1;   // stage ROW of the token this lane's token was merged into
+        if (r > 0 && tok >= 0) {
+            rep = __ldg(a.assign_q + (int64_t)h * a.n_tokens + bi.start + tok) - bi.start;
+            if (rep < 0 || rep >= n) {
+                atomicCAS(a.status, kDevOk, kDevBadIndex);
+                rep = tok;
+            }
+            rep = bm.row_of_token(rep);
+        }
+        if (!mbar_wait_bounded(mbar0 + 8 * buf, parity, a.status, kDevTimeoutMatchLoad)) {
+            failed = true;
+            break;
+        }
+        if (r == 0) {   // nothing merged in this block: every deviation is 0
+            if (tok >= 0) eps[tok] = 0.f;
+        } else {
+            const uint32_t blk = stage0 + buf * STAGE_BYTES;
+            const unsigned kept = __ballot_sync(0xffffffffu, rep == lane);
+            const int n_kept = __popc(kept);
+            const int row_of = rep >= 0 ? __popc(kept & ((1u << rep) - 1u)) : -1;
+            const unsigned group = __match_any_sync(0xffffffffu, row_of);
+            const int group_size = __popc(group);
+            if (rep == lane) rcnt[row_of] = 1.0f / (float)group_size;
+            // group sums = W x on the tensor cores, exactly as in merge_tc_kernel
+            uint32_t bf[2][4][4];
+            const int n_ks = box_rows > 16 ? 2 : 1;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                if (ks < n_ks) {
+                    const int row = 16 * ks + (lane & 7) + ((lane >> 3) & 1) * 8;
+                    const uint32_t rowaddr = blk + row * kRowBytes;
+#pragma unroll
+                    for (int np = 0; np < 4; ++np) ldmatrix_x4_trans(bf[ks][np], rowaddr + (((2 * np + (lane >> 4)) ^ (row & 7)) << 4));
+                }
+            }
+            int rw[2][4];
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                rw[ks][0] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq);
+                rw[ks][1] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 1);
+                rw[ks][2] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 8);
+                rw[ks][3] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 9);
+            }
+            __syncwarp();   // reciprocal group sizes visible
+            const int n_mt = n_kept > 16 ? 2 : 1;
+#pragma unroll 1
+            for (int mt = 0; mt < n_mt; ++mt) {
+                const int r0 = 16 * mt + g, r1 = r0 + 8;
+                float c[8][4];
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < 2; ++ks) {
+                    if (ks < n_ks) {
+                        uint32_t af[4];
+                        af[0] = (rw[ks][0] == r0 ? 0x3f80u : 0u) | (rw[ks][1] == r0 ? 0x3f800000u : 0u);
+                        af[1] = (rw[ks][0] == r1 ? 0x3f80u : 0u) | (rw[ks][1] == r1 ? 0x3f800000u : 0u);
+                        af[2] = (rw[ks][2] == r0 ? 0x3f80u : 0u) | (rw[ks][3] == r0 ? 0x3f800000u : 0u);
+                        af[3] = (rw[ks][2] == r1 ? 0x3f80u : 0u) | (rw[ks][3] == r1 ? 0x3f800000u : 0u);
+#pragma unroll
+                        for (int nt = 0; nt < 8; ++nt) mma_bf16_16816(c[nt], af, bf[ks][nt >> 1][2 * (nt & 1)], bf[ks][nt >> 1][2 * (nt & 1) + 1]);
+                    }
+                }
+                const float i0 = r0 < n_kept ? rcnt[r0] : 0.f, i1 = r1 < n_kept ? rcnt[r1] : 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {   // the means stay in fp32 (no rounding to bf16 before the distance)
+                    if (r0 < n_kept) {
+                        cent[r0 * kCentStride + nt * 8 + 2 * tq] = c[nt][0] * i0;
+                        cent[r0 * kCentStride + nt * 8 + 2 * tq + 1] = c[nt][1] * i0;
+                    }
+                    if (r1 < n_kept) {
+                        cent[r1 * kCentStride + nt * 8 + 2 * tq] = c[nt][2] * i1;
+                        cent[r1 * kCentStride + nt * 8 + 2 * tq + 1] = c[nt][3] * i1;
+                    }
+                }
+            }
+            __syncwarp();   // means visible
+            float dev = 0.f;
+            if (tok >= 0) {
+                float d2 = 0.f;
+                if (group_size >= 2) {   // distance of this lane's token (stage row `lane`) to its group's mean
+                    const unsigned char* row = stage + buf * STAGE_BYTES + lane * kRowBytes;
+                    const float* cr = cent + row_of * kCentStride;
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        float x[8];
+                        unpack8(*reinterpret_cast<const uint4*>(row + ((ch ^ (lane & 7)) << 4)), x);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float d = x[e] - cr[ch * 8 + e];
+                            d2 = fmaf(d, d, d2);
+                        }
+                    }
+                }
+                dev = sqrtf(d2);
+                eps[tok] = dev;
+            }
+            // level 0 of the threshold selection: histogram of the top 11 bits (zeros are not counted), one atomic per distinct bin
+            const int bin = (int)(__float_as_uint(dev) >> 21);
+            const unsigned peers = __match_any_sync(0xffffffffu, bin);
+            if (bin > 0 && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+        }
+        __syncwarp();   // every lane is done with the stage and the tables
+        if (more && lane == 0) issue(nxt, buf);
+    }
+    if (failed) {
+        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2048; i += kDevWarps * 32) {
+        const int c = hist[i];
+        if (c) atomicAdd(a.sel + kSelHist + i, c);
+    }
+    finish_level(a, 0, hist);
+}
+
+// ---- tau = the (K+1)-th largest deviation over all heads (K = the budget): radix select on the bit patterns of the
+// non-negative floats (they order like the values), 11 + 11 + 10 bits.  Level 0's histogram is built by the
+// deviation kernel while it writes the deviations; two refinement kernels rescan them (2 MB, resident in L2) for the
+// elements inside the prefix chosen so far.  In each kernel the CTA that finishes last walks the histogram down from
+// the largest bin until the remaining rank falls inside one, and leaves prefix and rank for the next level.
+// Zeros are never counted at level 0: the walk ends in bin 0 whatever it holds.
+
+// One warp: bin and remaining rank for histogram h[nb] (shared memory), as the sequential walk
+//   above = 0; for (bin = nb - 1; bin > 0 && above + h[bin] <= rank; --bin) above += h[bin];  rank -= above
+__device__ __forceinline__ void select_bin(const int* h, int nb, int rank, int* bin_out, int* rank_out) {
+    const int lane = threadIdx.x & 31, per = nb >> 5, lo = lane * per;
+    int c = 0;
+    for (int i = 0; i < per; ++i) c += h[lo + i];
+    if (lane == 0) c -= h[0];   // bin 0 ends the walk: it is never added
+    int incl = c;               // this lane's bins and all higher ones
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += o;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, incl > rank);
+    if (hit == 0) {             // fewer than rank + 1 elements above bin 0
+        if (lane == 0) {
+            *bin_out = 0;
+            *rank_out = rank - incl;
+        }
+        return;
+    }
+    if (lane == 31 - __clz(hit)) {   // the walk stops inside this lane's bins
+        int above = incl - c, b = lo + per - 1;
+        for (; b > lo; --b) {
+            if (above + h[b] > rank) break;
+            above += h[b];
+        }
+        *bin_out = b;
+        *rank_out = rank - above;
+    }
+}
+
+// End of a level, called by every thread of every CTA after the CTA's histogram has been added to the global one:
+// the CTA that arrives last selects the bin.  hist: 2048 ints of shared memory.
+__device__ void finish_level(const OutlierArgs& a, int level, int* hist) {
+    __shared__ int s_last, s_bin, s_rank;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(a.sel + kSelDone + level, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const int64_t count = (int64_t)a.heads * a.n_tokens;
+    if (level == 0 && (a.budget <= 0 || a.budget >= count)) {   // nothing is an outlier (tau = +inf) / everything is (tau = -1)
+        if (threadIdx.x == 0) {
+            *a.tau = a.budget <= 0 ? INFINITY : -1.0f;
+            a.sel[kSelFinished] = 1;
+        }
+        return;
+    }
+    const int nb = level == 2 ? 1024 : 2048, shift = level == 0 ? 21 : (level == 1 ? 10 : 0);
+    for (int i = threadIdx.x; i < nb; i += blockDim.x) hist[i] = __ldcg(a.sel + kSelHist + level * 2048 + i);
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int rank = level == 0 ? (int)a.budget : __ldcg(a.sel + kSelRank + level - 1);
+        select_bin(hist, nb, rank, &s_bin, &s_rank);
+        __syncwarp();
+        if (threadIdx.x == 0) {
+            const uint32_t prefix = (level == 0 ? 0u : (uint32_t)__ldcg(a.sel + kSelPrefix + level - 1)) | ((uint32_t)s_bin << shift);
+            if (level < 2) {
+                a.sel[kSelPrefix + level] = (int)prefix;
+                a.sel[kSelRank + level] = s_rank;
+            } else {
+                *a.tau = __uint_as_float(prefix);
+            }
+        }
+    }
+}
+
+constexpr int kRefineThreads = 256;
+// LEVEL 1: histogram of bits 20-10 of the deviations whose bits 31-21 equal the level-0 choice; LEVEL 2: of bits 9-0
+// of those whose bits 31-10 equal the choice so far.
+template <int LEVEL>
+__global__ void __launch_bounds__(kRefineThreads) refine_kernel(const OutlierArgs a) {
+    __shared__ int hist[2048];
+    if (__ldcg(a.sel + kSelFinished)) return;   // (same answer in every thread of every CTA)
+    constexpr int NB = LEVEL == 1 ? 2048 : 1024, SHIFT = LEVEL == 1 ? 10 : 0;
+    constexpr uint32_t MASK = LEVEL == 1 ? 0xffe00000u : 0xfffffc00u;
+    for (int i = threadIdx.x; i < NB; i += kRefineThreads) hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = (uint32_t)__ldcg(a.sel + kSelPrefix + LEVEL - 1);
+    const int64_t count = (int64_t)a.heads * a.n_tokens, quads = count >> 2;
+    const uint4* bits4 = reinterpret_cast<const uint4*>(a.eps);   // (the array comes from cudaMalloc: 16-byte aligned)
+    auto tally = [&](uint32_t b) {
+        if ((b & MASK) == prefix) atomicAdd(&hist[(b >> SHIFT) & (NB - 1)], 1);
+    };
+    for (int64_t i = (int64_t)blockIdx.x * kRefineThreads + threadIdx.x; i < quads; i += (int64_t)gridDim.x * kRefineThreads) {
+        const uint4 b = __ldg(bits4 + i);
+        tally(b.x);
+        tally(b.y);
+        tally(b.z);
+        tally(b.w);
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (int)(count & 3)) tally(__float_as_uint(a.eps[(quads << 2) + threadIdx.x]));
+    __syncthreads();
+    for (int i = threadIdx.x; i < NB; i += kRefineThreads) {
+        const int c = hist[i];
+        if (c) atomicAdd(a.sel + kSelHist + LEVEL * 2048 + i, c);
+    }
+    finish_level(a, LEVEL, hist);
+}
+
+// Outliers leave their groups (Sec. 3.4 item 4): one warp per (head, block), lane = token of the block.
+// An outlier maps to itself; the other tokens of a group stay together, under their old representative if
+// that is not an outlier, else under the remaining member with the lowest position.
+__global__ void __launch_bounds__(256) filter_kernel(const OutlierArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t task = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (task >= (int64_t)a.heads * a.n_blocks) return;
+    const int h = (int)(task / a.n_blocks), b = (int)(task - (int64_t)h * a.n_blocks);
+    const BlockInfo bi = a.blocks[b];
+    const int n = bi.n;
+    const float tau = *a.tau;
+    const int32_t* A = a.assign_q + (int64_t)h * a.n_tokens + bi.start;
+    int32_t* A_out = a.assign_q_out + (int64_t)h * a.n_tokens + bi.start;
+    int rep = -1 - lane;   // lanes without a token match nobody
+    bool outl = false;
+    if (lane < n) {
+        rep = A[lane] - bi.start;
+        if (rep < 0 || rep >= n) {
+            atomicCAS(a.status, kDevOk, kDevBadIndex);
+            rep = lane;
+        }
+        outl = a.eps[(int64_t)h * a.n_tokens + bi.start + lane] > tau;
+    }
+    const unsigned out_mask = __ballot_sync(0xffffffffu, outl);
+    const unsigned group = __match_any_sync(0xffffffffu, rep);
+    int now = lane;
+    if (lane < n && !outl) now = ((out_mask >> rep) & 1u) ? __ffs(group & ~out_mask) - 1 : rep;
+    const unsigned kept = __ballot_sync(0xffffffffu, lane < n && now == lane);
+    if (lane < n) A_out[lane] = bi.start + now;
+    if (lane == 0) {
+        a.kept_cnt[(int64_t)h * a.n_blocks + b] = __popc(kept);
+        if (out_mask) atomicAdd(a.sel + kSelOutliers, __popc(out_mask));
+    }
+}
+
+// Per head: merged row of every block's first kept token = specials + exclusive prefix sum of the kept counts;
+// merged length; then, over the heads, the index of each head's first 128-row query tile.  One CTA, a warp per head.
+__global__ void __launch_bounds__(1024, 1) offsets_kernel(const OutlierArgs a) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    for (int h = warp; h < a.heads; h += n_warps) {
+        int running = a.n_special_total;
+        for (int b0 = 0; b0 < a.n_blocks; b0 += 32) {
+            const int b = b0 + lane;
+            const int c = b < a.n_blocks ? a.kept_cnt[(int64_t)h * a.n_blocks + b] : 0;
+            int incl = c;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            if (b < a.n_blocks) a.moff_var[(int64_t)h * a.n_blocks + b] = running + incl - c;
+            running += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) a.mq_head[h] = running;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int h = 0; h < a.heads; ++h) {
+            a.tile_prefix[h] = t;
+            t += (a.mq_head[h] + 127) / 128;
+        }
+        a.tile_prefix[a.heads] = t;
+    }
+}
+
+cudaError_t launch_deviation(const OutlierArgs& a, int sm_count, cudaStream_t stream) {
+    CUtensorMap mq;
+    if (!encode_block_map(&mq, a.src_q, a.layout, a.heads)) return cudaErrorInvalidValue;
+    const int64_t n_tasks = (int64_t)a.heads * a.n_blocks;
+    int64_t grid = (n_tasks + kDevWarps - 1) / kDevWarps;
+    if (grid > 2ll * sm_count) grid = 2ll * sm_count;
+    if (grid < 1) grid = 1;
+    deviation_kernel<<<(unsigned)grid, kDevWarps * 32, kDevSmem, stream>>>(mq, a);
+    return cudaGetLastError();
+}
+cudaError_t launch_threshold(const OutlierArgs& a, int sm_count, cudaStream_t stream) {
+    const int64_t quads = ((int64_t)a.heads * a.n_tokens) >> 2;
+    int64_t grid = (quads + kRefineThreads * 4 - 1) / (kRefineThreads * 4);   // about four 16-byte loads per thread
+    if (grid > 2ll * sm_count) grid = 2ll * sm_count;
+    if (grid < 1) grid = 1;
+    refine_kernel<1><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    refine_kernel<2><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream) {
+    const int64_t threads = (int64_t)a.heads * a.n_blocks * 32;
+    filter_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    offsets_kernel<<<1, 1024, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------
 // a5. Head-wise unmerge + inverse reorder + head concat (Eq. 5-7): every original token
 //     copies the attention output of the merged query token it went into.
 //     8 threads move one 128-byte (token, head) row.  A CTA works on one head and 128
@@ -1171,6 +1591,7 @@ cudaError_t configure_kernels() {
     HTTM_SET_SMEM((match_kernel<8, true>), match_smem_bytes(256));
     HTTM_SET_SMEM((match_kernel<4, false>), match_smem_bytes(128));
     HTTM_SET_SMEM((match_kernel<8, false>), match_smem_bytes(256));
+    HTTM_SET_SMEM(deviation_kernel, kDevSmem);
     HTTM_SET_SMEM(merge_tc_kernel<false>, kMergeTcSmem);
     HTTM_SET_SMEM(merge_tc_kernel<true>, kMergeTcSmem);
     HTTM_SET_SMEM((merge_multi_kernel<2, false>), merge_multi_smem(64));

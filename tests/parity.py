@@ -72,6 +72,7 @@ def check_merged(gpu_bits: np.ndarray, exact: np.ndarray, what=""):
     error of the kernel: |err| <= half a bf16 step (2^-8 |exact|) + 4e-6 x the largest magnitude."""
     got = bits_to_f64(gpu_bits)
     assert got.shape == exact.shape, f"{what}: shape {got.shape} != {exact.shape}"
+    assert np.isfinite(got).all(), f"{what}: non-finite merged value"
     err = np.abs(got - exact)
     bound = np.abs(exact) * 2.0 ** -8 + 4e-6 * max(float(np.abs(exact).max()), 1e-30)
     bad = err > bound
@@ -131,5 +132,79 @@ def full_check(g, rho_q, rho_kv, q, k, v, ex, out_bits, sample_tokens=None, what
         for hd in range(g.heads):
             assert np.array_equal(out_bits[:, hd * D:(hd + 1) * D], ex["o_m"][hd][res.rank_q[hd][inv]]), \
                 f"{what}: unmerge of head {hd} is not a pure copy"
+    stats["rms"] = rms
+    return stats
+
+
+DEV_TOL = 1e-5   # deviations: |gpu - oracle| <= DEV_TOL x (largest |q| + the deviation): fp32 means, differences and sums of 64 squares
+
+
+def filtered_check(g, rho_q, rho_kv, gamma, q, k, v, ex, out_bits, n_outliers, sample_tokens=None, what="", peaky=False):
+    """Query outlier filtering (Sec. 3.4, Algorithm 2) against its oracle.
+    ex: exports pi, blk_start, assign_q0 (map of the initial merging), assign_q (after the outliers left), assign_k,
+    eps, tau, mq_head, rank_q, q_m, k_m, v_m, o_m (q_m, o_m with N rows per head, head h's first mq_head[h] valid).
+    Rules: the matching maps as in check_maps; deviations within DEV_TOL; the threshold is the (K+1)-th largest of
+    the deviations under test, within DEV_TOL of the oracle's; the outlier decision agrees with the oracle's for
+    every token whose deviation is further than 2 x DEV_TOL from the oracle's threshold; the filtered map is exactly
+    what the oracle's rule makes of the decisions under test; everything downstream continues from that map."""
+    from oracle import httm_outlier as flt
+    res0 = orc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
+    assert np.array_equal(ex["pi"].astype(np.int64), res0.pi), f"{what}: reorder permutation differs"
+    qr, kr = orc.reorder(g, res0.pi, q), orc.reorder(g, res0.pi, k)
+    nq = check_maps(g, rho_q, res0.blk_start, qr, res0.assign_q, res0.margin_best_q, res0.margin_sel_q, ex["assign_q0"], what + " A_q (initial)")
+    nk = check_maps(g, rho_kv, res0.blk_start, kr, res0.assign_k, res0.margin_best_k, res0.margin_sel_k, ex["assign_k"], what + " A_k")
+    aq0 = ex["assign_q0"].astype(np.int64)
+    eps = flt.deviations(aq0, qr)
+    eps_gpu = ex["eps"].astype(np.float64)
+    tol = DEV_TOL * (float(np.abs(bits_to_f64(qr)).max()) + eps)
+    err = np.abs(eps_gpu - eps)
+    assert (err <= tol).all(), f"{what}: deviation off by {err.max():.3e} (tolerance {tol.flat[err.argmax()]:.3e})"
+    alone = np.stack([np.bincount(aq0[hd], minlength=aq0.shape[1])[aq0[hd]] == 1 for hd in range(aq0.shape[0])])
+    assert (eps_gpu[alone] == 0).all(), f"{what}: tokens on their own must have deviation exactly 0"
+    K = flt.outlier_budget(eps.size, gamma)
+    tau, tau_gpu = flt.outlier_threshold(eps, gamma), float(ex["tau"][0])
+    outl_gpu = eps_gpu > tau_gpu
+    if K <= 0:
+        assert tau_gpu == float("inf") and not outl_gpu.any()
+    elif K >= eps.size:
+        assert outl_gpu.all()
+    else:
+        assert outl_gpu.sum() <= K < (eps_gpu >= tau_gpu).sum(), f"{what}: tau is not the (K+1)-th largest deviation"
+        assert abs(tau_gpu - tau) <= DEV_TOL * (float(np.abs(bits_to_f64(qr)).max()) + tau), f"{what}: tau {tau_gpu} vs {tau}"
+        clear = np.abs(eps - tau) > 2 * tol
+        assert np.array_equal(outl_gpu[clear], (eps > tau)[clear]), f"{what}: outlier decisions differ outside the margin"
+    in_blocks = int(outl_gpu[:, int(ex["blk_start"][0]):].sum())   # (special tokens are in no block and never merged)
+    assert n_outliers == in_blocks, f"{what}: outlier counter {n_outliers} != {in_blocks}"
+    aq = flt.filter_map(aq0, outl_gpu)
+    assert np.array_equal(ex["assign_q"].astype(np.int64), aq), f"{what}: filtered map differs from the rule applied to the decisions"
+    res = flt.global_attention_filtered(g, rho_q, rho_kv, gamma, q, k, v, attend=False, assign_q_filtered=aq,
+                                        assign_q_initial=aq0, assign_k=ex["assign_k"].astype(np.int64))
+    assert ex["mq_head"].tolist() == res.M_q, f"{what}: merged query lengths {ex['mq_head'].tolist()} != {res.M_q}"
+    stats = {"ambiguous_blocks_q": nq, "ambiguous_blocks_k": nk, "outliers": int(outl_gpu.sum()), "tau": tau_gpu,
+             "undecided": int((~(np.abs(eps - tau) > 2 * tol)).sum()) if 0 < K < eps.size else 0, "M_q": res.M_q}
+    fr = [check_merged(ex[n], ref, f"{what} {n}") for n, ref in (("k_m", res.k_m), ("v_m", res.v_m))]
+    for hd in range(g.heads):
+        assert np.array_equal(ex["rank_q"][hd].astype(np.int64), res.rank_q[hd]), f"{what}: rank_q of head {hd} differs"
+        fr.append(check_merged(ex["q_m"][hd][:res.M_q[hd]], res.q_m[hd], f"{what} q_m head {hd}"))
+    stats["merged_exactly_rounded"] = min(fr)
+    D = g.head_dim
+    inv = np.empty_like(res.pi)
+    inv[res.pi] = np.arange(len(res.pi))
+    if sample_tokens is None:
+        o_m = [orc.attention(res.q_m[hd][None], res.k_m[hd:hd + 1], res.v_m[hd:hd + 1])[0] for hd in range(g.heads)]
+        out = np.concatenate([o_m[hd][res.rank_q[hd][inv]] for hd in range(g.heads)], axis=1)
+        rms = float(np.sqrt(np.mean(out ** 2)))
+        for hd in range(g.heads):
+            check_output(ex["o_m"][hd][:res.M_q[hd]], o_m[hd], rms, f"{what} O_m head {hd}", peaky)
+        stats["out_err"] = check_output(out_bits, out, rms, what + " out", peaky)
+    else:
+        pos = inv[np.asarray(sample_tokens)]
+        rows = np.concatenate([orc.attention(res.q_m[hd][res.rank_q[hd][pos]][None], res.k_m[hd:hd + 1], res.v_m[hd:hd + 1])[0]
+                               for hd in range(g.heads)], axis=1)
+        rms = float(np.sqrt(np.mean(rows ** 2)))
+        stats["out_err"] = check_output(out_bits[sample_tokens], rows, rms, what + " out (sampled)", peaky)
+    for hd in range(g.heads):   # unmerge is a pure copy of O_m rows: on ALL tokens, bit-exactly
+        assert np.array_equal(out_bits[:, hd * D:(hd + 1) * D], ex["o_m"][hd][res.rank_q[hd][inv]]), \
+            f"{what}: unmerge of head {hd} is not a pure copy"
     stats["rms"] = rms
     return stats

@@ -1,0 +1,141 @@
+"""Parity of the CUDA path with query outlier filtering switched on (Sec. 3.4, Algorithm 2) against its CPU oracle.
+All tests here need a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import httm_oracle as orc
+from paper_2511_21317_b200 import binding as hb
+from paper_2511_21317_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+NAMES = {"pi": hb.X_PI, "blk_start": hb.X_BLOCK_START, "assign_q0": hb.X_ASSIGN_Q_INITIAL, "assign_q": hb.X_ASSIGN_Q,
+         "assign_k": hb.X_ASSIGN_K, "eps": hb.X_DEVIATION, "tau": hb.X_THRESHOLD, "mq_head": hb.X_MERGED_Q_HEAD,
+         "rank_q": hb.X_RANK_Q, "q_m": hb.X_Q_MERGED, "k_m": hb.X_K_MERGED, "v_m": hb.X_V_MERGED, "o_m": hb.X_O_MERGED}
+
+
+def run_filtered(wl, gamma, q=None, k=None, v=None, sample=None, peaky=False):
+    if q is None:
+        q, k, v = synth.make_qkv(wl)
+    g = orc.Geometry.of(wl)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        ctx.set_outlier_fraction(gamma)
+        assert ctx.query(hb.Q_MERGED_Q_ROWS) == wl.n_tokens
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        before = ctx.launch_count()
+        out = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert ctx.launch_count() - before == 9
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        ex = {name: ctx.export(what) for name, what in NAMES.items()}
+        stats = parity.filtered_check(g, wl.ratio_q, wl.ratio_kv, gamma, q, k, v, ex, hb.bits_from_bf16(out),
+                                      ctx.query(hb.Q_OUTLIERS), sample, wl.name, peaky)
+        # determinism: a second call gives bit-identical results
+        out2 = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert torch.equal(out, out2)
+        for name, what in NAMES.items():
+            if name not in ("q_m", "o_m"):   # (rows past a head's merged length are not defined)
+                assert np.array_equal(ex[name], ctx.export(what)), f"{name} differs between two identical calls"
+    return stats
+
+
+@pytest.mark.parametrize("gamma", [0.002, 0.05, 0.3])
+def test_tiny_config_filtered(gamma):
+    wl = synth.WORKLOADS["tiny"]
+    stats = run_filtered(wl, gamma)
+    assert stats["outliers"] > 0 and stats["out_err"] <= parity.OUT_TOL
+    assert len(set(stats["M_q"])) > 1          # one global budget: the heads keep different numbers of query tokens
+
+
+GEOMS = [
+    # name, frames, grid_h, grid_w, blk, ratio_q, ratio_kv, n_camera, n_register, heads, gamma
+    ("clipped_all_dims", 3, 5, 6, (2, 2, 4), 0.5, 0.7, 1, 1, 2, 0.1),
+    ("window_1x1", 3, 3, 3, (2, 1, 1), 0.5, 0.5, 1, 4, 2, 0.1),
+    ("single_token_blocks", 2, 2, 2, (1, 1, 1), 0.9, 0.9, 1, 0, 1, 0.5),
+    ("no_specials", 4, 8, 8, (2, 4, 4), 0.5, 0.75, 0, 0, 3, 0.02),
+    ("frames_not_divisible", 5, 9, 9, (2, 4, 4), 0.7, 0.8, 1, 4, 2, 0.07),
+    ("ratio_zero_q", 4, 8, 8, (2, 4, 4), 0.0, 0.6, 1, 4, 2, 0.1),
+    ("ratio_099", 4, 9, 9, (2, 4, 4), 0.99, 0.99, 1, 4, 2, 0.2),
+    ("one_frame", 1, 12, 12, (2, 4, 4), 0.5, 0.5, 1, 4, 2, 0.05),
+    ("many_heads", 2, 8, 8, (2, 4, 4), 0.7, 0.7, 1, 4, 37, 0.05),
+    ("tile_boundaries", 4, 16, 16, (2, 4, 4), 0.75, 0.7, 1, 4, 5, 0.04),
+]
+
+
+@pytest.mark.parametrize("case", GEOMS, ids=[c[0] for c in GEOMS])
+def test_adversarial_geometries_filtered(case):
+    name, S, h, w, blk, rq, rkv, ncam, nreg, H, gamma = case
+    wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, n_camera=ncam, n_register=nreg, heads=H, seed=3)
+    run_filtered(wl, gamma, peaky=True)
+
+
+def test_everything_an_outlier_equals_unmerged_queries():
+    wl = synth.Workload("all_out", 3, 7, 9, 2, 4, 4, 0.7, 0.5, heads=3)
+    stats = run_filtered(wl, 1.0)
+    assert stats["M_q"] == [wl.n_tokens] * wl.heads
+
+
+def test_ties_and_zero_vectors_filtered():
+    wl = synth.Workload("ties", 2, 8, 8, 2, 4, 4, 0.5, 0.5, heads=2, n_camera=1, n_register=1)
+    x = synth.make_identical_block_tokens(wl, seed=4)       # identical tokens in a block: every deviation is 0
+    q, k, v = synth.make_qkv(wl)
+    z = q.copy()
+    z[:, 10:40, :] = 0
+    run_filtered(wl, 0.1, x, k, v, peaky=True)
+    run_filtered(wl, 0.1, z, z, v, peaky=True)
+
+
+def test_switching_the_filter_off_restores_the_plain_path():
+    wl = synth.Workload("toggle", 4, 9, 9, 2, 4, 4, 0.7, 0.7, heads=4)
+    q, k, v = synth.make_qkv(wl)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        plain = ctx.global_attention(dq, dk, dv).clone()
+        with pytest.raises(hb.HttmError):
+            ctx.export(hb.X_DEVIATION)
+        ctx.set_outlier_fraction(0.1)
+        filtered = ctx.global_attention(dq, dk, dv).clone()
+        torch.cuda.synchronize()
+        assert not torch.equal(plain, filtered)
+        assert ctx.query(hb.Q_OUTLIERS) > 0
+        ctx.set_outlier_fraction(0.0)
+        assert ctx.query(hb.Q_MERGED_Q_ROWS) == ctx.m_q and ctx.query(hb.Q_OUTLIERS) == 0
+        before = ctx.launch_count()
+        again = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert ctx.launch_count() - before == 4
+        assert torch.equal(plain, again)
+        assert ctx.export(hb.X_Q_MERGED).shape == (wl.heads, ctx.m_q, 64)
+
+
+def test_filter_argument_errors():
+    wl = synth.Workload("big_blocks", 4, 8, 8, 4, 4, 4, 0.5, 0.5, heads=2)          # 64-token blocks
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        with pytest.raises(hb.HttmError) as e:
+            ctx.set_outlier_fraction(0.1)
+        assert e.value.code == hb.ERR_UNSUPPORTED
+        ctx.set_outlier_fraction(0.0)
+    wl = synth.Workload("ok", 2, 8, 8, 2, 4, 4, 0.5, 0.5, heads=2)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        for bad in (-0.1, 1.5, float("nan")):
+            with pytest.raises(hb.HttmError) as e:
+                ctx.set_outlier_fraction(bad)
+            assert e.value.code == hb.ERR_INVALID_ARG
+        with pytest.raises(hb.HttmError):
+            ctx.launch_stage(hb.STAGE_OUTLIER_FILTER, *(hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(wl)))
+
+
+def test_medium_config_filtered_full_size_sampled():
+    """The benchmark's workload with the filter on: maps, deviations, threshold, merged tensors on all tokens,
+    attention output on sampled tokens."""
+    wl = synth.WORKLOADS["medium"]
+    rng = np.random.default_rng(1)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 48), [0, 4, 5, wl.n_tokens - 1]]))
+    stats = run_filtered(wl, 0.01, sample=toks)
+    K = int(np.floor(0.01 * wl.heads * wl.n_tokens + 1e-9))
+    assert K - 4 <= stats["outliers"] <= K          # (K unless fp32 deviations tie at the threshold)
+    assert stats["out_err"] <= parity.OUT_TOL
