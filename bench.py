@@ -346,10 +346,53 @@ def run_ours(args, wl):
             line["cpu_baseline"] = {"value": N / sec, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
                                     "sample": info["sample"], "seconds": info["seconds"], "ms_per_layer_extrapolated": sec * 1e3}
             line["parity_sample"] = parity_sample(ctx, hb, wl, kept, out)
+        if world == 1 and args.outlier_fraction > 0:
+            line["outlier_filter"] = filtered_variant(args, wl, hb, dq, dk, dv, local)
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def filtered_variant(args, wl, hb, dq, dk, dv, device_index):
+    """The same step with query outlier filtering on (Sec. 3.4): public call and per-stage times, in a context of its own."""
+    import torch
+    ctx = hb.Httm(hb.HttmConfig.of(wl, device=device_index))
+    try:
+        if ctx.query(hb.Q_MAX_BLOCK_TOKENS) > 32:
+            return {"skipped": "outlier filtering supports merging blocks of at most 32 tokens"}
+        ctx.set_outlier_fraction(args.outlier_fraction)
+        out = ctx.new_output()
+        stream = torch.cuda.current_stream()
+        steps = max(3, min(args.steps, 100))
+        for _ in range(3):
+            ctx.global_attention(dq, dk, dv, out)
+        torch.cuda.synchronize()
+        l0 = ctx.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            ctx.global_attention(dq, dk, dv, out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        launches = (ctx.launch_count() - l0) // steps
+        order = [hb.STAGE_MATCH_DIRECT, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE_DIRECT, hb.STAGE_ATTENTION, hb.STAGE_UNMERGE]
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(order) + 1)] for _ in range(steps)]
+        for s_ in range(steps):
+            evs[s_][0].record(stream)
+            for i, st in enumerate(order):
+                ctx.launch_stage(st, dq, dk, dv, out)
+                evs[s_][i + 1].record(stream)
+        torch.cuda.synchronize()
+        stage_ms = {hb.STAGE_NAMES[st]: sum(evs[s_][i].elapsed_time(evs[s_][i + 1]) for s_ in range(steps)) / steps
+                    for i, st in enumerate(order)}
+        mq = ctx.export(hb.X_MERGED_Q_HEAD)
+        return {"fraction": args.outlier_fraction, "ms_per_step": e0.elapsed_time(e1) / steps, "steps": steps,
+                "gpu_launches_per_step": int(launches), "stages_ms": stage_ms, "outliers": ctx.query(hb.Q_OUTLIERS),
+                "merged_query_length_per_head": {"min": int(mq.min()), "max": int(mq.max()), "unfiltered": ctx.m_q},
+                "device_status": ctx.query(hb.Q_DEVICE_STATUS)}
+    finally:
+        ctx.close()
 
 
 def parity_sample(ctx, hb, wl, kept, out):
@@ -386,6 +429,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-rows", type=int, default=4096, help="merged query rows per head the CPU oracle attends (sample)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--outlier-fraction", type=float, default=0.01,
+                    help="also time the step with query outlier filtering at this fraction (extra block of the line; 0: skip)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
     if args.ratio is not None:

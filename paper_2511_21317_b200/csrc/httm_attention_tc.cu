@@ -30,7 +30,9 @@ constexpr int KV_STAGES = 3;
 constexpr int TILE_BYTES = BM * kRowBytes;   // 16 KB
 constexpr int NTHREADS = 320;   // producer warp, MMA warp, 2 x 4 softmax warps: registers are granted per four warps, so 168 per thread as with twelve
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row exchange*/;
+constexpr int kTableHeads = 256;   // head tables (per-head query lengths) of up to this many heads are kept in shared memory
+constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row exchange*/ +
+                           (2 * kTableHeads + 4) * 4 /*head tables*/;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
 struct Barriers {
@@ -213,13 +215,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc::prefetch_tensormap(&map_k);
         tc::prefetch_tensormap(&map_v);
     }
+    // per-head query lengths: every pass looks its head up (binary search over the tile table): keep the tables on chip
+    int32_t* s_prefix = reinterpret_cast<int32_t*>(smem + (2 + 2 * KV_STAGES) * TILE_BYTES + 256 + 1024);   // [heads + 1]
+    int32_t* s_mq = s_prefix + kTableHeads + 4;                                                               // [heads]
+    const bool tables_on_chip = VAR && p.heads <= kTableHeads;
+    if (tables_on_chip) {
+        for (int i = tid; i <= p.heads; i += NTHREADS) {
+            s_prefix[i] = p.tile_prefix[i];
+            if (i < p.heads) s_mq[i] = p.mq_head[i];
+        }
+    }
     if (warp == 1) tc::tmem_alloc(tc::smem_addr(&bars->tmem_base), TMEM_COLS);
     tc::fence_before_sync();
     __syncthreads();
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
     // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the first 64 columns of its S
-    PassWalker<VAR> walker(p.rounds, p.total_tiles, p.tiles_per_head, p.tile_prefix, p.heads);
+    const int32_t* mq_table = tables_on_chip ? s_mq : p.mq_head;
+    PassWalker<VAR> walker(p.rounds, p.total_tiles, p.tiles_per_head, tables_on_chip ? s_prefix : p.tile_prefix, p.heads);
     Pass ps;
 
     if (warp == 0) {
@@ -397,7 +410,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         bool ok = true;
         for (int pass = 0; ok && walker.next(&ps); ++pass) {
             const int n_score = ps.pair ? 2 * n_tiles : n_tiles;
-            const int mq_rows = VAR ? p.mq_head[ps.head] : p.m_q;   // valid query rows of this head
+            const int mq_rows = VAR ? mq_table[ps.head] : p.m_q;   // valid query rows of this head
             // this group's score tiles are k = 2 i + x; in a pair pass they come from key tile i, in a single pass from key tile k
             const int n_own = ps.pair ? n_tiles : (n_tiles - x + 1) / 2;
             {

@@ -87,6 +87,7 @@ constexpr int kSelOutliers = 0;    // tokens the filter took out of their groups
 constexpr int kSelDone = 1;        // [3] CTAs that have finished level 0, 1, 2
 constexpr int kSelPrefix = 4;      // [2] bits of tau fixed after level 0, 1
 constexpr int kSelRank = 6;        // [2] rank (counted from the largest) still to be skipped inside that prefix
+constexpr int kSelOffsetsDone = 9; // heads whose block offsets are complete
 constexpr int kSelFinished = 8;    // tau is final (budget 0 or everything): the refinement kernels return at once
 constexpr int kSelHist = 16;       // [3][2048] histograms of bits 31-21, 20-10, 9-0
 constexpr int kSelWords = kSelHist + 3 * 2048;

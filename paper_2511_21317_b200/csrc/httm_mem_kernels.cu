@@ -1136,10 +1136,11 @@ cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count,
 //                      merged length, and the head's first 128-row query tile (for the attention kernel)
 // ------------------------------------------------------------------------------------
 __device__ void finish_level(const OutlierArgs& a, int level, int* hist);   // (threshold selection, below)
-constexpr int kDevWarps = 6;   // 6 x 16.3 KB of shared memory: two CTAs per SM
-constexpr int kCentStride = 65;                                        // floats per centroid row: odd, so that row-wise reads spread over the banks
-constexpr int kDevAux = 32 * kCentStride * 4 + 32 * 4 + 16;           // centroids, reciprocal group sizes, 2 mbarriers
-constexpr int kDevSmem = kDevWarps * (2 * 32 * kRowBytes + kDevAux) + 2048 * 4 /*histogram*/ + 1024 /*alignment slack*/;
+constexpr int kDevWarps = 6;     // 6 x 16.2 KB of shared memory: two CTAs per SM
+constexpr int kDevStages = 3;    // block loads in flight per warp (the kernel is bound by bytes in flight)
+constexpr int kCentStride = 65;  // floats per mean: odd, so that reads of different means spread over the banks
+constexpr int kDevAux = 16 * kCentStride * 4 + 16 * 4 + 32;   // means of the groups of two or more (at most 16 in 32 tokens), reciprocal sizes, mbarriers
+constexpr int kDevSmem = kDevWarps * (kDevStages * 32 * kRowBytes + kDevAux) + 2048 * 4 /*histogram*/ + 1024 /*alignment slack*/;
 
 __global__ void __launch_bounds__(kDevWarps * 32, 2)
 deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a) {
@@ -1148,17 +1149,16 @@ deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a)
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;   // MMA accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
-    unsigned char* stage = smem + (size_t)warp * 2 * STAGE_BYTES;
-    unsigned char* aux = smem + (size_t)kDevWarps * 2 * STAGE_BYTES + (size_t)warp * kDevAux;
-    float* cent = reinterpret_cast<float*>(aux);                  // [32][65] group means
-    float* rcnt = cent + 32 * kCentStride;                         // [32] 1 / group size
-    int* hist = reinterpret_cast<int*>(smem + (size_t)kDevWarps * (2 * STAGE_BYTES + kDevAux));   // [2048] bits 31-21 of this CTA's deviations
+    unsigned char* stage = smem + (size_t)warp * kDevStages * STAGE_BYTES;
+    unsigned char* aux = smem + (size_t)kDevWarps * kDevStages * STAGE_BYTES + (size_t)warp * kDevAux;
+    float* cent = reinterpret_cast<float*>(aux);                   // [16][65] group means
+    float* rcnt = cent + 16 * kCentStride;                         // [16] 1 / group size
+    int* hist = reinterpret_cast<int*>(smem + (size_t)kDevWarps * (kDevStages * STAGE_BYTES + kDevAux));   // [2048] bits 31-21 of this CTA's deviations
     for (int i = threadIdx.x; i < 2048; i += kDevWarps * 32) hist[i] = 0;
     __syncthreads();
-    const uint32_t mbar0 = smem_u32(aux + 32 * kCentStride * 4 + 32 * 4), stage0 = smem_u32(stage);
+    const uint32_t mbar0 = smem_u32(aux + 16 * kCentStride * 4 + 16 * 4), stage0 = smem_u32(stage);
     if (lane == 0) {
-        mbar_init(mbar0, 1);
-        mbar_init(mbar0 + 8, 1);
+        for (int st = 0; st < kDevStages; ++st) mbar_init(mbar0 + 8 * st, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -1167,10 +1167,8 @@ deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a)
     const int box_f = min(L.blk_frames, L.frames), box_h = min(L.blk_h, L.grid_h), box_w = min(L.blk_w, L.grid_w);
     const int box_rows = box_f * box_h * box_w;
     const int own_t = lane / (box_h * box_w), own_y = (lane / box_w) % box_h, own_x = lane % box_w;
-    for (int q = box_rows * 8 + lane; q < 32 * 8; q += 32) {   // rows no load ever writes enter the MMAs with weight 0: keep them finite
-        *reinterpret_cast<uint4*>(stage + q * 16) = make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(stage + STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
-    }
+    for (int q = box_rows * 8 + lane; q < 32 * 8; q += 32)   // rows no load ever writes enter the MMAs with weight 0: keep them finite
+        for (int st = 0; st < kDevStages; ++st) *reinterpret_cast<uint4*>(stage + st * STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
     __syncwarp();
     BoxMap bm;
     bm.clipped = false;
@@ -1187,17 +1185,17 @@ deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a)
         mbar_expect_tx(mb, (uint32_t)box_rows * kRowBytes);
         tma_block_load(stage0 + buf * STAGE_BYTES, &map_q, mb, bg.x0, bg.y0, bg.s0, c.h);
     };
-    if (first < n_tasks && lane == 0) issue(nxt, 0);
-    nxt.advance();
-    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
-    nxt.advance();
+#pragma unroll
+    for (int st = 0; st < kDevStages; ++st) {
+        if (first + st * stride < n_tasks && lane == 0) issue(nxt, st);
+        nxt.advance();
+    }
 
-    int it = 0;
+    int buf = 0;
+    uint32_t parity = 0;
     bool failed = false;
-    for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
-        const int buf = it & 1;
-        const uint32_t parity = (it >> 1) & 1;
-        const bool more = task + 2 * stride < n_tasks;
+    for (int64_t task = first; task < n_tasks; task += stride, cur.advance(), nxt.advance()) {
+        const bool more = task + kDevStages * stride < n_tasks;
         const int h = cur.h;
         const BlockInfo bi = a.blocks[cur.u];
         const BlockGeom bg = a.geom[cur.u];
@@ -1222,13 +1220,13 @@ deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a)
             if (tok >= 0) eps[tok] = 0.f;
         } else {
             const uint32_t blk = stage0 + buf * STAGE_BYTES;
-            const unsigned kept = __ballot_sync(0xffffffffu, rep == lane);
-            const int n_kept = __popc(kept);
-            const int row_of = rep >= 0 ? __popc(kept & ((1u << rep) - 1u)) : -1;
-            const unsigned group = __match_any_sync(0xffffffffu, row_of);
-            const int group_size = __popc(group);
-            if (rep == lane) rcnt[row_of] = 1.0f / (float)group_size;
-            // group sums = W x on the tensor cores, exactly as in merge_tc_kernel
+            // groups of two or more tokens get a mean; row of the mean = rank of the group's representative among them
+            const unsigned group = __match_any_sync(0xffffffffu, rep);   // (lanes without a token share rep = -1: ignored below)
+            const int group_size = rep >= 0 ? __popc(group) : 0;
+            const unsigned multi = __ballot_sync(0xffffffffu, rep == lane && group_size >= 2);
+            const int row_of = group_size >= 2 ? __popc(multi & ((1u << rep) - 1u)) : -1;
+            if (rep == lane && group_size >= 2) rcnt[row_of] = 1.0f / (float)group_size;
+            // group sums = W x on the tensor cores, as in merge_tc_kernel: W [16 means][32 tokens] of zeros and ones
             uint32_t bf[2][4][4];
             const int n_ks = box_rows > 16 ? 2 : 1;
 #pragma unroll
@@ -1240,52 +1238,43 @@ deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a)
                     for (int np = 0; np < 4; ++np) ldmatrix_x4_trans(bf[ks][np], rowaddr + (((2 * np + (lane >> 4)) ^ (row & 7)) << 4));
                 }
             }
-            int rw[2][4];
+            float c[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+            const int r0 = g, r1 = g + 8;
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
-                rw[ks][0] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq);
-                rw[ks][1] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 1);
-                rw[ks][2] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 8);
-                rw[ks][3] = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 9);
+                if (ks < n_ks) {
+                    const int w0 = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq), w1 = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 1);
+                    const int w2 = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 8), w3 = __shfl_sync(0xffffffffu, row_of, 16 * ks + 2 * tq + 9);
+                    uint32_t af[4];
+                    af[0] = (w0 == r0 ? 0x3f80u : 0u) | (w1 == r0 ? 0x3f800000u : 0u);
+                    af[1] = (w0 == r1 ? 0x3f80u : 0u) | (w1 == r1 ? 0x3f800000u : 0u);
+                    af[2] = (w2 == r0 ? 0x3f80u : 0u) | (w3 == r0 ? 0x3f800000u : 0u);
+                    af[3] = (w2 == r1 ? 0x3f80u : 0u) | (w3 == r1 ? 0x3f800000u : 0u);
+#pragma unroll
+                    for (int nt = 0; nt < 8; ++nt) mma_bf16_16816(c[nt], af, bf[ks][nt >> 1][2 * (nt & 1)], bf[ks][nt >> 1][2 * (nt & 1) + 1]);
+                }
             }
             __syncwarp();   // reciprocal group sizes visible
-            const int n_mt = n_kept > 16 ? 2 : 1;
-#pragma unroll 1
-            for (int mt = 0; mt < n_mt; ++mt) {
-                const int r0 = 16 * mt + g, r1 = r0 + 8;
-                float c[8][4];
+            const int n_cent = __popc(multi);
+            const float i0 = r0 < n_cent ? rcnt[r0] : 0.f, i1 = r1 < n_cent ? rcnt[r1] : 0.f;
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
-#pragma unroll
-                for (int ks = 0; ks < 2; ++ks) {
-                    if (ks < n_ks) {
-                        uint32_t af[4];
-                        af[0] = (rw[ks][0] == r0 ? 0x3f80u : 0u) | (rw[ks][1] == r0 ? 0x3f800000u : 0u);
-                        af[1] = (rw[ks][0] == r1 ? 0x3f80u : 0u) | (rw[ks][1] == r1 ? 0x3f800000u : 0u);
-                        af[2] = (rw[ks][2] == r0 ? 0x3f80u : 0u) | (rw[ks][3] == r0 ? 0x3f800000u : 0u);
-                        af[3] = (rw[ks][2] == r1 ? 0x3f80u : 0u) | (rw[ks][3] == r1 ? 0x3f800000u : 0u);
-#pragma unroll
-                        for (int nt = 0; nt < 8; ++nt) mma_bf16_16816(c[nt], af, bf[ks][nt >> 1][2 * (nt & 1)], bf[ks][nt >> 1][2 * (nt & 1) + 1]);
-                    }
+            for (int nt = 0; nt < 8; ++nt) {   // the means stay in fp32 (no rounding to bf16 before the distance)
+                if (r0 < n_cent) {
+                    cent[r0 * kCentStride + nt * 8 + 2 * tq] = c[nt][0] * i0;
+                    cent[r0 * kCentStride + nt * 8 + 2 * tq + 1] = c[nt][1] * i0;
                 }
-                const float i0 = r0 < n_kept ? rcnt[r0] : 0.f, i1 = r1 < n_kept ? rcnt[r1] : 0.f;
-#pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {   // the means stay in fp32 (no rounding to bf16 before the distance)
-                    if (r0 < n_kept) {
-                        cent[r0 * kCentStride + nt * 8 + 2 * tq] = c[nt][0] * i0;
-                        cent[r0 * kCentStride + nt * 8 + 2 * tq + 1] = c[nt][1] * i0;
-                    }
-                    if (r1 < n_kept) {
-                        cent[r1 * kCentStride + nt * 8 + 2 * tq] = c[nt][2] * i1;
-                        cent[r1 * kCentStride + nt * 8 + 2 * tq + 1] = c[nt][3] * i1;
-                    }
+                if (r1 < n_cent) {
+                    cent[r1 * kCentStride + nt * 8 + 2 * tq] = c[nt][2] * i1;
+                    cent[r1 * kCentStride + nt * 8 + 2 * tq + 1] = c[nt][3] * i1;
                 }
             }
             __syncwarp();   // means visible
             float dev = 0.f;
             if (tok >= 0) {
                 float d2 = 0.f;
-                if (group_size >= 2) {   // distance of this lane's token (stage row `lane`) to its group's mean
+                if (row_of >= 0) {   // distance of this lane's token (stage row `lane`) to its group's mean
                     const unsigned char* row = stage + buf * STAGE_BYTES + lane * kRowBytes;
                     const float* cr = cent + row_of * kCentStride;
 #pragma unroll
@@ -1309,10 +1298,16 @@ deviation_kernel(const __grid_constant__ CUtensorMap map_q, const OutlierArgs a)
         }
         __syncwarp();   // every lane is done with the stage and the tables
         if (more && lane == 0) issue(nxt, buf);
+        if (++buf == kDevStages) {
+            buf = 0;
+            parity ^= 1u;
+        }
     }
-    if (failed) {
-        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
-        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+    if (failed) {   // give copies that may still be in flight a bounded chance to land before the shared memory is released
+        for (int st = 0; st < kDevStages; ++st) {
+            mbar_wait_bounded(mbar0 + 8 * st, parity, a.status, kDevTimeoutMatchLoad);
+            mbar_wait_bounded(mbar0 + 8 * st, parity ^ 1u, a.status, kDevTimeoutMatchLoad);
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < 2048; i += kDevWarps * 32) {
@@ -1468,32 +1463,54 @@ __global__ void __launch_bounds__(256) filter_kernel(const OutlierArgs a) {
     }
 }
 
-// Per head: merged row of every block's first kept token = specials + exclusive prefix sum of the kept counts;
-// merged length; then, over the heads, the index of each head's first 128-row query tile.  One CTA, a warp per head.
-__global__ void __launch_bounds__(1024, 1) offsets_kernel(const OutlierArgs a) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
-    for (int h = warp; h < a.heads; h += n_warps) {
-        int running = a.n_special_total;
-        for (int b0 = 0; b0 < a.n_blocks; b0 += 32) {
-            const int b = b0 + lane;
-            const int c = b < a.n_blocks ? a.kept_cnt[(int64_t)h * a.n_blocks + b] : 0;
-            int incl = c;
+// Per head (one CTA each): merged row of every block's first kept token = specials + exclusive prefix sum of the kept
+// counts, and the merged length.  The CTA that finishes last builds, over the heads, the index of each head's first
+// 128-row query tile (for the attention kernel).
+constexpr int kOffsetsThreads = 1024;
+__global__ void __launch_bounds__(kOffsetsThreads, 1) offsets_kernel(const OutlierArgs a) {
+    __shared__ int warp_sum[32];
+    __shared__ int s_last;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, h = blockIdx.x;
+    const int32_t* cnt = a.kept_cnt + (int64_t)h * a.n_blocks;
+    int32_t* moff = a.moff_var + (int64_t)h * a.n_blocks;
+    int running = a.n_special_total;
+    for (int b0 = 0; b0 < a.n_blocks; b0 += kOffsetsThreads) {
+        const int b = b0 + threadIdx.x;
+        const int c = b < a.n_blocks ? cnt[b] : 0;
+        int incl = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {   // inclusive scan of the 32 warp totals
+            int w = warp_sum[lane];
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const int o = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += o;
+                const int o = __shfl_up_sync(0xffffffffu, w, off);
+                if (lane >= off) w += o;
             }
-            if (b < a.n_blocks) a.moff_var[(int64_t)h * a.n_blocks + b] = running + incl - c;
-            running += __shfl_sync(0xffffffffu, incl, 31);
+            warp_sum[lane] = w;
         }
-        if (lane == 0) a.mq_head[h] = running;
+        __syncthreads();
+        if (b < a.n_blocks) moff[b] = running + (warp > 0 ? warp_sum[warp - 1] : 0) + incl - c;
+        running += warp_sum[31];
+        __syncthreads();   // the totals are read before the next chunk overwrites them
+    }
+    if (threadIdx.x == 0) {
+        a.mq_head[h] = running;
+        __threadfence();
+        s_last = atomicAdd(a.sel + kSelOffsetsDone, 1) == (int)gridDim.x - 1;
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (s_last && threadIdx.x == 0) {
+        __threadfence();
         int t = 0;
-        for (int h = 0; h < a.heads; ++h) {
-            a.tile_prefix[h] = t;
-            t += (a.mq_head[h] + 127) / 128;
+        for (int hh = 0; hh < a.heads; ++hh) {
+            a.tile_prefix[hh] = t;
+            t += (__ldcg(a.mq_head + hh) + 127) / 128;
         }
         a.tile_prefix[a.heads] = t;
     }
@@ -1525,7 +1542,7 @@ cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream) {
     filter_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    offsets_kernel<<<1, 1024, 0, stream>>>(a);
+    offsets_kernel<<<(unsigned)a.heads, kOffsetsThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

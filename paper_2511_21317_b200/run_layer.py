@@ -1,6 +1,7 @@
 """Run a few HTTM global-attention layers of a named synthetic workload and nothing else.
 
     python -m paper_2511_21317_b200.run_layer --workload medium --calls 2 [--dense 1] [--stages 1] [--ratio 0.9] [--block 4x4x4]
+                                              [--outlier-fraction 0.01]
 
 A profiler is pointed at this command: few launches, no timing loops, no CPU work besides
 the input generator.  It prints the merged lengths and the device status word, and exits
@@ -27,6 +28,7 @@ def main() -> int:
     ap.add_argument("--heads", type=int, default=None, help="override the number of heads")
     ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
     ap.add_argument("--block", default=None, help="override the block shape, e.g. 4x4x4")
+    ap.add_argument("--outlier-fraction", type=float, default=0.0, help="query outlier filtering (Sec. 3.4) in the public calls")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
     if args.heads is not None:
@@ -42,11 +44,14 @@ def main() -> int:
     with hb.Httm(hb.HttmConfig.of(wl, device=0)) as ctx:
         dq, dk, dv = (hb.bf16_from_bits(x, "cuda:0") for x in (q, k, v))
         out = ctx.new_output()
+        if args.outlier_fraction > 0:
+            ctx.set_outlier_fraction(args.outlier_fraction)
         for _ in range(args.calls):
             ctx.global_attention(dq, dk, dv, out)
         for _ in range(args.dense):
             ctx.dense_attention(dq, dk, dv, out)
         direct = True   # every supported geometry has the direct kernels
+        ctx.set_outlier_fraction(0.0)
         for _ in range(args.stages):
             for st in [0, 1, 2] + ([5, 6] if direct else []) + [3, 4]:
                 ctx.launch_stage(st, dq, dk, dv, out)
