@@ -48,6 +48,10 @@ class Workload:
     head_dim: int = 64
     sigma: float = 0.1
     seed: int = 0
+    # Shape of the patch grid the synthetic field is drawn on, when it differs from (grid_h, grid_w): the 1-D block
+    # regime hands the library a frame's patch tokens as one run (grid 1 x P) of a field_h x field_w image.
+    field_h: int = 0
+    field_w: int = 0
 
     @property
     def n_special(self) -> int:
@@ -76,6 +80,9 @@ WORKLOADS = {
     "medium": _wl("medium", 24, 37, (2, 4, 4), 0.7),
     "large": _wl("large", 100, 37, (4, 4, 4), 0.8, sigma=0.3),
     "stack_layer": _wl("stack_layer", 48, 37, (2, 4, 4), 0.7),
+    # The paper's own block regime (Sec. 4.1): runs of n_s = 128 patch tokens in raster order over n_t = 30 frames
+    # (blocks of 3840 tokens), 90 % of the queries and 70 % of the keys / values merged.
+    "paper_1d": Workload("paper_1d", 60, 1, 37 * 37, 30, 1, 128, 0.9, 0.7, field_h=37, field_w=37),
 }
 
 
@@ -116,7 +123,10 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 
 
 def _one_head(wl: Workload, tensor: int, head: int) -> np.ndarray:
-    S, h, w, D, nsp = wl.frames, wl.grid_h, wl.grid_w, wl.head_dim, wl.n_special
+    S, D, nsp = wl.frames, wl.head_dim, wl.n_special
+    h, w = (wl.field_h, wl.field_w) if wl.field_h > 0 else (wl.grid_h, wl.grid_w)
+    if h * w != wl.grid_h * wl.grid_w:
+        raise ValueError("field_h x field_w must hold as many patches as grid_h x grid_w")
     P = wl.tokens_per_frame
     # lattice [D][8][8]
     lat = _normals(_stream_key(wl.seed, tensor, head, 0), np.arange(D * _LATTICE * _LATTICE)).reshape(

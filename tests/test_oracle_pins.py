@@ -461,3 +461,54 @@ def test_merged_length_golden_table():
     for S, grid, bt, bh, bw, rho, M in rows:
         g = orc.Geometry(int(S), 5, int(grid), int(grid), 16, 64, int(bt), int(bh), int(bw))
         assert orc.merged_len(g, float(rho)) == int(M)
+
+
+# ---------------------------------------------------------------- the paper's 1-D block regime (Sec. 3.3 / 4.1)
+
+
+def test_runs_of_one_grid_row_equal_row_windows():
+    """Sec. 3.3 defines spatial blocks as runs of n_s consecutive tokens of a frame.  Handing the frame over as a
+    1 x (h w) grid with 1 x n_s windows is that definition; for n_s = w the runs are the rows of the h x w grid, so
+    both geometries must give the same permutation, maps and output."""
+    h, w, S = 4, 6, 5
+    g2 = geom(S=S, nsp=2, h=h, w=w, H=2, D=8, blk=(3, 1, w))
+    g1 = geom(S=S, nsp=2, h=1, w=h * w, H=2, D=8, blk=(3, 1, w))
+    N = orc.num_tokens(g2)
+    q, k, v = (rand_bf16((2, N, 8), s) for s in (71, 72, 73))
+    a = orc.global_attention(g2, 0.6, 0.4, q, k, v)
+    b = orc.global_attention(g1, 0.6, 0.4, q, k, v)
+    assert np.array_equal(a.pi, b.pi) and np.array_equal(a.blk_start, b.blk_start)
+    assert np.array_equal(a.assign_q, b.assign_q) and np.array_equal(a.assign_k, b.assign_k)
+    assert np.array_equal(a.out, b.out)
+
+
+def test_large_run_blocks_match_by_brute_force():
+    """Blocks of several hundred tokens (runs of 100 tokens over 4 frames, the last run ragged): the map equals a plain
+    loop over src x dst cosines with the top-r rule, at the budgets of the paper's configuration (0.9 / 0.7)."""
+    g = geom(S=4, nsp=1, h=1, w=230, H=1, D=16, blk=(4, 1, 100))
+    pi, bs = orc.temporal_reorder(g)
+    assert np.diff(bs).tolist() == [400, 400, 120]
+    x = rand_bf16((1, orc.num_tokens(g), 16), 9)
+    xr = as_f64(orc.reorder(g, pi, x))[0]
+    for rho in (0.9, 0.7):
+        A = orc.match(g, bs, rho, orc.reorder(g, pi, x), margins=False)[0]
+        for b in range(len(bs) - 1):
+            base, n = int(bs[b]), int(bs[b + 1] - bs[b])
+            r = min(int(np.floor(rho * n + 1e-9)), n - 1)
+            nd = min(-(-n // 4), n - r)
+            dst = [j for j in range(n) if ((j + 1) * nd) // n > (j * nd) // n]
+            assert len(dst) == nd
+            blk = xr[base:base + n]
+            nrm = np.maximum(np.sqrt((blk * blk).sum(1)), 1e-12)
+            best = []
+            for a in range(n):
+                if a in dst:
+                    continue
+                sims = [float(blk[a] @ blk[d]) / (nrm[a] * nrm[d]) for d in dst]
+                j = max(range(nd), key=lambda t: (sims[t], -t))
+                best.append((-sims[j], a, dst[j]))
+            best.sort()
+            expect = np.arange(n)
+            for _, a, d in best[:r]:
+                expect[a] = d
+            assert np.array_equal(A[base:base + n] - base, expect)
