@@ -39,7 +39,7 @@ extern "C" {
 typedef enum {
     HTTM_OK = 0,
     HTTM_ERR_INVALID_ARG = -1, /* null pointer, value out of range, overlapping output */
-    HTTM_ERR_UNSUPPORTED = -2, /* head_dim != 64, block of more than 256 tokens, ...  */
+    HTTM_ERR_UNSUPPORTED = -2, /* head_dim != 64, block of more than 4096 tokens, ... */
     HTTM_ERR_ALIGNMENT = -3,   /* pointer not 16-byte aligned / stride not multiple of 8 */
     HTTM_ERR_NOMEM = -4,       /* device or host allocation failed                     */
     HTTM_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed (see last_error)  */
@@ -117,7 +117,12 @@ enum {
     HTTM_STAGE_UNMERGE = 4,
     HTTM_STAGE_MATCH_DIRECT = 5,
     HTTM_STAGE_MERGE_DIRECT = 6,
-    HTTM_STAGE_OUTLIER_FILTER = 7 /* between 5 and 6, only after httm_set_outlier_fraction(> 0): five small kernels */
+    HTTM_STAGE_OUTLIER_FILTER = 7,/* between 5 and 6, only after httm_set_outlier_fraction(> 0): five small kernels */
+    /* merging blocks of 257 .. 4096 tokens (the paper's runs of 128 tokens over 30 frames, Sec. 4.1): stages 1, 5, 6 are
+     * UNSUPPORTED; the order is 0, 8, 9, 2, 3, 4.  8: cosine of every token with every dst token of its block on the
+     * tensor cores + best dst per token; 9: the r best src of every block merge (map written) */
+    HTTM_STAGE_BIG_SCORES = 8,
+    HTTM_STAGE_BIG_SELECT = 9
 };
 
 /*

@@ -52,6 +52,13 @@ struct httm_ctx {
     int32_t* d_sel = nullptr;   // state of the threshold selection, first word = outlier counter
     float *d_eps = nullptr, *d_tau = nullptr;
     __nv_bfloat16 *d_qm_var = nullptr, *d_om_var = nullptr;
+    // large merging blocks (257 .. 4096 tokens, Sec. 4.1): matching as a tensor-core contraction, see httm_big_blocks.cu
+    std::vector<BigItem> big_items;
+    BigItem* d_big_items = nullptr;
+    float *d_inv_norm_q = nullptr, *d_inv_norm_k = nullptr;
+    uint32_t *d_best_key_q = nullptr, *d_best_key_k = nullptr;
+    int32_t *d_best_pos_q = nullptr, *d_best_pos_k = nullptr;
+    bool big() const { return max_block > kMaxBlockTokens; }
     bool filtering() const { return outlier_fraction > 0.0; }
     int32_t q_rows() const { return filtering() ? n_tokens : m_q; }   // rows per head of Q_m and O_m
     // staging for the host-buffer entry point (allocated on first use)
@@ -93,7 +100,8 @@ struct httm_ctx {
     void release() {
         void* ptrs[] = {d_geom, d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
                         d_vr, d_qm,     d_km,       d_vm,       d_om,     hs[0].q,  hs[0].k,  hs[0].v, hs[0].out, hs[1].q, hs[1].k, hs[1].v, hs[1].out,
-                        d_assign_qf, d_kept_cnt, d_moff_var, d_mq_head, d_tile_prefix, d_sel, d_eps, d_tau, d_qm_var, d_om_var};
+                        d_assign_qf, d_kept_cnt, d_moff_var, d_mq_head, d_tile_prefix, d_sel, d_eps, d_tau, d_qm_var, d_om_var,
+                        d_big_items, d_inv_norm_q, d_inv_norm_k, d_best_key_q, d_best_key_k, d_best_pos_q, d_best_pos_k};
         for (void* p : ptrs)
             if (p) cudaFree(p);
         for (HostSet& h : hs)
@@ -177,6 +185,8 @@ int stage_reorder(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const
     a.pi = c->d_pi;
     a.n_tokens = c->n_tokens;
     a.heads = c->cfg.heads;
+    a.inv_norm[0] = c->d_inv_norm_q;   // (null unless the context has large blocks)
+    a.inv_norm[1] = c->d_inv_norm_k;
     c->launches++;
     return check_cuda(c, launch_reorder(a, s), "reorder launch");
 }
@@ -198,8 +208,39 @@ SourceLayout source_layout(const httm_ctx* c) {
 // the reordered copies are not needed on the hot path (the 16-bit block coordinates bound the scene size).
 bool direct_mode(const httm_ctx* c) { return c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767; }
 
+BigMatchArgs big_match_args(httm_ctx* c) {
+    BigMatchArgs a{};
+    a.xr[0] = c->d_qr;
+    a.xr[1] = c->d_kr;
+    a.inv_norm[0] = c->d_inv_norm_q;
+    a.inv_norm[1] = c->d_inv_norm_k;
+    a.best_key[0] = c->d_best_key_q;
+    a.best_key[1] = c->d_best_key_k;
+    a.best_pos[0] = c->d_best_pos_q;
+    a.best_pos[1] = c->d_best_pos_k;
+    a.assign[0] = c->d_assign_q;
+    a.assign[1] = c->d_assign_k;
+    a.blocks = c->d_blocks;
+    a.items = c->d_big_items;
+    a.n_items = (int32_t)c->big_items.size();
+    a.n_blocks = c->n_blocks;
+    a.n_tokens = c->n_tokens;
+    a.heads = c->cfg.heads;
+    a.status = c->d_status;
+    return a;
+}
+int stage_big_scores(httm_ctx* c, cudaStream_t s) {
+    c->launches++;
+    return check_cuda(c, launch_big_scores(big_match_args(c), c->sm_count, s), "large-block score launch");
+}
+int stage_big_select(httm_ctx* c, cudaStream_t s) {
+    c->launches++;
+    return check_cuda(c, launch_big_select(big_match_args(c), s), "large-block select launch");
+}
+
 // src: the original Q, K, V (direct mode) or nullptr (blocks come from the reordered copies)
 int stage_match(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
+    if (c->big()) return c->fail(HTTM_ERR_UNSUPPORTED, "blocks of more than 256 tokens are matched by the large-block stages");
     MatchArgs a{};
     if (src) {
         a.geom = c->d_geom;
@@ -221,6 +262,7 @@ int stage_match(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
 }
 
 int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
+    if (c->big() && src) return c->fail(HTTM_ERR_UNSUPPORTED, "blocks of more than 256 tokens are merged from the reordered copies");
     MergeArgs a{};
     if (src) {
         a.geom = c->d_geom;
@@ -248,6 +290,7 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.m_k = c->m_k;
     a.status = c->d_status;
     c->launches++;
+    if (c->big()) return check_cuda(c, launch_big_merge(a, s), "large-block merge launch");
     return check_cuda(c, launch_merge(a, c->max_block, c->sm_count, s), "merge launch");
 }
 
@@ -339,6 +382,14 @@ int dense_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const ht
 int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out,
                 cudaStream_t s) {
     int rc;
+    if (c->big()) {   // six kernels: reorder (+ norms), scores, select, merge, attention, unmerge
+        if ((rc = stage_reorder(c, q, k, v, s))) return rc;
+        if ((rc = stage_big_scores(c, s))) return rc;
+        if ((rc = stage_big_select(c, s))) return rc;
+        if ((rc = stage_merge(c, s))) return rc;
+        if ((rc = stage_attention(c, s))) return rc;
+        return stage_unmerge(c, out, s);
+    }
     if (direct_mode(c)) {   // four kernels: the temporal reorder is folded into the block loads of match and merge
         const httm_tensor src[3] = {q, k, v};
         if ((rc = stage_match(c, s, src))) return rc;
@@ -390,7 +441,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
         return bad(HTTM_ERR_UNSUPPORTED, "too many tokens (N <= 2^24 and N*heads < 2^31)");
     const int64_t bf = std::min<int64_t>(cfg->blk_frames, cfg->frames), bh = std::min<int64_t>(cfg->blk_h, cfg->grid_h),
                   bw = std::min<int64_t>(cfg->blk_w, cfg->grid_w);
-    if (bf * bh * bw > kMaxBlockTokens) return bad(HTTM_ERR_UNSUPPORTED, "a merging block may hold at most 256 tokens");
+    if (bf * bh * bw > kMaxBigBlockTokens) return bad(HTTM_ERR_UNSUPPORTED, "a merging block may hold at most 4096 tokens");
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) {
         cudaGetLastError();
@@ -429,6 +480,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
                 moff_q += bi.n - bi.r_q;
                 moff_k += bi.n - bi.r_k;
                 c->max_block = std::max(c->max_block, bi.n);
+                for (int row0 = 0; row0 < bi.n; row0 += kBigSliceRows) c->big_items.push_back(BigItem{(int32_t)c->blocks.size(), row0});
                 c->blk_start.push_back(pos);
                 c->blocks.push_back(bi);
                 c->geom.push_back(BlockGeom{(int16_t)g0, (int16_t)y0, (int16_t)x0, (int16_t)f, (int16_t)hh, (int16_t)ww});
@@ -463,6 +515,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
                                                prop.major, prop.minor));
     c->sm_count = prop.multiProcessorCount;
     if ((rc = check_cuda(c, configure_kernels(), "cudaFuncSetAttribute"))) return done(rc);
+    if ((rc = check_cuda(c, configure_big_blocks(), "cudaFuncSetAttribute"))) return done(rc);
 
     const size_t H = cfg->heads, N = c->n_tokens;
     if ((rc = c->alloc(&c->d_pi, N)) || (rc = c->alloc(&c->d_pi_inv, N)) || (rc = c->alloc(&c->d_blocks, c->blocks.size())) || (rc = c->alloc(&c->d_geom, c->geom.size())) ||
@@ -473,6 +526,15 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
         (rc = c->alloc(&c->d_vm, H * c->m_k * kHeadDim)) || (rc = c->alloc(&c->d_om, H * c->m_q * kHeadDim)))
         return done(rc);
 
+    if (c->big()) {
+        if ((rc = c->alloc(&c->d_big_items, c->big_items.size())) || (rc = c->alloc(&c->d_inv_norm_q, H * N)) ||
+            (rc = c->alloc(&c->d_inv_norm_k, H * N)) || (rc = c->alloc(&c->d_best_key_q, H * N)) || (rc = c->alloc(&c->d_best_key_k, H * N)) ||
+            (rc = c->alloc(&c->d_best_pos_q, H * N)) || (rc = c->alloc(&c->d_best_pos_k, H * N)))
+            return done(rc);
+        if ((rc = check_cuda(c, cudaMemcpy(c->d_big_items, c->big_items.data(), c->big_items.size() * sizeof(BigItem), cudaMemcpyHostToDevice),
+                             "item table upload")))
+            return done(rc);
+    }
     // uploads; special tokens are never merged: their map entries are constants, written once
     std::vector<int32_t> ident(H * N);
     for (size_t hd = 0; hd < H; ++hd)
@@ -616,6 +678,10 @@ int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm
         case HTTM_STAGE_UNMERGE:
             if ((rc = check_tensor(c, out, "out"))) return rc;
             return stage_unmerge(c, out, s);
+        case HTTM_STAGE_BIG_SCORES:
+        case HTTM_STAGE_BIG_SELECT:
+            if (!c->big()) return c->fail(HTTM_ERR_UNSUPPORTED, "the large-block stages need merging blocks of more than 256 tokens");
+            return stage == HTTM_STAGE_BIG_SCORES ? stage_big_scores(c, s) : stage_big_select(c, s);
         case HTTM_STAGE_OUTLIER_FILTER:
             if (!c->filtering()) return c->fail(HTTM_ERR_INVALID_ARG, "outlier filtering is off: call httm_set_outlier_fraction first");
             if ((rc = check_tensor(c, q, "q"))) return rc;

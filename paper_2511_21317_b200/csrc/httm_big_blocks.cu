@@ -1,0 +1,603 @@
+// Matching and merging for LARGE merging blocks (257 .. 4096 tokens): the paper's own regime of runs of
+// n_s = 128 tokens over n_t = 30 frames, 3840 tokens per block (Sec. 3.3, Sec. 4.1).  A block no longer fits one
+// warp's stage, and its similarity step (Eq. 1) is a real dense contraction: n tokens x n_dst dst tokens x 64.
+//
+//   big_scores_kernel   cosine of every token of a block with every dst token of the block on the 5th-generation
+//                       tensor cores (tcgen05.mma, accumulators in tensor memory), fused with the row-wise
+//                       arg-max: per token the best dst and the best cosine
+//   big_select_kernel   the r src tokens with the best cosines merge (Sec. 3.2): exact radix select per block,
+//                       ties by position; writes the assignment map
+//   big_merge_kernel    mean of every group (Sec. 3.2): tokens sorted by (merged row, position), one warp
+//                       gathers the members of a row in that order; writes merged Q / K / V and rank_q
+// All three read the reordered copies (a block is a contiguous run of rows there).
+#include "httm_internal.h"
+#include "tc_sm100.cuh"
+
+namespace httm {
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------ shared helpers
+__device__ __forceinline__ uint32_t score_key(float s) {   // unsigned keys order like the floats
+    const uint32_t b = __float_as_uint(s);
+    return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+}
+// token number (inside a block of n tokens) of dst d of n_dst evenly spaced dst tokens: the positions j with
+// floor((j + 1) n_dst / n) > floor(j n_dst / n), i.e. j = ceil((d + 1) n / n_dst) - 1
+__device__ __forceinline__ int dst_position(int d, int n, int nd) { return ((d + 1) * n + nd - 1) / nd - 1; }
+__device__ __forceinline__ bool is_dst_position(int j, int n, int nd) { return ((j + 1) * nd) / n > (j * nd) / n; }
+
+// ------------------------------------------------------------------------------------------------ scores
+constexpr int TILE = 128;                        // rows of an operand tile
+constexpr int TILE_BYTES = TILE * kRowBytes;     // 16 KB
+constexpr int kDstTiles = kMaxBigDst / TILE;     // 8 resident dst tiles
+constexpr int kSrcTilesPerItem = kBigSliceRows / TILE;   // 8
+constexpr int SC_THREADS = 320;                  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: arg-max (two column halves x four lane quadrants)
+constexpr int SC_TMEM_COLS = 512;                // two score buffers of 256 columns (one token tile x two dst tiles)
+
+struct ScoreBars {
+    uint64_t a_full[2], a_empty[2];   // ring of token tiles
+    uint64_t s_full[2], s_empty[2];   // score buffers
+    uint64_t x_full[2], x_done[2];    // exchange of the two column halves' results, by token-tile parity
+    uint32_t tmem_base;
+    int abort_flag;
+};
+constexpr int SC_OFF_A = kDstTiles * TILE_BYTES;                 // token tiles behind the dst tiles
+constexpr int SC_OFF_INV = SC_OFF_A + 2 * TILE_BYTES;            // float [1024] inverse norms of the dst tokens
+constexpr int SC_OFF_XCH = SC_OFF_INV + kMaxBigDst * 4;          // [2][128] (best, arg) of column half 1
+constexpr int SC_OFF_BARS = SC_OFF_XCH + 2 * TILE * 8;
+constexpr int SC_SMEM = SC_OFF_BARS + 256 + 1024 /*alignment slack*/;
+
+__global__ void __launch_bounds__(SC_THREADS, 1)
+big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const BigMatchArgs a) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t s_b = tc::smem_addr(smem), s_a = s_b + SC_OFF_A;
+    float* inv_d = reinterpret_cast<float*>(smem + SC_OFF_INV);
+    float2* xch = reinterpret_cast<float2*>(smem + SC_OFF_XCH);
+    ScoreBars* bars = reinterpret_cast<ScoreBars*>(smem + SC_OFF_BARS);
+    volatile int* abort_flag = &bars->abort_flag;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        bars->abort_flag = 0;
+        for (int i = 0; i < 2; ++i) {
+            tc::mbar_init(tc::smem_addr(&bars->a_full[i]), 1);
+            tc::mbar_init(tc::smem_addr(&bars->a_empty[i]), 1);
+            tc::mbar_init(tc::smem_addr(&bars->s_full[i]), 1);
+            tc::mbar_init(tc::smem_addr(&bars->s_empty[i]), 256);
+            tc::mbar_init(tc::smem_addr(&bars->x_full[i]), 128);
+            tc::mbar_init(tc::smem_addr(&bars->x_done[i]), 128);
+        }
+        tc::fence_barrier_init();
+        tc::prefetch_tensormap(&map_q);
+        tc::prefetch_tensormap(&map_k);
+    }
+    if (warp == 1) tc::tmem_alloc(tc::smem_addr(&bars->tmem_base), SC_TMEM_COLS);
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem = bars->tmem_base;
+
+    // completions so far of every barrier (each role counts its own): they give the phase parities across work items
+    uint32_t n_a[2] = {0, 0}, n_s[2] = {0, 0};   // token tiles per ring stage, score tiles per buffer
+    uint32_t n_x[2] = {0, 0};                    // exchanges per parity slot
+    const int64_t total = 2ll * a.heads * a.n_items;
+    constexpr uint32_t idesc = tc::idesc_bf16(128, 256, false, false);
+    constexpr uint64_t kTileStep = TILE_BYTES >> 4;   // descriptor address field counts 16-byte units
+
+    for (int64_t item = blockIdx.x;; item += gridDim.x) {
+        __syncthreads();   // every role is done with the previous item: dst tiles and tables may be rewritten
+        if (item >= total || bars->abort_flag) break;   // (the flag is only set between two of these barriers: same answer in every thread)
+        const int t = (int)(item / ((int64_t)a.heads * a.n_items));
+        const int64_t rem = item - (int64_t)t * a.heads * a.n_items;
+        const int h = (int)(rem / a.n_items);
+        const BigItem it = a.items[rem - (int64_t)h * a.n_items];
+        const BlockInfo bi = a.blocks[it.block];
+        const int n = bi.n, r = t == 0 ? bi.r_q : bi.r_k, nd = t == 0 ? bi.nd_q : bi.nd_k;
+        if (r == 0) continue;   // nothing merges in this block (uniform)
+        const int n_dd = (nd + 2 * TILE - 1) / (2 * TILE);                        // pairs of dst tiles
+        const int n_st = min(kSrcTilesPerItem, (n - it.row0 + TILE - 1) / TILE);  // token tiles of this slice
+        const int64_t head_row0 = (int64_t)h * a.n_tokens + bi.start;             // row of the block's first token in [H][N]
+
+        // ---- dst tokens of the block -> resident tiles (128-byte swizzle, as a tiled bulk copy would leave them)
+        {
+            const __nv_bfloat16* x = a.xr[t] + head_row0 * kHeadDim;
+            const float* inv = a.inv_norm[t] + head_row0;
+            const int chunk = tid & 7;
+            for (int d = tid >> 3; d < n_dd * 2 * TILE; d += SC_THREADS / 8) {
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);   // rows past the last dst token: zeros (their scores are masked)
+                float w = 0.f;
+                if (d < nd) {
+                    const int pos = dst_position(d, n, nd);
+                    v = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * kHeadDim) + chunk);
+                    w = __ldg(inv + pos);
+                }
+                const int row = d & (TILE - 1);
+                *reinterpret_cast<uint4*>(smem + (d >> 7) * TILE_BYTES + row * kRowBytes + ((chunk ^ (row & 7)) << 4)) = v;
+                if (chunk == 0) inv_d[d] = w;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor cores read these tiles through the async proxy
+        }
+        __syncthreads();
+
+        if (warp == 0) {
+            // ------------------------------------------------------------------ producer: token tiles of the slice
+            if (tc::elect_one()) {
+                for (int i = 0; i < n_st; ++i) {
+                    const int st = i & 1;
+                    if (!tc::mbar_wait(tc::smem_addr(&bars->a_empty[st]), (n_a[st] & 1u) ^ 1u, abort_flag)) break;
+                    const uint32_t bar = tc::smem_addr(&bars->a_full[st]);
+                    tc::mbar_expect_tx(bar, TILE_BYTES);
+                    // rows past the block's end belong to the next block (finite, results dropped) or are zero filled past N
+                    tc::tma_load_3d(s_a + st * TILE_BYTES, t == 0 ? &map_q : &map_k, bar, 0, bi.start + it.row0 + i * TILE, h);
+                    ++n_a[st];
+                }
+            } else {
+                for (int i = 0; i < n_st; ++i) ++n_a[i & 1];
+            }
+            __syncwarp();
+        } else if (warp == 1) {
+            // ------------------------------------------------------------------ issuer: S = X_tile . X_dst^T
+            if (tc::elect_one()) {
+                const uint64_t da0 = tc::smem_desc_sw128(s_a), db0 = tc::smem_desc_sw128(s_b);
+                bool ok = true;
+                auto issue = [&](uint32_t t_s, uint64_t da, uint64_t db, uint32_t bar) {   // four K = 16 steps over the 64 channels
+                    tc::mma_ss_c<false>(t_s, da, db, idesc);
+                    tc::mma_ss_c<true>(t_s, da + 2, db + 2, idesc);
+                    tc::mma_ss_c<true>(t_s, da + 4, db + 4, idesc);
+                    tc::mma_ss_c<true>(t_s, da + 6, db + 6, idesc);
+                    tc::mma_commit(bar);
+                };
+                for (int i = 0; ok && i < n_st; ++i) {
+                    const int st = i & 1;
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->a_full[st]), n_a[st] & 1u, abort_flag);
+                    if (!ok) break;
+                    tc::fence_after_sync();
+#pragma unroll
+                    for (int jj = 0; jj < kDstTiles / 2; ++jj) {   // buffer jj & 1: operands are bases plus constants
+                        if (jj < n_dd) {
+                            const int b = jj & 1;
+                            ok = ok && tc::mbar_wait(tc::smem_addr(&bars->s_empty[b]), (n_s[b] & 1u) ^ 1u, abort_flag);
+                            if (ok) {
+                                tc::fence_after_sync();
+                                issue(tmem + b * 256, da0 + (uint64_t)st * kTileStep, db0 + (uint64_t)(2 * jj) * kTileStep,
+                                      tc::smem_addr(&bars->s_full[b]));
+                                ++n_s[b];
+                            }
+                        }
+                    }
+                    if (ok) tc::mma_commit(tc::smem_addr(&bars->a_empty[st]));   // the tile may be refilled when these MMAs are done
+                    ++n_a[st];
+                }
+            } else {
+                for (int i = 0; i < n_st; ++i) {
+                    ++n_a[i & 1];
+                    for (int jj = 0; jj < n_dd; ++jj) ++n_s[jj & 1];
+                }
+            }
+            __syncwarp();
+        } else {
+            // ------------------------------------------------------------------ arg-max over the dst tokens, one thread per token and column half
+            const int half = (warp - 2) >> 2;                  // 0: dst tile 2 jj, 1: dst tile 2 jj + 1
+            const int row = (warp & 3) * 32 + lane;            // row of the token tile = lane of tensor memory
+            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+            bool ok = true;
+            for (int i = 0; ok && i < n_st; ++i) {
+                float best = -INFINITY;
+                int arg = 0;
+                for (int jj = 0; ok && jj < n_dd; ++jj) {
+                    const int b = jj & 1;
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->s_full[b]), n_s[b] & 1u, abort_flag);
+                    if (!ok) break;
+                    tc::fence_after_sync();
+                    ++n_s[b];
+                    const int col0 = (2 * jj + half) * TILE;   // first dst of this thread's 128 columns
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+                        uint32_t raw[64];
+                        const uint32_t taddr = tmem + b * 256 + half * TILE + part * 64 + lane_addr;
+                        tc::tmem_ld32(taddr, raw);
+                        tc::tmem_ld32(taddr + 32, raw + 32);
+                        tc::tmem_wait_ld();
+                        if (part == 1) {   // both parts are in registers: the buffer can take the next scores
+                            tc::fence_before_sync();
+                            tc::mbar_arrive(tc::smem_addr(&bars->s_empty[b]));
+                        }
+                        const int c0 = col0 + part * 64;
+                        if (c0 < nd) {     // (uniform in the warp)
+                            const float4* w4 = reinterpret_cast<const float4*>(inv_d + c0);
+                            float v[64];
+                            float m = -INFINITY;
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) {
+                                const float4 w = w4[q];
+                                v[4 * q + 0] = __uint_as_float(raw[4 * q + 0]) * w.x;
+                                v[4 * q + 1] = __uint_as_float(raw[4 * q + 1]) * w.y;
+                                v[4 * q + 2] = __uint_as_float(raw[4 * q + 2]) * w.z;
+                                v[4 * q + 3] = __uint_as_float(raw[4 * q + 3]) * w.w;
+                            }
+                            if (c0 + 64 > nd) {   // the block's last dst tokens: mask the columns behind them
+#pragma unroll
+                                for (int c = 0; c < 64; ++c)
+                                    if (c0 + c >= nd) v[c] = -INFINITY;
+                            }
+#pragma unroll
+                            for (int c = 0; c < 64; c += 2) m = tc::fmax3(m, v[c], v[c + 1]);
+                            if (m > best) {   // rare after the first tiles: find the first column holding the maximum
+                                best = m;
+                                int first = 63;
+#pragma unroll
+                                for (int c = 62; c >= 0; --c)
+                                    if (v[c] == m) first = c;
+                                arg = c0 + first;
+                            }
+                        }
+                    }
+                }
+                if (!ok) break;
+                // the two column halves of a token meet: half 1 hands (best, arg) over, half 0 decides (ties: lowest dst)
+                const int slot = i & 1;
+                if (half == 1) {
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->x_done[slot]), (n_x[slot] & 1u) ^ 1u, abort_flag);
+                    if (!ok) break;
+                    xch[slot * TILE + row] = make_float2(best, __int_as_float(arg));
+                    tc::mbar_arrive(tc::smem_addr(&bars->x_full[slot]));
+                } else {
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->x_full[slot]), n_x[slot] & 1u, abort_flag);
+                    if (!ok) break;
+                    const float2 o = xch[slot * TILE + row];
+                    tc::mbar_arrive(tc::smem_addr(&bars->x_done[slot]));
+                    const int oarg = __float_as_int(o.y);
+                    if (o.x > best || (o.x == best && oarg < arg)) {
+                        best = o.x;
+                        arg = oarg;
+                    }
+                    const int p = it.row0 + i * TILE + row;   // token number inside the block
+                    if (p < n) {
+                        const float w = __ldg(a.inv_norm[t] + head_row0 + p);
+                        a.best_key[t][head_row0 + p] = score_key(best * w);
+                        a.best_pos[t][head_row0 + p] = dst_position(arg, n, nd);
+                    }
+                }
+                ++n_x[slot];
+            }
+        }
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tc::tmem_dealloc(tmem, SC_TMEM_COLS);
+    if (tid == 0 && bars->abort_flag) atomicCAS(a.status, kDevOk, kDevTimeoutBigMatch);
+}
+
+// ------------------------------------------------------------------------------------------------ selection
+// One CTA per (tensor, head, block); thread i owns tokens 4 i .. 4 i + 3 of the block, so that counts taken in
+// thread order are counts in position order.
+constexpr int SEL_THREADS = 1024;
+
+// one warp: walking down from the largest of 256 bins, the bin in which the running count reaches `want`
+// (1 <= want <= total); *bin_out = that bin, *want_out = want minus the count of all higher bins
+__device__ __forceinline__ void pick_bin(const int* h, int want, int* bin_out, int* want_out) {
+    const int lane = threadIdx.x & 31, lo = lane * 8;
+    int c = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c += h[lo + i];
+    int incl = c;   // this lane's bins and all higher ones
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += o;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, incl >= want);
+    if (hit == 0) {   // cannot happen for want <= total; keep the result defined
+        if (lane == 0) {
+            *bin_out = 0;
+            *want_out = 1;
+        }
+        return;
+    }
+    if (lane == 31 - __clz(hit)) {
+        int above = incl - c, b = lo + 7;
+        for (; b > lo; --b) {
+            if (above + h[b] >= want) break;
+            above += h[b];
+        }
+        *bin_out = b;
+        *want_out = want - above;
+    }
+}
+
+__global__ void __launch_bounds__(SEL_THREADS, 1) big_select_kernel(const BigMatchArgs a) {
+    __shared__ int hist[256];
+    __shared__ int warp_sum[32];
+    __shared__ int s_bin, s_want;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int per_tensor = a.heads * a.n_blocks;
+    const int t = blockIdx.x / per_tensor, h = (blockIdx.x % per_tensor) / a.n_blocks, b = blockIdx.x % a.n_blocks;
+    const BlockInfo bi = a.blocks[b];
+    const int n = bi.n, r = t == 0 ? bi.r_q : bi.r_k, nd = t == 0 ? bi.nd_q : bi.nd_k;
+    const int64_t base = (int64_t)h * a.n_tokens + bi.start;
+    int32_t* A = a.assign[t] + base;
+    if (r == 0) {   // nothing merges: identity
+        for (int j = tid; j < n; j += SEL_THREADS) A[j] = bi.start + j;
+        return;
+    }
+    uint32_t key[4];
+    bool src[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        src[e] = j < n && !is_dst_position(j, n, nd);
+        key[e] = src[e] ? a.best_key[t][base + j] : 0u;
+    }
+    const int n_src = n - nd;
+    bool merged[4] = {src[0], src[1], src[2], src[3]};
+    if (r < n_src) {
+        // T = the r-th largest key: radix select, 8 bits a pass
+        uint32_t prefix = 0, mask = 0;
+        int want = r;
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool in = src[e] && (key[e] & mask) == prefix;
+                const int bin = in ? (int)((key[e] >> shift) & 255u) : -1;
+                const unsigned peers = __match_any_sync(0xffffffffu, bin);   // one atomic per distinct bin of the warp
+                if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+            }
+            __syncthreads();
+            if (warp == 0) pick_bin(hist, want, &s_bin, &s_want);
+            __syncthreads();
+            prefix |= (uint32_t)s_bin << shift;
+            mask |= 255u << shift;
+            want = s_want;
+            __syncthreads();   // s_bin, s_want and hist are rewritten in the next pass
+        }
+        // keys above T merge; of the keys equal to T the first `want` in position order (Sec. 3.2 ties: lowest position)
+        int eq = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) eq += (src[e] && key[e] == prefix) ? 1 : 0;
+        int incl = eq;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += o;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int w = warp_sum[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, w, off);
+                if (lane >= off) w += o;
+            }
+            warp_sum[lane] = w;
+        }
+        __syncthreads();
+        int before = (warp > 0 ? warp_sum[warp - 1] : 0) + incl - eq;   // equal keys at lower positions
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (src[e] && key[e] == prefix) {
+                merged[e] = before < want;
+                ++before;
+            } else {
+                merged[e] = src[e] && key[e] > prefix;
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        if (j < n) {
+            int target = j;
+            if (merged[e]) {
+                target = a.best_pos[t][base + j];
+                if (target < 0 || target >= n) {   // cannot happen after the score kernel; never write a bad index
+                    atomicCAS(a.status, kDevOk, kDevBadIndex);
+                    target = j;
+                }
+            }
+            A[j] = bi.start + target;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ merging
+// One CTA per (map in {Q, K}, head, block) - the K map also merges V - plus CTAs that copy the special tokens.
+constexpr int MG_THREADS = 1024;
+constexpr int MG_SMEM = kMaxBigBlockTokens * 4 /*keys*/ + kMaxBigBlockTokens * 2 /*row of kept token*/ + (kMaxBigBlockTokens + 4) * 4 /*segments*/ + 256;
+
+__device__ __forceinline__ void unpack8f(const uint4& raw, float* f) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArgs a, int sp_chunks) {
+    extern __shared__ __align__(16) unsigned char mg_smem[];
+    uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);                                     // [P] (merged row << 12) | position
+    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + kMaxBigBlockTokens * 4);            // [n] merged row of a kept token, -1
+    int* seg = reinterpret_cast<int*>(mg_smem + kMaxBigBlockTokens * 6);                       // [n_kept + 1] first sorted index of every merged row
+    int* warp_sum = seg + kMaxBigBlockTokens + 4;                                              // [32]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_block_ctas = 2 * a.heads * a.n_blocks;
+    const int ch = lane & 7, sub = lane >> 3;   // 16-byte chunk of a row; which of four rows in flight
+
+    if ((int)blockIdx.x >= n_block_ctas) {
+        // special tokens: never merged, first in the merged order; 128 rows of one head per CTA, all three tensors
+        const int idx = blockIdx.x - n_block_ctas, h = idx / sp_chunks, row = (idx % sp_chunks) * 128 + (tid >> 3);
+        if (row < a.n_special_total) {
+            for (int t = 0; t < 3; ++t) {
+                const int m_len = t == 0 ? a.m_q : a.m_k;
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(a.xr[t] + ((int64_t)h * a.n_tokens + row) * kHeadDim) + (tid & 7));
+                reinterpret_cast<uint4*>(a.merged[t] + ((int64_t)h * m_len + row) * kHeadDim)[tid & 7] = v;
+            }
+        }
+        return;
+    }
+    const int per_map = a.heads * a.n_blocks;
+    const int m = blockIdx.x / per_map, h = (blockIdx.x % per_map) / a.n_blocks, b = blockIdx.x % a.n_blocks;
+    const BlockInfo bi = a.blocks[b];
+    const int n = bi.n, r = m == 0 ? bi.r_q : bi.r_k, moff = m == 0 ? bi.moff_q : bi.moff_k, m_len = m == 0 ? a.m_q : a.m_k;
+    const int n_kept = n - r;
+    const int64_t base = (int64_t)h * a.n_tokens + bi.start;
+    const int32_t* A = a.assign[m] + base;
+
+    // merged row of every kept token = its rank among the kept tokens, in position order
+    int rep[4];
+    int kept = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        rep[e] = -1;
+        if (j < n) {
+            rep[e] = A[j] - bi.start;
+            if (rep[e] < 0 || rep[e] >= n) {   // corrupt map: record, treat as kept
+                atomicCAS(a.status, kDevOk, kDevBadIndex);
+                rep[e] = j;
+            }
+            kept += rep[e] == j ? 1 : 0;
+        }
+    }
+    int incl = kept;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_sum[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, w, off);
+            if (lane >= off) w += o;
+        }
+        warp_sum[lane] = w;
+    }
+    __syncthreads();
+    int next_row = (warp > 0 ? warp_sum[warp - 1] : 0) + incl - kept;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        if (j < n) row_of[j] = rep[e] == j ? (int16_t)next_row++ : (int16_t)-1;
+    }
+    __syncthreads();
+    // sort the tokens by (merged row, position): the members of every row become one ascending run
+    int P = 512;
+    while (P < n) P <<= 1;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        uint32_t key = 0xffffffffu;
+        if (j < n) {
+            int row = row_of[rep[e]];
+            if (row < 0 || row >= n_kept) {   // target is not a kept token, or more kept tokens than the budget allows: corrupt map
+                atomicCAS(a.status, kDevOk, kDevBadIndex);
+                row = 0xfffff;                // sorts behind every valid row, is never gathered
+            } else if (m == 0) {
+                a.rank_q[base + j] = moff + row;
+            }
+            key = ((uint32_t)row << 12) | (uint32_t)j;
+        }
+        if (j < P) keys[j] = key;
+    }
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int jj = k >> 1; jj > 0; jj >>= 1) {
+            for (int i = tid; i < P; i += MG_THREADS) {
+                const int ixj = i ^ jj;
+                if (ixj > i) {
+                    const uint32_t x = keys[i], y = keys[ixj];
+                    if ((x > y) == ((i & k) == 0)) {
+                        keys[i] = y;
+                        keys[ixj] = x;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = tid; i <= n; i += MG_THREADS) {
+        const int row = i < n ? (int)(keys[i] >> 12) : n_kept;
+        const int prev = i > 0 ? (int)(keys[i - 1] >> 12) : -1;
+        if (row != prev && prev < n_kept)   // every row from prev + 1 to row starts here (rows without members cannot occur in a valid map)
+            for (int q = prev + 1; q <= min(row, n_kept); ++q) seg[q] = i;
+    }
+    __syncthreads();
+    // one warp per merged row: four members in flight (lanes 8 s .. 8 s + 7 read member s, s + 4, ...), fp32 sums,
+    // combined in a fixed order: the result does not depend on scheduling
+    for (int t = (m == 0 ? 0 : 1); t <= (m == 0 ? 0 : 2); ++t) {
+        const __nv_bfloat16* x = a.xr[t] + base * kHeadDim;
+        __nv_bfloat16* out = a.merged[t] + ((int64_t)h * m_len + moff) * kHeadDim;
+        for (int row = warp; row < n_kept; row += MG_THREADS / 32) {
+            const int i0 = seg[row], i1 = seg[row + 1];
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int i = i0 + sub; i < i1; i += 4) {
+                const int pos = (int)(keys[i] & 4095u);
+                float f[8];
+                unpack8f(__ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * kHeadDim) + ch), f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] += f[e];
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 8);
+                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+            }
+            if (sub == 0 && i1 > i0) {
+                const float inv = 1.0f / (float)(i1 - i0);
+                uint4 o;
+                o.x = pack2(acc[0] * inv, acc[1] * inv);
+                o.y = pack2(acc[2] * inv, acc[3] * inv);
+                o.z = pack2(acc[4] * inv, acc[5] * inv);
+                o.w = pack2(acc[6] * inv, acc[7] * inv);
+                reinterpret_cast<uint4*>(out + (int64_t)row * kHeadDim)[ch] = o;
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t configure_big_blocks() {
+    cudaError_t e = cudaFuncSetAttribute(big_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(big_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM);
+}
+
+cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t stream) {
+    CUtensorMap mq, mk;
+    if (!encode_rows_tensor_map(&mq, a.xr[0], a.n_tokens, a.heads, kHeadDim, (int64_t)a.n_tokens * kHeadDim, TILE) ||
+        !encode_rows_tensor_map(&mk, a.xr[1], a.n_tokens, a.heads, kHeadDim, (int64_t)a.n_tokens * kHeadDim, TILE))
+        return cudaErrorInvalidValue;
+    const int64_t total = 2ll * a.heads * a.n_items;
+    int ctas = sm_count < 1 ? 1 : sm_count;
+    if (ctas > total) ctas = (int)total;
+    if (ctas < 1) ctas = 1;
+    big_scores_kernel<<<ctas, SC_THREADS, SC_SMEM, stream>>>(mq, mk, a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_big_select(const BigMatchArgs& a, cudaStream_t stream) {
+    big_select_kernel<<<2 * a.heads * a.n_blocks, SEL_THREADS, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_big_merge(const MergeArgs& a, cudaStream_t stream) {
+    const int sp_chunks = (a.n_special_total + 127) / 128;
+    big_merge_kernel<<<2 * a.heads * a.n_blocks + a.heads * sp_chunks, MG_THREADS, MG_SMEM, stream>>>(a, sp_chunks);
+    return cudaGetLastError();
+}
+
+}  // namespace httm

@@ -9,14 +9,18 @@ namespace httm {
 
 constexpr int kHeadDim = 64;          // channels per head the kernels are written for
 constexpr int kRowBytes = kHeadDim * 2;  // one token of one head, bf16
-constexpr int kMaxBlockTokens = 256;  // largest merging block the match / merge kernels stage
+constexpr int kMaxBlockTokens = 256;  // largest merging block the warp-per-block match / merge kernels stage
+constexpr int kMaxBigBlockTokens = 4096;   // largest merging block of the large-block path (Sec. 4.1: 128 tokens x 30 frames = 3840)
+constexpr int kMaxBigDst = 1024;           // its dst tokens (a quarter of the block) stay in shared memory
+constexpr int kBigSliceRows = 1024;        // rows of a block one work item of the score kernel handles
 
 // Device status word values (first error wins).
 enum : int {
     kDevOk = 0,
     kDevTimeoutMatchLoad = 1,   // match kernel: bulk copy of a block did not complete in time
     kDevTimeoutAttention = 2,   // attention kernel: a pipeline barrier did not complete in time
-    kDevBadIndex = 3            // an index read from a map was out of range (skipped)
+    kDevBadIndex = 3,           // an index read from a map was out of range (skipped)
+    kDevTimeoutBigMatch = 4     // large-block score kernel: a pipeline barrier did not complete in time
 };
 
 // One merging block (Sec. 3.3): tokens [start, start + n) of the reordered sequence.
@@ -52,6 +56,23 @@ struct ReorderArgs {
     __nv_bfloat16* dst[3];   // [H][N][64] contiguous
     const int32_t* pi;       // [N]
     int32_t n_tokens, heads;
+    float* inv_norm[2];      // optional, [H][N] each: 1 / max(|x|, 1e-12) of the reordered Q and K tokens (large-block path)
+};
+
+// Large-block path (blocks of 257 .. 4096 tokens; Sec. 4.1's 128 x 30 regime): matching as a dense contraction.
+struct BigItem {
+    int32_t block, row0;     // rows [row0, row0 + kBigSliceRows) of this block
+};
+struct BigMatchArgs {
+    const __nv_bfloat16* xr[2];   // reordered Q, K [H][N][64]
+    const float* inv_norm[2];     // [H][N]
+    uint32_t* best_key[2];        // [H][N] order-preserving key of every token's best cosine to a dst token
+    int32_t* best_pos[2];         // [H][N] token number, inside the block, of that dst
+    int32_t* assign[2];           // [H][N] out (select kernel)
+    const BlockInfo* blocks;
+    const BigItem* items;         // the slices of all blocks (the same list for every tensor and head)
+    int32_t n_items, n_blocks, n_tokens, heads;
+    int32_t* status;
 };
 
 struct MatchArgs {
@@ -143,6 +164,10 @@ cudaError_t launch_unmerge(const UnmergeArgs& a, cudaStream_t stream);
 cudaError_t launch_deviation(const OutlierArgs& a, int sm_count, cudaStream_t stream);
 cudaError_t launch_threshold(const OutlierArgs& a, int sm_count, cudaStream_t stream);
 cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream);   // map rewrite + per-head offsets (two kernels)
+cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 contraction + row argmax
+cudaError_t launch_big_select(const BigMatchArgs& a, cudaStream_t stream);                  // top-r per (tensor, head, block)
+cudaError_t launch_big_merge(const MergeArgs& a, cudaStream_t stream);                      // sort by merged row + gather means
+cudaError_t configure_big_blocks();
 cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 / TMEM kernel
 cudaError_t configure_attention();
 cudaError_t configure_kernels();   // one-time function attributes (dynamic shared memory sizes)

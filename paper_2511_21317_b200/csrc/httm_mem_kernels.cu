@@ -72,6 +72,7 @@ constexpr int kReorderThreads = 256;
 constexpr int kReorderUnroll = 4;
 constexpr int kReorderTokensPerCta = (kReorderThreads / 8) * kReorderUnroll;
 
+template <bool NORMS>   // NORMS: also write 1 / max(|x|, 1e-12) of every Q and K token (the large-block matcher needs them)
 __global__ void __launch_bounds__(kReorderThreads) reorder_kernel(const __grid_constant__ ReorderArgs a) {
     const int t = blockIdx.z, h = blockIdx.y;
     const int chunk = threadIdx.x & 7, slot = threadIdx.x >> 3;
@@ -83,18 +84,33 @@ __global__ void __launch_bounds__(kReorderThreads) reorder_kernel(const __grid_c
 #pragma unroll
     for (int u = 0; u < kReorderUnroll; ++u) {
         const int p = base + u * (kReorderThreads / 8) + slot;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
         if (p < a.n_tokens) v[u] = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)__ldg(a.pi + p) * st));
     }
 #pragma unroll
     for (int u = 0; u < kReorderUnroll; ++u) {
         const int p = base + u * (kReorderThreads / 8) + slot;
         if (p < a.n_tokens) *reinterpret_cast<uint4*>(dst + (int64_t)p * kHeadDim) = v[u];
+        if (NORMS && t < 2) {   // the eight threads of a row are neighbouring lanes
+            float x[8];
+            unpack8(v[u], x);
+            float s = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s = fmaf(x[e], x[e], s);
+            s += __shfl_xor_sync(0xffffffffu, s, 1);
+            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            s += __shfl_xor_sync(0xffffffffu, s, 4);
+            if (chunk == 0 && p < a.n_tokens) a.inv_norm[t][(int64_t)h * a.n_tokens + p] = fminf(rsqrtf(s), 1e12f);
+        }
     }
 }
 
 cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream) {
     dim3 grid((a.n_tokens + kReorderTokensPerCta - 1) / kReorderTokensPerCta, a.heads, 3);
-    reorder_kernel<<<grid, kReorderThreads, 0, stream>>>(a);
+    if (a.inv_norm[0])
+        reorder_kernel<true><<<grid, kReorderThreads, 0, stream>>>(a);
+    else
+        reorder_kernel<false><<<grid, kReorderThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

@@ -51,7 +51,7 @@ def test_create_rejects_bad_configs(lib):
         return binding.HttmConfig(**base)
 
     for bad, code in ((make(frames=0), -1), (make(ratio_q=1.0), -1), (make(ratio_kv=-0.1), -1), (make(head_dim=128), -2),
-                      (make(grid_h=64, grid_w=64, blk_h=32, blk_w=32), -2), (make(blk_w=0), -1), (make(device=99), -1)):
+                      (make(grid_h=128, grid_w=128, blk_h=64, blk_w=64), -2), (make(blk_w=0), -1), (make(device=99), -1)):
         with pytest.raises(binding.HttmError) as e:
             binding.Httm(bad)
         assert e.value.code == code, (bad, e.value)
