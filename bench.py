@@ -247,8 +247,9 @@ def run_ours(args, wl):
     # ---- per-kernel durations: every kernel of the path launched on its own with events between them.
     #      Order: reorder, match, merge (the separate kernels), then - where the geometry allows it - match and
     #      merge reading their blocks straight from Q/K/V (the two that the public call uses), attention, unmerge.
-    direct = True   # every supported geometry has the direct kernels
-    order = [0, 1, 2] + ([5, 6] if direct else []) + [3, 4]
+    big = ctx.query(hb.Q_MAX_BLOCK_TOKENS) > 256   # large blocks: reorder (+ norms), scores, select, merge, attention, unmerge
+    direct = not big   # every other supported geometry has the direct kernels
+    order = [0, 8, 9, 2, 3, 4] if big else [0, 1, 2, 5, 6, 3, 4]
     stage_ms = {st: 0.0 for st in order}
     evs = [[ev() for _ in range(len(order) + 1)] for _ in range(args.steps)]
     for s_ in range(args.steps):
@@ -304,10 +305,23 @@ def run_ours(args, wl):
         }
         attn_flops = 4.0 * H * Mq * Mk * D
         alg["match_direct"], alg["merge_direct"] = alg["match"], alg["merge"]
+        alg["big_select"] = 2 * H * N * (4 + 4 + 4)   # keys and best dst read, map written
+        # the large-block score kernel is a contraction: every token of a block against the block's dst tokens
+        big_flops = 0.0
+        if big:
+            for n in np.diff(ctx.export(hb.X_BLOCK_START).astype(np.int64)):
+                for ratio in (wl.ratio_q, wl.ratio_kv):
+                    r = min(int(np.floor(ratio * n + 1e-9)), n - 1)
+                    nd = min(-(-n // 4), n - r)
+                    big_flops += 2.0 * H * n * nd * D if r > 0 else 0.0
         kernels = {}
         for st in order:
             name, ms = hb.STAGE_NAMES[st], float(stage_ms[st])
-            if name == "attention":
+            if name == "big_scores":
+                tf = big_flops / (ms * 1e-3) / 1e12
+                kernels[name] = {"ms": ms, "tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                                 "algorithmic_gflop": big_flops / 1e9}
+            elif name == "attention":
                 tf = attn_flops / (ms * 1e-3) / 1e12
                 kernels[name] = {"ms": ms, "tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
                                  "frac_of_nominal_2250": tf / 2250.0}
@@ -315,7 +329,7 @@ def run_ours(args, wl):
                 gbs = alg[name] / (ms * 1e-3) / 1e9
                 kernels[name] = {"ms": ms, "algorithmic_mb": alg[name] / 1e6, "gbs": gbs,
                                  "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0}
-        used = ([5, 6] if direct else [0, 1, 2]) + [3, 4]
+        used = [0, 8, 9, 2, 3, 4] if big else ([5, 6] if direct else [0, 1, 2]) + [3, 4]
         path = {"kernels_of_the_public_call": [hb.STAGE_NAMES[st] for st in used],
                 "sum_of_their_stage_times_ms": float(sum(stage_ms[st] for st in used))}
         attn_ms = float(stage_ms[3])
@@ -346,7 +360,7 @@ def run_ours(args, wl):
             line["cpu_baseline"] = {"value": N / sec, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
                                     "sample": info["sample"], "seconds": info["seconds"], "ms_per_layer_extrapolated": sec * 1e3}
             line["parity_sample"] = parity_sample(ctx, hb, wl, kept, out)
-        if world == 1 and args.outlier_fraction > 0:
+        if world == 1 and args.outlier_fraction > 0 and not big:
             line["outlier_filter"] = filtered_variant(args, wl, hb, dq, dk, dv, local)
         print(json.dumps(line), flush=True)
     ctx.close()

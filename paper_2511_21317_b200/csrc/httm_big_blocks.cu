@@ -535,33 +535,45 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArg
             for (int q = prev + 1; q <= min(row, n_kept); ++q) seg[q] = i;
     }
     __syncthreads();
-    // one warp per merged row: four members in flight (lanes 8 s .. 8 s + 7 read member s, s + 4, ...), fp32 sums,
-    // combined in a fixed order: the result does not depend on scheduling
+    // eight lanes per merged row (a lane owns one 16-byte chunk of the row), four rows per warp at a time, four
+    // members of a row in flight: the gather is bound by load latency, so it needs many loads in the air.  Member
+    // i of a row goes to accumulator i mod 4; the four are added in a fixed order: the result does not depend on
+    // scheduling.
     for (int t = (m == 0 ? 0 : 1); t <= (m == 0 ? 0 : 2); ++t) {
         const __nv_bfloat16* x = a.xr[t] + base * kHeadDim;
         __nv_bfloat16* out = a.merged[t] + ((int64_t)h * m_len + moff) * kHeadDim;
-        for (int row = warp; row < n_kept; row += MG_THREADS / 32) {
+        for (int row = warp * 4 + sub; row < n_kept; row += (MG_THREADS / 32) * 4) {
             const int i0 = seg[row], i1 = seg[row + 1];
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int i = i0 + sub; i < i1; i += 4) {
-                const int pos = (int)(keys[i] & 4095u);
-                float f[8];
-                unpack8f(__ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * kHeadDim) + ch), f);
+            float acc[4][8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] += f[e];
-            }
+            for (int u = 0; u < 4; ++u)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 8);
-                acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+                for (int e = 0; e < 8; ++e) acc[u][e] = 0.f;
+            for (int i = i0; i < i1; i += 4) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (i + u < i1) v[u] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)(keys[i + u] & 4095u) * kHeadDim) + ch);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    float f[8];
+                    unpack8f(v[u], f);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[u][e] += f[e];
+                }
             }
-            if (sub == 0 && i1 > i0) {
+            if (i1 > i0) {
                 const float inv = 1.0f / (float)(i1 - i0);
+                float r8[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) r8[e] = ((acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e])) * inv;
                 uint4 o;
-                o.x = pack2(acc[0] * inv, acc[1] * inv);
-                o.y = pack2(acc[2] * inv, acc[3] * inv);
-                o.z = pack2(acc[4] * inv, acc[5] * inv);
-                o.w = pack2(acc[6] * inv, acc[7] * inv);
+                o.x = pack2(r8[0], r8[1]);
+                o.y = pack2(r8[2], r8[3]);
+                o.z = pack2(r8[4], r8[5]);
+                o.w = pack2(r8[6], r8[7]);
                 reinterpret_cast<uint4*>(out + (int64_t)row * kHeadDim)[ch] = o;
             }
         }
