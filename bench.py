@@ -29,7 +29,7 @@ from paper_2511_21317_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (ncu, profiles/ncu_full_medium_five_kernels.txt);
 # None for workloads that were not captured, and to be reset to None whenever the attention kernel changes.
-ATTENTION_DRAM_TRAFFIC = {"medium": 64751360 + 6856448}
+ATTENTION_DRAM_TRAFFIC = {"medium": 64933120 + 5256960}
 METRIC = "httm_global_attention_layer_throughput"
 UNIT = "tokens/s"
 

@@ -24,7 +24,8 @@ def main() -> int:
     ap.add_argument("--calls", type=int, default=2, help="httm_global_attention calls")
     ap.add_argument("--dense", type=int, default=0, help="httm_dense_attention calls")
     ap.add_argument("--stages", type=int, default=0, help="rounds of every kernel launched on its own (reorder, match, merge, "
-                    "match and merge with direct block loads where supported, attention, unmerge)")
+                    "match and merge with direct block loads, attention, unmerge; for large blocks reorder, scores, select, "
+                    "merge, attention, unmerge)")
     ap.add_argument("--heads", type=int, default=None, help="override the number of heads")
     ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
     ap.add_argument("--block", default=None, help="override the block shape, e.g. 4x4x4")
@@ -50,10 +51,10 @@ def main() -> int:
             ctx.global_attention(dq, dk, dv, out)
         for _ in range(args.dense):
             ctx.dense_attention(dq, dk, dv, out)
-        direct = True   # every supported geometry has the direct kernels
         ctx.set_outlier_fraction(0.0)
+        big = ctx.query(hb.Q_MAX_BLOCK_TOKENS) > 256   # large blocks: reorder (+ norms), scores, select, merge, attention, unmerge
         for _ in range(args.stages):
-            for st in [0, 1, 2] + ([5, 6] if direct else []) + [3, 4]:
+            for st in ([0, 8, 9, 2, 3, 4] if big else [0, 1, 2, 5, 6, 3, 4]):
                 ctx.launch_stage(st, dq, dk, dv, out)
         torch.cuda.synchronize()
         status = ctx.query(hb.Q_DEVICE_STATUS)
