@@ -167,7 +167,9 @@ struct TaskCursor {
 //     Token j of a block is owned, for the selection, by lane (j & 7) * 4 + ((j >> 3) & 1),
 //     slot j >> 4: the lane where the MMA accumulator layout leaves row j's results.
 // ------------------------------------------------------------------------------------
-__host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 64 ? 8 : (nmax <= 128 ? 4 : 2); }
+// warps per CTA (one CTA per SM): as many as the shared memory takes at two stages per warp; a warp works alone on its
+// blocks, so the number of warps per scheduler is what hides its instruction latencies
+__host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 32 ? 8 : (nmax <= 64 ? 12 : (nmax <= 128 ? 6 : 3)); }
 __host__ __device__ constexpr int match_aux_bytes(int nmax) { return nmax * 4 + 16; }   // inverse norms + 2 mbarriers
 __host__ __device__ constexpr int match_smem_bytes(int nmax) {
     return match_warps_per_cta(nmax) * (2 * nmax * kRowBytes + match_aux_bytes(nmax)) + 1024 /*alignment slack*/;
@@ -865,7 +867,7 @@ static cudaError_t launch_merge_tc(const MergeArgs& a, int sm_count, cudaStream_
 //     (row tile, token step) with ldmatrix.trans from the swizzled TMA stage (blocks come from the
 //     reordered copies).  Group sizes are counted with shared-memory atomics.
 // ------------------------------------------------------------------------------------
-__host__ __device__ constexpr int merge_multi_warps(int nmax) { return nmax <= 64 ? 8 : (nmax <= 128 ? 4 : 2); }
+__host__ __device__ constexpr int merge_multi_warps(int nmax) { return nmax <= 64 ? 12 : (nmax <= 128 ? 6 : 3); }   // as for the match kernel
 __host__ __device__ constexpr int merge_multi_aux(int nmax) { return nmax * 8 + 16; }   // counts, reciprocals, 2 mbarriers
 __host__ __device__ constexpr int merge_multi_smem(int nmax) {
     return merge_multi_warps(nmax) * (2 * nmax * kRowBytes + merge_multi_aux(nmax)) + 1024 /*alignment slack*/;

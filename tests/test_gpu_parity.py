@@ -196,7 +196,7 @@ def test_argument_errors_are_reported_before_any_launch():
         assert call(t(good[0]), t(good[1]), t(good[2]), T(good[0].data_ptr(), D, H * D)) == hb.ERR_INVALID_ARG   # aliasing
         assert ctx._lib.httm_dense_attention(ctx._h, t(good[0]), t(good[1]), T(None, 0, 0), o, ctx._stream(None)) == hb.ERR_INVALID_ARG
         assert b"null" in ctx._lib.httm_last_error(ctx._h)
-        assert ctx._lib.httm_launch_stage(ctx._h, 9, t(good[0]), t(good[1]), t(good[2]), o, ctx._stream(None)) == hb.ERR_INVALID_ARG
+        assert ctx._lib.httm_launch_stage(ctx._h, 99, t(good[0]), t(good[1]), t(good[2]), o, ctx._stream(None)) == hb.ERR_INVALID_ARG
         buf = np.empty(3, dtype=np.int32)
         assert ctx._lib.httm_export(ctx._h, hb.X_PI, buf.ctypes.data, buf.nbytes, None) == hb.ERR_INVALID_ARG
         assert ctx.launch_count() == n0
