@@ -1,0 +1,110 @@
+"""Pins of the first-frame-anchoring oracle against what the paper's description and the mathematics fix."""
+import numpy as np
+import pytest
+
+from oracle import httm_anchor as anc
+from oracle import httm_oracle as orc
+from paper_2511_21317_b200 import synth
+
+
+def case(seed=0, S=5, h=5, w=6, blk=(4, 2, 4), heads=2, nsp=(1, 1)):
+    wl = synth.Workload("a", S, h, w, blk[0], blk[1], blk[2], 0.7, 0.6, heads=heads, n_camera=nsp[0], n_register=nsp[1], seed=seed, sigma=0.5)
+    return wl, orc.Geometry.of(wl), synth.make_qkv(wl)
+
+
+def frame_of_position(g, pi):
+    return pi // (g.n_special + g.grid_h * g.grid_w)
+
+
+def test_first_frame_tokens_are_kept_and_collect_the_merges_of_their_blocks():
+    wl, g, (q, k, v) = case()
+    res = anc.global_attention(g, 0.7, 0.6, q, k, v, attend=False)
+    frame = frame_of_position(g, res.pi)
+    idx = np.arange(res.pi.size)
+    first_group = np.zeros(res.pi.size, dtype=bool)
+    for b, n, n0 in anc.anchored_blocks(g, res.blk_start):
+        first_group[res.blk_start[b]:res.blk_start[b + 1]] = True
+    for A in (res.assign_q, res.assign_k):
+        for hd in range(g.heads):
+            assert (A[hd][frame == 0] == idx[frame == 0]).all()                    # the reference frame stays intact
+            merged = (A[hd] != idx) & first_group
+            assert merged.any() and (frame[A[hd][merged]] == 0).all()               # merges of these blocks go into frame 0
+            assert (frame[idx[merged]] > 0).all()
+
+
+def test_map_against_plain_loops():
+    wl, g, (q, k, v) = case(seed=3, heads=1)
+    pi, bs = orc.temporal_reorder(g)
+    xr = orc.reorder(g, pi, q)
+    x = orc.bf16_to_double(xr)[0]
+    for rho in (0.3, 0.7, 0.95):
+        A, _, _ = anc.match(g, bs, rho, xr)
+        plain = orc.match(g, bs, rho, xr, margins=False)
+        first = {b: (n, n0) for b, n, n0 in anc.anchored_blocks(g, bs)}
+        for b in range(len(bs) - 1):
+            base, n = int(bs[b]), int(bs[b + 1] - bs[b])
+            if b not in first:
+                assert np.array_equal(A[0, base:base + n], plain[0, base:base + n])   # later frame groups: unchanged
+                continue
+            n0 = first[b][1]
+            r = min(int(np.floor(rho * n + 1e-9)), n - n0)
+            nrm = [max(float(np.sqrt((x[base + j] ** 2).sum())), 1e-12) for j in range(n)]
+            cand = []
+            for a in range(n0, n):
+                sims = [float(x[base + a] @ x[base + d]) / (nrm[a] * nrm[d]) for d in range(n0)]
+                d = max(range(n0), key=lambda t: (sims[t], -t))
+                cand.append((-sims[d], a, d))
+            cand.sort()
+            expect = np.arange(n)
+            for _, a, d in cand[:r]:
+                expect[a] = d
+            assert np.array_equal(A[0, base:base + n] - base, expect)
+
+
+def test_budget_and_closed_form_length():
+    wl, g, (q, k, v) = case(seed=5)
+    for rho in (0.0, 0.5, 0.7, 0.99):
+        res = anc.global_attention(g, rho, rho, q, k, v, attend=False)
+        assert res.M_q == anc.merged_len(g, rho) == res.M_k
+        idx = np.arange(res.pi.size)
+        for b, n, n0 in anc.anchored_blocks(g, res.blk_start):
+            lo, hi = int(res.blk_start[b]), int(res.blk_start[b + 1])
+            r = min(int(np.floor(rho * n + 1e-9)), n - n0)
+            for hd in range(g.heads):
+                assert int((res.assign_q[hd, lo:hi] != idx[lo:hi]).sum()) == r
+    # more src than the plain rule would merge can go: at 0.99 every later-frame token of the first group is merged
+    res = anc.global_attention(g, 0.99, 0.99, q, k, v, attend=False)
+    for b, n, n0 in anc.anchored_blocks(g, res.blk_start):
+        lo = int(res.blk_start[b])
+        assert (res.assign_q[:, lo + n0:lo + n] < lo + n0).all()
+
+
+def test_blocks_inside_the_first_frame_merge_nothing_and_ratio_zero_is_dense_attention():
+    wl, g, (q, k, v) = case(seed=7, S=3, blk=(1, 2, 4))
+    res = anc.global_attention(g, 0.7, 0.7, q, k, v, attend=False)
+    idx = np.arange(res.pi.size)
+    for b, n, n0 in anc.anchored_blocks(g, res.blk_start):
+        assert n0 == n
+        lo, hi = int(res.blk_start[b]), int(res.blk_start[b + 1])
+        assert (res.assign_q[:, lo:hi] == idx[lo:hi]).all()
+    wl, g, (q, k, v) = case(seed=8)
+    out = anc.global_attention(g, 0.0, 0.0, q, k, v).out
+    assert np.allclose(out, orc.dense_attention(g, q, k, v), rtol=1e-9, atol=1e-12)
+
+
+def test_margins_follow_the_plain_convention():
+    wl, g, (q, k, v) = case(seed=9, heads=1)
+    pi, bs = orc.temporal_reorder(g)
+    xr = orc.reorder(g, pi, q)
+    A, mb, ms = anc.match(g, bs, 0.5, xr)
+    x = orc.bf16_to_double(xr)[0]
+    b, n, n0 = anc.anchored_blocks(g, bs)[0]
+    base = int(bs[b])
+    blk = x[base:base + n]
+    xn = blk / np.maximum(np.linalg.norm(blk, axis=1, keepdims=True), 1e-12)
+    sim = xn[n0:] @ xn[:n0].T
+    srt = np.sort(sim, axis=1)
+    assert np.allclose(mb[0, base + n0:base + n], srt[:, -1] - srt[:, -2])
+    best = np.sort(sim.max(axis=1))[::-1]
+    r = min(int(np.floor(0.5 * n + 1e-9)), n - n0)
+    assert ms[0, b] == pytest.approx(best[r - 1] - best[r])
