@@ -57,6 +57,14 @@ typedef struct {
                                      blocks are clipped at the grid / sequence end     */
     double ratio_q, ratio_kv;     /* fraction of tokens merged away, in [0, 1)         */
     int32_t device;               /* CUDA device ordinal                               */
+    int32_t anchor_first_frame;   /* 0, or 1: first-frame anchoring (the paper's appendix on error mitigation): in every
+                                     merging block that contains frame 0 the dst tokens are exactly the block's tokens of
+                                     frame 0 and every other token of the block is a src token, so the reference frame is
+                                     never merged away and similar tokens of later frames merge INTO it; there the budget
+                                     is r = min(floor(ratio*n + 1e-9), n - n0) with n0 the block's tokens of frame 0.
+                                     UNSUPPORTED where n0 exceeds what the match kernels hold (a quarter of the largest
+                                     block: blocks of up to 256 tokens need at least 4 frames per block) and in
+                                     httm_global_attention_static.  (The field takes the struct's former padding.)  */
 } httm_config;
 
 typedef struct {

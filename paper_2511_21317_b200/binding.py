@@ -46,7 +46,7 @@ class HttmError(RuntimeError):
 class _Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("frames", "n_camera", "n_register", "grid_h", "grid_w", "heads", "head_dim",
                                                "blk_frames", "blk_h", "blk_w")] + [
-        ("ratio_q", ctypes.c_double), ("ratio_kv", ctypes.c_double), ("device", ctypes.c_int32)]
+        ("ratio_q", ctypes.c_double), ("ratio_kv", ctypes.c_double), ("device", ctypes.c_int32), ("anchor_first_frame", ctypes.c_int32)]
 
 
 class _Tensor(ctypes.Structure):
@@ -103,13 +103,15 @@ class HttmConfig:
     heads: int = 16
     head_dim: int = 64
     device: int = 0
+    anchor_first_frame: int = 0   # 1: the tokens of frame 0 are the dst tokens of their blocks (first-frame anchoring)
 
     @staticmethod
     def of(obj, device: int = 0) -> "HttmConfig":
         """Build from any record with the same attribute names (e.g. a synthetic workload)."""
         names = ("frames", "grid_h", "grid_w", "blk_frames", "blk_h", "blk_w", "ratio_q", "ratio_kv", "n_camera",
                  "n_register", "heads", "head_dim")
-        return HttmConfig(**{n: getattr(obj, n) for n in names}, device=device)
+        return HttmConfig(**{n: getattr(obj, n) for n in names}, device=device,
+                          anchor_first_frame=int(getattr(obj, "anchor_first_frame", 0)))
 
 
 def _null_tensor() -> _Tensor:
@@ -123,7 +125,8 @@ class Httm:
         self._lib = load_library()
         self.cfg = cfg
         c = _Config(cfg.frames, cfg.n_camera, cfg.n_register, cfg.grid_h, cfg.grid_w, cfg.heads, cfg.head_dim,
-                    cfg.blk_frames, cfg.blk_h, cfg.blk_w, float(cfg.ratio_q), float(cfg.ratio_kv), cfg.device)
+                    cfg.blk_frames, cfg.blk_h, cfg.blk_w, float(cfg.ratio_q), float(cfg.ratio_kv), cfg.device,
+                    int(cfg.anchor_first_frame))
         h = ctypes.c_void_p()
         rc = self._lib.httm_create(ctypes.byref(c), ctypes.byref(h))
         if rc != OK:
@@ -282,7 +285,7 @@ def global_attention_static(cfg: HttmConfig, q, k, v, out, stream=None):
         raise HttmError(ERR_INVALID_ARG, "out: expected CUDA bfloat16 [tokens][heads*head_dim]")
     o = out.view(N, H, D)
     c = _Config(cfg.frames, cfg.n_camera, cfg.n_register, cfg.grid_h, cfg.grid_w, H, D, cfg.blk_frames, cfg.blk_h,
-                cfg.blk_w, float(cfg.ratio_q), float(cfg.ratio_kv), cfg.device)
+                cfg.blk_w, float(cfg.ratio_q), float(cfg.ratio_kv), cfg.device, int(cfg.anchor_first_frame))
     if stream is None:
         stream = torch.cuda.current_stream(cfg.device)
     rc = lib.httm_global_attention_static(

@@ -433,6 +433,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
         return bad(HTTM_ERR_INVALID_ARG, "sizes must be positive (special-token counts non-negative)");
     if (!(cfg->ratio_q >= 0.0 && cfg->ratio_q < 1.0) || !(cfg->ratio_kv >= 0.0 && cfg->ratio_kv < 1.0))
         return bad(HTTM_ERR_INVALID_ARG, "merge ratios must lie in [0, 1)");
+    if (cfg->anchor_first_frame != 0 && cfg->anchor_first_frame != 1) return bad(HTTM_ERR_INVALID_ARG, "anchor_first_frame must be 0 or 1");
     if (cfg->head_dim != kHeadDim) return bad(HTTM_ERR_UNSUPPORTED, "head_dim must be 64");
     if (cfg->heads > 65535) return bad(HTTM_ERR_UNSUPPORTED, "at most 65535 heads");
     const int64_t per_frame = (int64_t)cfg->n_camera + cfg->n_register + (int64_t)cfg->grid_h * cfg->grid_w;
@@ -464,6 +465,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
     for (int s = 0; s < S; ++s)
         for (int j = 0; j < nsp; ++j) c->pi[pos++] = s * P + j;
     int32_t moff_q = pos, moff_k = pos;
+    int anchored_nd_max = 0;
     for (int g0 = 0; g0 < S; g0 += cfg->blk_frames) {
         const int f = std::min(cfg->blk_frames, S - g0);
         for (int y0 = 0; y0 < h; y0 += cfg->blk_h) {
@@ -473,8 +475,17 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
                 BlockInfo bi{};
                 bi.start = pos;
                 bi.n = f * hh * ww;
+                bi.n_rule = bi.n;
                 block_budget(bi.n, cfg->ratio_q, &bi.r_q, &bi.nd_q);
                 block_budget(bi.n, cfg->ratio_kv, &bi.r_k, &bi.nd_k);
+                if (cfg->anchor_first_frame && g0 == 0) {   // the block's tokens of frame 0 are its dst tokens, all others src
+                    const int n0 = hh * ww;
+                    bi.n_rule = n0;
+                    bi.nd_q = bi.nd_k = n0;
+                    bi.r_q = std::min<int64_t>((int64_t)std::floor(cfg->ratio_q * (double)bi.n + 1e-9), bi.n - n0);
+                    bi.r_k = std::min<int64_t>((int64_t)std::floor(cfg->ratio_kv * (double)bi.n + 1e-9), bi.n - n0);
+                    anchored_nd_max = std::max(anchored_nd_max, n0);
+                }
                 bi.moff_q = moff_q;
                 bi.moff_k = moff_k;
                 moff_q += bi.n - bi.r_q;
@@ -492,6 +503,13 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
     }
     c->blk_start.push_back(pos);
     c->n_blocks = (int32_t)c->blocks.size();
+    {   // the match kernels hold a quarter of their largest block as dst tokens (the large-block path 1024)
+        const int cap = c->max_block > kMaxBlockTokens ? kMaxBigDst : (c->max_block <= 32 ? 8 : (c->max_block <= 64 ? 16 : (c->max_block <= 128 ? 32 : 64)));
+        if (anchored_nd_max > cap) {
+            delete c;
+            return bad(HTTM_ERR_UNSUPPORTED, "first-frame anchoring: a block's tokens of frame 0 exceed a quarter of the largest block (use more frames per block)");
+        }
+    }
     c->m_q = moff_q;
     c->m_k = moff_k;
     for (int32_t p = 0; p < c->n_tokens; ++p) c->pi_inv[c->pi[p]] = p;

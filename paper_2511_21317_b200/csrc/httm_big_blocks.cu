@@ -22,10 +22,13 @@ __device__ __forceinline__ uint32_t score_key(float s) {   // unsigned keys orde
     const uint32_t b = __float_as_uint(s);
     return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
 }
-// token number (inside a block of n tokens) of dst d of n_dst evenly spaced dst tokens: the positions j with
-// floor((j + 1) n_dst / n) > floor(j n_dst / n), i.e. j = ceil((d + 1) n / n_dst) - 1
-__device__ __forceinline__ int dst_position(int d, int n, int nd) { return ((d + 1) * n + nd - 1) / nd - 1; }
-__device__ __forceinline__ bool is_dst_position(int j, int n, int nd) { return ((j + 1) * nd) / n > (j * nd) / n; }
+// token number (inside its block) of dst d of n_dst dst tokens: the positions j < n_rule with
+// floor((j + 1) n_dst / n_rule) > floor(j n_dst / n_rule), i.e. j = ceil((d + 1) n_rule / n_dst) - 1.  n_rule is the
+// block length (evenly spaced dst tokens) or n_dst (the first n_dst tokens: first-frame anchoring), see BlockInfo.
+__device__ __forceinline__ int dst_position(int d, int n_rule, int nd) { return ((d + 1) * n_rule + nd - 1) / nd - 1; }
+__device__ __forceinline__ bool is_dst_position(int j, int n_rule, int nd) {
+    return j < n_rule && ((j + 1) * nd) / n_rule > (j * nd) / n_rule;
+}
 
 // ------------------------------------------------------------------------------------------------ scores
 constexpr int TILE = 128;                        // rows of an operand tile
@@ -109,7 +112,7 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);   // rows past the last dst token: zeros (their scores are masked)
                 float w = 0.f;
                 if (d < nd) {
-                    const int pos = dst_position(d, n, nd);
+                    const int pos = dst_position(d, bi.n_rule, nd);
                     v = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * kHeadDim) + chunk);
                     w = __ldg(inv + pos);
                 }
@@ -257,7 +260,7 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (p < n) {
                         const float w = __ldg(a.inv_norm[t] + head_row0 + p);
                         a.best_key[t][head_row0 + p] = score_key(best * w);
-                        a.best_pos[t][head_row0 + p] = dst_position(arg, n, nd);
+                        a.best_pos[t][head_row0 + p] = dst_position(arg, bi.n_rule, nd);
                     }
                 }
                 ++n_x[slot];
@@ -327,7 +330,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) big_select_kernel(const BigMat
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int j = 4 * tid + e;
-        src[e] = j < n && !is_dst_position(j, n, nd);
+        src[e] = j < n && !is_dst_position(j, bi.n_rule, nd);
         key[e] = src[e] ? a.best_key[t][base + j] : 0u;
     }
     const int n_src = n - nd;

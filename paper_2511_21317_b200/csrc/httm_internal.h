@@ -31,6 +31,10 @@ struct BlockInfo {
     int32_t start, n;
     int32_t r_q, nd_q, moff_q;
     int32_t r_k, nd_k, moff_k;
+    // dst positions: j is a dst token iff j < n_rule and floor((j + 1) n_dst / n_rule) > floor(j n_dst / n_rule).
+    // n_rule = n: n_dst evenly spaced tokens (Sec. 3.2 reading); n_rule = n_dst: the first n_dst tokens of the block,
+    // i.e. its tokens of frame 0 (first-frame anchoring).
+    int32_t n_rule;
 };
 
 // Where a merging block sits in the original layout (used when the kernels read the blocks straight from

@@ -326,10 +326,11 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             continue;
         }
         // floor(x / n) and floor(x / n_dst) by multiplication: exact for the operand ranges below (n <= 256, n_dst <= 64)
-        if (n != cached_n || nd != cached_nd) {
-            cached_n = n;
+        const int n_rule = bi.n_rule;   // n (evenly spaced dst tokens) or n_dst (the first n_dst tokens: first-frame anchoring)
+        if (n_rule != cached_n || nd != cached_nd) {
+            cached_n = n_rule;
             cached_nd = nd;
-            magic_n = (1u << 23) / (uint32_t)n + 1u;
+            magic_n = (1u << 23) / (uint32_t)n_rule + 1u;
             magic_nd = (1u << 23) / (uint32_t)nd + 1u;
         }
         BlockGeom bg{};
@@ -338,8 +339,8 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             bm.set(box_f, box_h, box_w, bg.frames, bg.rows, bg.cols);
         }
         const int n_rows = DIRECT ? box_rows : n;   // rows of the stage that may hold tokens
-        auto div_n = [&](int x) { return (int)(((uint32_t)x * magic_n) >> 23); };          // x < (n + 1) * n_dst
-        auto pos_of = [&](int d) { return (int)(((uint32_t)((d + 1) * n + nd - 1) * magic_nd) >> 23) - 1; };   // position of dst d
+        auto div_n = [&](int x) { return (int)(((uint32_t)x * magic_n) >> 23); };          // floor(x / n_rule), x < (n_rule + 1) * n_dst
+        auto pos_of = [&](int d) { return (int)(((uint32_t)((d + 1) * n_rule + nd - 1) * magic_nd) >> 23) - 1; };   // position of dst d
         const uint32_t blk = stage0 + buf * STAGE_BYTES;
         // ldmatrix address of 16-byte chunk `chunk` of row `row` (chunk c of row j sits at c ^ (j & 7))
         auto chunk_addr = [&](int row, int chunk) { return blk + row * kRowBytes + ((chunk ^ (row & 7)) << 4); };
@@ -460,8 +461,9 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
                 const int j = DIRECT ? (own_t[mt] * bg.rows + own_y[mt]) * bg.cols + own_x[mt] : rho;
                 tok[mt] = valid ? j : -1;
                 if (tq < 2 && valid) {
-                    const int dj = div_n(j * nd);
-                    if (!(div_n((j + 1) * nd) > dj)) {   // not a dst position: a src token
+                    const int jr = min(j, n_rule);   // (positions from n_rule on are src tokens; the clamp keeps the operand in range)
+                    const int dj = div_n(jr * nd);
+                    if (!(j < n_rule && div_n((jr + 1) * nd) > dj)) {   // not a dst position: a src token
                         is_src[mt] = true;
                         key[mt] = score_key((own_half ? top[1] : top[0]) * invn[rho]);
                         best[mt] = pos_of(own_half ? arg[1] : arg[0]);

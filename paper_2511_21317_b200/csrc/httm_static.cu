@@ -81,6 +81,7 @@ void build_plan(const httm_config& cfg, StaticPlan* p) {
                 BlockInfo bi{};
                 bi.start = pos;
                 bi.n = f * hh * ww;
+                bi.n_rule = bi.n;
                 budget(bi.n, cfg.ratio_q, &bi.r_q, &bi.nd_q);
                 budget(bi.n, cfg.ratio_kv, &bi.r_k, &bi.nd_k);
                 bi.moff_q = mq;
@@ -142,6 +143,7 @@ extern "C" int httm_global_attention_static(const httm_config* cfg, httm_tensor 
     const int64_t bf = std::min(cfg->blk_frames, cfg->frames), bh = std::min(cfg->blk_h, cfg->grid_h),
                   bw = std::min(cfg->blk_w, cfg->grid_w);
     if (bf * bh * bw > kMaxBlockTokens) return fail(HTTM_ERR_UNSUPPORTED, "a merging block may hold at most 256 tokens");
+    if (cfg->anchor_first_frame != 0) return fail(HTTM_ERR_UNSUPPORTED, "first-frame anchoring needs a context (httm_create)");
     // size check BEFORE any plan is built: an upper bound of the scratch need (merged length <= N)
     const int64_t N64 = (int64_t)cfg->frames * ((int64_t)cfg->n_camera + cfg->n_register + (int64_t)cfg->grid_h * cfg->grid_w);
     const int64_t H = cfg->heads;

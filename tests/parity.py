@@ -23,9 +23,10 @@ def bits_to_f64(bits: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
-def check_maps(g, rho, blk_start, xr_bits, a_oracle, margin_best, margin_sel, a_gpu, what=""):
+def check_maps(g, rho, blk_start, xr_bits, a_oracle, margin_best, margin_sel, a_gpu, what="", anchored=None):
     """Returns the number of (head, block) pairs where the maps differ (all justified by the
-    margin rule); raises AssertionError otherwise."""
+    margin rule); raises AssertionError otherwise.  anchored: {block: n0} for blocks under first-frame
+    anchoring (their first n0 tokens are the dst tokens, budget min(floor(rho n), n - n0))."""
     a_gpu = np.asarray(a_gpu, dtype=np.int64)
     assert a_gpu.shape == a_oracle.shape, f"{what}: map shape {a_gpu.shape} != {a_oracle.shape}"
     diff = a_gpu != a_oracle
@@ -41,6 +42,9 @@ def check_maps(g, rho, blk_start, xr_bits, a_oracle, margin_best, margin_sel, a_
             lo, hi = int(blk_start[b]), int(blk_start[b + 1])
             n = hi - lo
             r, nd = orc.block_budget(n, rho)
+            if anchored and int(b) in anchored:
+                nd = anchored[int(b)]
+                r = min(int(np.floor(rho * n + 1e-9)), n - nd)
             ambiguous = margin_sel[hd, b] < MARGIN or (margin_best[hd, lo:hi] < MARGIN).any()
             assert ambiguous, (f"{what}: head {hd} block {b}: map differs from the oracle but all margins are >= {MARGIN} "
                                f"(min best-margin {margin_best[hd, lo:hi].min():.3e}, selection margin {margin_sel[hd, b]:.3e})")
@@ -48,7 +52,10 @@ def check_maps(g, rho, blk_start, xr_bits, a_oracle, margin_best, margin_sel, a_
             x = bits_to_f64(xr_bits[hd, lo:hi])
             nrm = np.maximum(np.linalg.norm(x, axis=1, keepdims=True), 1e-12)
             xn = x / nrm
-            dst = np.array([j for j in range(n) if ((j + 1) * nd) // n > (j * nd) // n])
+            if anchored and int(b) in anchored:
+                dst = np.arange(nd)
+            else:
+                dst = np.array([j for j in range(n) if ((j + 1) * nd) // n > (j * nd) // n])
             src = np.array([j for j in range(n) if j not in set(dst.tolist())])
             sim = xn[src] @ xn[dst].T
             best = sim.max(axis=1)
@@ -97,18 +104,24 @@ def check_output(gpu_bits: np.ndarray, expect: np.ndarray, rms: float | None = N
     return float(err.max()) / rms
 
 
-def full_check(g, rho_q, rho_kv, q, k, v, ex, out_bits, sample_tokens=None, what="", peaky=False):
+def full_check(g, rho_q, rho_kv, q, k, v, ex, out_bits, sample_tokens=None, what="", peaky=False, anchor=False):
     """Element-by-element comparison of everything the library exposes.
     ex: dict of exports (numpy) with keys pi, blk_start, qr, kr, vr, assign_q, assign_k, rank_q, q_m, k_m, v_m, o_m.
     If sample_tokens is given, attention output is checked on those ORIGINAL tokens only."""
-    res = orc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
+    anchored = None
+    if anchor:   # first-frame anchoring: its own oracle, and the block rules for the margin check
+        from oracle import httm_anchor as anc
+        res = anc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
+        anchored = {b: n0 for b, n, n0 in anc.anchored_blocks(g, res.blk_start)}
+    else:
+        res = orc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
     assert np.array_equal(ex["pi"].astype(np.int64), res.pi), f"{what}: reorder permutation differs"
     assert np.array_equal(ex["blk_start"].astype(np.int64), res.blk_start), f"{what}: block table differs"
     qr, kr, vr = orc.reorder(g, res.pi, q), orc.reorder(g, res.pi, k), orc.reorder(g, res.pi, v)
     for name, ref in (("qr", qr), ("kr", kr), ("vr", vr)):
         assert np.array_equal(ex[name], ref), f"{what}: reordered {name} is not bit-exact"
-    nq = check_maps(g, rho_q, res.blk_start, qr, res.assign_q, res.margin_best_q, res.margin_sel_q, ex["assign_q"], what + " A_q")
-    nk = check_maps(g, rho_kv, res.blk_start, kr, res.assign_k, res.margin_best_k, res.margin_sel_k, ex["assign_k"], what + " A_k")
+    nq = check_maps(g, rho_q, res.blk_start, qr, res.assign_q, res.margin_best_q, res.margin_sel_q, ex["assign_q"], what + " A_q", anchored)
+    nk = check_maps(g, rho_kv, res.blk_start, kr, res.assign_k, res.margin_best_k, res.margin_sel_k, ex["assign_k"], what + " A_k", anchored)
     if nq or nk:   # maps differ inside the margin: the oracle continues from the validated maps
         res = orc.merged_attention_from_maps(g, res.pi, q, k, v, ex["assign_q"].astype(np.int64),
                                              ex["assign_k"].astype(np.int64), attend=False)

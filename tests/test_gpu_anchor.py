@@ -1,0 +1,116 @@
+"""Parity of the CUDA path with first-frame anchoring (the paper's appendix on error mitigation: all tokens of frame 0
+are dst tokens) against its CPU oracle.  All tests here need a B200."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import httm_anchor as anc
+from oracle import httm_oracle as orc
+from paper_2511_21317_b200 import binding as hb
+from paper_2511_21317_b200 import synth
+from tests import parity
+from tests.test_gpu_parity import exports
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run_anchored(wl, q=None, k=None, v=None, sample=None, peaky=False, outlier_fraction=0.0):
+    if q is None:
+        q, k, v = synth.make_qkv(wl)
+    g = orc.Geometry.of(wl)
+    cfg = dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=1)
+    with hb.Httm(cfg) as ctx:
+        assert ctx.m_q == anc.merged_len(g, wl.ratio_q) and ctx.m_k == anc.merged_len(g, wl.ratio_kv)
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        out = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        ctx.launch_stage(hb.STAGE_REORDER, dq, dk, dv)
+        ex = exports(ctx)
+        stats = parity.full_check(g, wl.ratio_q, wl.ratio_kv, q, k, v, ex, hb.bits_from_bf16(out), sample, wl.name, peaky, anchor=True)
+        # the reference frame is intact: its tokens map to themselves in every head
+        frame = ex["pi"] // wl.tokens_per_frame
+        idx = np.arange(wl.n_tokens)
+        for A in (ex["assign_q"], ex["assign_k"]):
+            assert (A[:, frame == 0] == idx[frame == 0]).all()
+        out2 = ctx.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        assert torch.equal(out, out2)
+    return stats
+
+
+GEOMS = [
+    # name, frames, grid_h, grid_w, blk, ratio_q, ratio_kv, n_camera, n_register, heads
+    ("four_frames_4x2", 8, 8, 8, (4, 4, 2), 0.7, 0.5, 1, 4, 2),            # 32-token blocks, 8 tokens of frame 0 each
+    ("clipped", 9, 7, 9, (4, 2, 4), 0.6, 0.8, 1, 1, 2),                    # clipped in space and in the last frame group
+    ("eight_frames_thin", 8, 6, 6, (8, 2, 2), 0.9, 0.9, 0, 0, 3),           # 4 of 32 tokens are dst: most of the block merges into frame 0
+    ("blocks_64", 8, 8, 8, (4, 4, 4), 0.7, 0.7, 1, 4, 2),
+    ("blocks_128", 8, 8, 16, (4, 4, 8), 0.5, 0.75, 1, 4, 2),
+    ("blocks_256", 9, 8, 8, (4, 8, 8), 0.8, 0.4, 1, 4, 1),
+    ("ratio_zero_q", 8, 8, 8, (4, 4, 2), 0.0, 0.6, 1, 4, 2),
+    ("runs_large_blocks", 12, 1, 200, (12, 1, 64), 0.9, 0.7, 1, 4, 2),     # large-block path: 768-token blocks, 64 dst each
+]
+
+
+@pytest.mark.parametrize("case", GEOMS, ids=[c[0] for c in GEOMS])
+def test_anchored_geometries(case):
+    name, S, h, w, blk, rq, rkv, ncam, nreg, H = case
+    wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, n_camera=ncam, n_register=nreg, heads=H, seed=7)
+    run_anchored(wl, peaky=True)
+
+
+def test_anchoring_changes_only_the_first_frame_group():
+    wl = synth.Workload("cmp", 8, 8, 8, 4, 4, 2, 0.7, 0.7, heads=2)
+    q, k, v = synth.make_qkv(wl)
+    dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+    with hb.Httm(hb.HttmConfig.of(wl)) as plain, hb.Httm(dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=1)) as anchored:
+        plain.global_attention(dq, dk, dv)
+        anchored.global_attention(dq, dk, dv)
+        torch.cuda.synchronize()
+        a0, a1 = plain.export(hb.X_ASSIGN_Q), anchored.export(hb.X_ASSIGN_Q)
+        bs = plain.export(hb.X_BLOCK_START)
+        later = int(bs[len(bs) // 2])            # first block of the second frame group (two groups of equally many blocks)
+        assert np.array_equal(a0[:, later:], a1[:, later:]) and not np.array_equal(a0[:, :later], a1[:, :later])
+
+
+def test_anchor_argument_errors():
+    wl = synth.Workload("two_frames", 4, 8, 8, 2, 4, 4, 0.7, 0.7, heads=2)        # 16 of 32 tokens would be dst
+    with pytest.raises(hb.HttmError) as e:
+        hb.Httm(dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=1))
+    assert e.value.code == hb.ERR_UNSUPPORTED
+    with pytest.raises(hb.HttmError) as e:
+        hb.Httm(dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=2))
+    assert e.value.code == hb.ERR_INVALID_ARG
+    wl = synth.Workload("ok", 8, 8, 8, 4, 4, 2, 0.7, 0.7, heads=2)
+    q, k, v = synth.make_qkv(wl)
+    dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+    out = torch.empty(wl.n_tokens, wl.heads * 64, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(hb.HttmError) as e:
+        hb.global_attention_static(dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=1), dq, dk, dv, out)
+    assert e.value.code == hb.ERR_UNSUPPORTED
+
+
+def test_anchoring_with_outlier_filtering_runs_and_keeps_the_reference_frame():
+    wl = synth.Workload("anchor_filter", 8, 8, 8, 4, 4, 2, 0.7, 0.7, heads=4)
+    q, k, v = synth.make_qkv(wl)
+    with hb.Httm(dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=1)) as ctx:
+        ctx.set_outlier_fraction(0.05)
+        out = ctx.global_attention(*(hb.bf16_from_bits(x, DEV) for x in (q, k, v)))
+        torch.cuda.synchronize()
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0 and torch.isfinite(out.float()).all()
+        A = ctx.export(hb.X_ASSIGN_Q)
+        frame = ctx.export(hb.X_PI) // wl.tokens_per_frame
+        assert (A[:, frame == 0] == np.arange(wl.n_tokens)[frame == 0]).all()
+        assert ctx.query(hb.Q_OUTLIERS) == int(np.floor(0.05 * wl.heads * wl.n_tokens + 1e-9))
+
+
+def test_medium_size_anchored_sampled():
+    """The benchmark's scene with 4-frame blocks and anchoring: maps and merged tensors on all tokens, output sampled."""
+    wl = synth.WORKLOADS["medium"].replace(blk_frames=4, blk_h=4, blk_w=2)
+    rng = np.random.default_rng(3)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 48), [0, 4, 5, wl.n_tokens - 1]]))
+    stats = run_anchored(wl, sample=toks)
+    assert stats["out_err"] <= parity.OUT_TOL
