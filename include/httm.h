@@ -115,8 +115,8 @@ enum {
 /* httm_launch_stage selectors.  0-4: the five separate kernels of the path (match and merge read the
  * reordered copies written by the reorder kernel).  5, 6: the match and merge kernels reading their blocks
  * straight from q, k, v (the temporal reorder folded into their tiled loads; UNSUPPORTED only for scenes of
- * more than 32767 frames, patch rows or patch columns).  httm_global_attention runs 5, 6, 3, 4
- * (0, 1, 2, 3, 4 for such oversized scenes); both orders give the same maps. */
+ * more than 32767 frames, patch rows or patch columns, or more than 32 special tokens per frame).
+ * httm_global_attention runs 5, 6, 3, 4 (0, 1, 2, 3, 4 for such scenes); both orders give the same maps. */
 enum {
     HTTM_STAGE_REORDER = 0,
     HTTM_STAGE_MATCH = 1,
@@ -153,7 +153,8 @@ int httm_create(const httm_config* cfg, httm_ctx** out);
  *   inverse reorder + head concat (Eq. 5-7).
  * Match and merge load each block's patch window straight from q, k, v and no reordered
  * copy is written (four kernels; HTTM_X_*_REORDERED hold what the last HTTM_STAGE_REORDER
- * wrote).  Scenes of more than 32767 frames / patch rows / patch columns take five.
+ * wrote).  Scenes of more than 32767 frames / patch rows / patch columns, or with more than 32 special
+ * tokens per frame, take five.
  * With ratio_q = ratio_kv = 0 the result equals httm_dense_attention up to rounding.
  * Errors: INVALID_ARG, ALIGNMENT, CUDA (launch failure); device-side wait time-outs
  * are reported by the next httm_query(HTTM_Q_DEVICE_STATUS) / httm_export.

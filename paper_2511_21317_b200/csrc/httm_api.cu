@@ -206,7 +206,11 @@ SourceLayout source_layout(const httm_ctx* c) {
 
 // The match and merge kernels read every block straight from Q/K/V (tiled TMA loads of the block's patch window):
 // the reordered copies are not needed on the hot path (the 16-bit block coordinates bound the scene size).
-bool direct_mode(const httm_ctx* c) { return c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767; }
+// A frame's special tokens are staged by one load of n_special rows into the 32-row stage of the merge kernel: more of
+// them per frame take the path over the reordered copies (special tokens in chunks of 32).
+bool direct_mode(const httm_ctx* c) {
+    return c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767 && c->n_special <= 32;
+}
 
 BigMatchArgs big_match_args(httm_ctx* c) {
     BigMatchArgs a{};
@@ -590,7 +594,7 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
         return HTTM_OK;
     }
     if (c->max_block > 32) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering supports merging blocks of at most 32 tokens");
-    if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering needs a scene of at most 32767 frames / patch rows / patch columns");
+    if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering needs a scene of at most 32767 frames / patch rows / patch columns and at most 32 special tokens per frame");
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
     if (!c->d_eps) {
@@ -706,7 +710,7 @@ int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm
             return stage_outlier(c, q, s);
         case HTTM_STAGE_MATCH_DIRECT:
         case HTTM_STAGE_MERGE_DIRECT: {
-            if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "direct stages need a scene of at most 32767 frames / patch rows / patch columns");
+            if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "direct stages need a scene of at most 32767 frames / patch rows / patch columns and at most 32 special tokens per frame");
             if ((rc = check_tensor(c, q, "q")) || (rc = check_tensor(c, k, "k")) || (rc = check_tensor(c, v, "v"))) return rc;
             const httm_tensor src[3] = {q, k, v};
             return stage == HTTM_STAGE_MATCH_DIRECT ? stage_match(c, s, src) : stage_merge(c, s, src);

@@ -66,6 +66,8 @@ GEOMS = [
     ("block_64", 9, 10, 10, (4, 4, 4), 0.5, 0.9, 1, 4, 2),
     ("block_256_max", 5, 9, 8, (4, 8, 8), 0.8, 0.3, 1, 4, 1),
     ("one_frame", 1, 12, 12, (2, 4, 4), 0.5, 0.5, 1, 4, 2),
+    ("many_specials", 3, 6, 6, (2, 4, 4), 0.5, 0.5, 1, 44, 2),      # 45 special tokens per frame: the path over the reordered copies
+    ("many_specials_64", 3, 8, 8, (4, 4, 4), 0.6, 0.6, 3, 67, 2),
 ]
 
 
