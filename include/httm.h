@@ -177,6 +177,18 @@ int httm_global_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tens
 int httm_set_outlier_fraction(httm_ctx* ctx, double fraction);
 
 /*
+ * The projections around the path (Algorithm 1: Q, K, V = x W_qkv before it, out = Attn W_o after it) for callers
+ * that want no library matmul next to the path:  y[n_rows][out_features] = x[n_rows][in_features] . w^T  with the
+ * weight given as w[out_features][in_features] (the layout a linear layer stores), all bf16 on the context's device,
+ * fp32 accumulation, one rounding to bf16; ldx / ldw / ldy are the row strides in elements.  No bias.  One kernel on
+ * `stream` (tcgen05 GEMM).  x and w are only read; y must not overlap them.
+ * Errors: INVALID_ARG, ALIGNMENT (pointers 16-byte aligned, strides multiples of 8), UNSUPPORTED (in_features must be
+ * a multiple of 64, out_features a multiple of 8), CUDA; a device-side wait time-out is reported like the others.
+ */
+int httm_linear(httm_ctx* ctx, const void* x, int64_t ldx, const void* w, int64_t ldw, void* y, int64_t ldy,
+                int64_t n_rows, int32_t in_features, int32_t out_features, void* cuda_stream);
+
+/*
  * Exact multi-head softmax attention over all N tokens (the unmerged baseline the
  * paper's speed-ups are measured against, Sec. 4.1), same attention kernel, output
  * written directly in `out`'s layout.  Same argument rules and errors as above.

@@ -33,7 +33,7 @@ _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPO
 EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
-    "httm_global_attention_static", "httm_selftest_tensor_core", "httm_set_outlier_fraction",
+    "httm_global_attention_static", "httm_selftest_tensor_core", "httm_set_outlier_fraction", "httm_linear",
 )
 
 
@@ -70,6 +70,7 @@ def load_library() -> ctypes.CDLL:
     L.httm_global_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_dense_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_set_outlier_fraction.argtypes = [vp, ctypes.c_double]
+    L.httm_linear.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, ctypes.c_int32, ctypes.c_int32, vp]
     L.httm_attention_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
     L.httm_launch_stage.argtypes = [vp, ctypes.c_int, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_query.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64)]
@@ -212,6 +213,21 @@ class Httm:
     def set_outlier_fraction(self, fraction: float):
         """Query outlier filtering (Sec. 3.4) for the later calls; 0 switches it off."""
         self._check(self._lib.httm_set_outlier_fraction(self._h, float(fraction)))
+
+    def linear(self, x: torch.Tensor, w: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
+        """y = x . w^T with x [n][in], w [out][in] (rows may be strided), bf16 CUDA tensors; returns y [n][out]."""
+        for t, name in ((x, "x"), (w, "w")):
+            if t.dtype != torch.bfloat16 or not t.is_cuda or t.dim() != 2 or t.stride(1) != 1:
+                raise HttmError(ERR_INVALID_ARG, f"{name}: expected a CUDA bfloat16 matrix with contiguous rows")
+        if w.shape[1] != x.shape[1]:
+            raise HttmError(ERR_INVALID_ARG, "w: expected [out_features][in_features]")
+        if out is None:
+            out = torch.empty(x.shape[0], w.shape[0], dtype=torch.bfloat16, device=x.device)
+        elif out.dtype != torch.bfloat16 or not out.is_cuda or out.shape != (x.shape[0], w.shape[0]) or out.stride(1) != 1:
+            raise HttmError(ERR_INVALID_ARG, "out: expected a CUDA bfloat16 matrix [n][out_features] with contiguous rows")
+        self._check(self._lib.httm_linear(self._h, x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), out.data_ptr(), out.stride(0),
+                                          x.shape[0], x.shape[1], w.shape[0], self._stream(stream)))
+        return out
 
     def launch_stage(self, stage: int, q=None, k=None, v=None, out=None, stream=None):
         tq = self._tensor(q, "q") if q is not None else _null_tensor()

@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libhttm.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["httm_api.cu", "httm_mem_kernels.cu", "httm_attention_tc.cu", "httm_big_blocks.cu", "httm_static.cu",
+SOURCES = ["httm_api.cu", "httm_mem_kernels.cu", "httm_attention_tc.cu", "httm_big_blocks.cu", "httm_linear.cu", "httm_static.cu",
            "httm_umma_selftest.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

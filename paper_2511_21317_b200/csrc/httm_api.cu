@@ -538,6 +538,7 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
     c->sm_count = prop.multiProcessorCount;
     if ((rc = check_cuda(c, configure_kernels(), "cudaFuncSetAttribute"))) return done(rc);
     if ((rc = check_cuda(c, configure_big_blocks(), "cudaFuncSetAttribute"))) return done(rc);
+    if ((rc = check_cuda(c, configure_linear(), "cudaFuncSetAttribute"))) return done(rc);
 
     const size_t H = cfg->heads, N = c->n_tokens;
     if ((rc = c->alloc(&c->d_pi, N)) || (rc = c->alloc(&c->d_pi_inv, N)) || (rc = c->alloc(&c->d_blocks, c->blocks.size())) || (rc = c->alloc(&c->d_geom, c->geom.size())) ||
@@ -618,6 +619,39 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
     }
     c->outlier_fraction = fraction;
     return HTTM_OK;
+}
+
+int httm_linear(httm_ctx* c, const void* x, int64_t ldx, const void* w, int64_t ldw, void* y, int64_t ldy, int64_t n_rows,
+                int32_t in_features, int32_t out_features, void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (n_rows < 0 || in_features < 1 || out_features < 1 || n_rows > (1ll << 31) - 256)
+        return c->fail(HTTM_ERR_INVALID_ARG, "linear: sizes out of range");
+    if (n_rows == 0) return HTTM_OK;   // nothing to do (an empty matrix may come with a null pointer)
+    if (!x || !w || !y) return c->fail(HTTM_ERR_INVALID_ARG, "linear: null pointer");
+    if (in_features % 64 != 0 || out_features % 8 != 0)
+        return c->fail(HTTM_ERR_UNSUPPORTED, "linear: in_features must be a multiple of 64 and out_features a multiple of 8");
+    if ((((uintptr_t)x | (uintptr_t)w | (uintptr_t)y) & 15u) != 0 || ldx % 8 != 0 || ldw % 8 != 0 || ldy % 8 != 0)
+        return c->fail(HTTM_ERR_ALIGNMENT, "linear: pointers must be 16-byte aligned and leading dimensions multiples of 8");
+    if (ldx < in_features || ldw < in_features || ldy < out_features)
+        return c->fail(HTTM_ERR_INVALID_ARG, "linear: a leading dimension is smaller than its row");
+    if (overlaps(y, ((n_rows - 1) * ldy + out_features) * 2, x, ((n_rows - 1) * ldx + in_features) * 2) ||
+        overlaps(y, ((n_rows - 1) * ldy + out_features) * 2, w, ((int64_t)(out_features - 1) * ldw + in_features) * 2))
+        return c->fail(HTTM_ERR_INVALID_ARG, "linear: y overlaps an input");
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    LinearArgs a{};
+    a.x = static_cast<const __nv_bfloat16*>(x);
+    a.w = static_cast<const __nv_bfloat16*>(w);
+    a.y = static_cast<__nv_bfloat16*>(y);
+    a.ldx = ldx;
+    a.ldw = ldw;
+    a.ldy = ldy;
+    a.n_rows = n_rows;
+    a.in_features = in_features;
+    a.out_features = out_features;
+    a.status = c->d_status;
+    c->launches++;
+    return check_cuda(c, launch_linear(a, c->sm_count, static_cast<cudaStream_t>(cuda_stream)), "linear launch");
 }
 
 int httm_dense_attention(httm_ctx* c, httm_tensor q, httm_tensor k, httm_tensor v, httm_tensor out, void* cuda_stream) {

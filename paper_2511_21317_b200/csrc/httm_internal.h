@@ -20,7 +20,8 @@ enum : int {
     kDevTimeoutMatchLoad = 1,   // match kernel: bulk copy of a block did not complete in time
     kDevTimeoutAttention = 2,   // attention kernel: a pipeline barrier did not complete in time
     kDevBadIndex = 3,           // an index read from a map was out of range (skipped)
-    kDevTimeoutBigMatch = 4     // large-block score kernel: a pipeline barrier did not complete in time
+    kDevTimeoutBigMatch = 4,    // large-block score kernel: a pipeline barrier did not complete in time
+    kDevTimeoutLinear = 5       // projection GEMM: a pipeline barrier did not complete in time
 };
 
 // One merging block (Sec. 3.3): tokens [start, start + n) of the reordered sequence.
@@ -160,6 +161,14 @@ struct AttentionArgs {
     const int32_t* tile_prefix;
 };
 
+struct LinearArgs {   // y[n_rows][out] = x[n_rows][in] . w[out][in]^T, leading dimensions in elements
+    const __nv_bfloat16 *x, *w;
+    __nv_bfloat16* y;
+    int64_t ldx, ldw, ldy, n_rows;
+    int32_t in_features, out_features;
+    int32_t* status;
+};
+
 // Launchers (each enqueues exactly one kernel on `stream`; returns the CUDA error).
 cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream);
 cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
@@ -172,6 +181,8 @@ cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t 
 cudaError_t launch_big_select(const BigMatchArgs& a, cudaStream_t stream);                  // top-r per (tensor, head, block)
 cudaError_t launch_big_merge(const MergeArgs& a, cudaStream_t stream);                      // sort by merged row + gather means
 cudaError_t configure_big_blocks();
+cudaError_t launch_linear(const LinearArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 GEMM for the projections
+cudaError_t configure_linear();
 cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 / TMEM kernel
 cudaError_t configure_attention();
 cudaError_t configure_kernels();   // one-time function attributes (dynamic shared memory sizes)
