@@ -169,10 +169,13 @@ struct TaskCursor {
 // ------------------------------------------------------------------------------------
 // warps per CTA (one CTA per SM): as many as the shared memory takes at two stages per warp; a warp works alone on its
 // blocks, so the number of warps per scheduler is what hides its instruction latencies
-__host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 32 ? 8 : (nmax <= 64 ? 12 : (nmax <= 128 ? 6 : 3)); }
+__host__ __device__ constexpr int match_warps_per_cta(int nmax) { return nmax <= 32 ? 8 : (nmax <= 64 ? 16 : (nmax <= 128 ? 12 : 6)); }
+// stages per warp: blocks of more than 64 tokens keep a warp busy for many microseconds, far longer than a load takes; one
+// stage there buys twice the warps for the same shared memory
+__host__ __device__ constexpr int match_stages(int nmax) { return nmax <= 32 ? 2 : 1; }
 __host__ __device__ constexpr int match_aux_bytes(int nmax) { return nmax * 4 + 16; }   // inverse norms + 2 mbarriers
 __host__ __device__ constexpr int match_smem_bytes(int nmax) {
-    return match_warps_per_cta(nmax) * (2 * nmax * kRowBytes + match_aux_bytes(nmax)) + 1024 /*alignment slack*/;
+    return match_warps_per_cta(nmax) * (match_stages(nmax) * nmax * kRowBytes + match_aux_bytes(nmax)) + 1024 /*alignment slack*/;
 }
 
 // tiled TMA load {64 channels, rows, heads} -> this CTA's shared memory; the channel coordinate is 0
@@ -242,15 +245,16 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     constexpr int MT = NMAX / 16;        // 16-token row tiles
     constexpr int NT = NMAX / 32;        // 8-dst column tiles (n_dst <= NMAX / 4)
     constexpr bool KEEP_A = PASSES == 1; // row-tile fragments stay in registers between the two passes
+    constexpr int STAGES = match_stages(NMAX);
     constexpr uint32_t STAGE_BYTES = NMAX * kRowBytes;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;   // accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
-    unsigned char* aux = smem + (size_t)WARPS * 2 * STAGE_BYTES + (size_t)warp * match_aux_bytes(NMAX);
+    unsigned char* aux = smem + (size_t)WARPS * STAGES * STAGE_BYTES + (size_t)warp * match_aux_bytes(NMAX);
     float* invn = reinterpret_cast<float*>(aux);                                   // [NMAX]
-    const uint32_t mbar0 = smem_u32(aux + NMAX * 4);                               // 2 mbarriers
-    const uint32_t stage0 = smem_u32(smem + (size_t)warp * 2 * STAGE_BYTES);       // [2][NMAX][128], 1024-aligned
+    const uint32_t mbar0 = smem_u32(aux + NMAX * 4);                               // 2 mbarriers (one used with a single stage)
+    const uint32_t stage0 = smem_u32(smem + (size_t)warp * STAGES * STAGE_BYTES);  // [STAGES][NMAX][128], 1024-aligned
 
     if (lane == 0) {
         mbar_init(mbar0, 1);
@@ -296,8 +300,10 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     };
     if (first < n_tasks && lane == 0) issue(nxt, 0);
     nxt.advance();
-    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
-    nxt.advance();
+    if (STAGES == 2) {
+        if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+        nxt.advance();
+    }
 
     int cached_n = -1, cached_nd = -1;
     uint32_t magic_n = 0, magic_nd = 0;
@@ -305,9 +311,9 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     int it = 0;
     bool failed = false;
     for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
-        const int buf = it & 1;
-        const uint32_t parity = (it >> 1) & 1;
-        const bool more = task + 2 * stride < n_tasks;
+        const int buf = STAGES == 2 ? (it & 1) : 0;
+        const uint32_t parity = STAGES == 2 ? ((it >> 1) & 1) : (it & 1);
+        const bool more = task + STAGES * stride < n_tasks;
         const BlockInfo bi = a.blocks[cur.u];
         const int n = bi.n, r = cur.t == 0 ? bi.r_q : bi.r_k, nd = cur.t == 0 ? bi.nd_q : bi.nd_k;
         int32_t* A = a.assign[cur.t] + (int64_t)cur.h * a.n_tokens + bi.start;
@@ -522,8 +528,8 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
     if (failed) {
         // give copies that may still be in flight a bounded chance to land before the CTA's
         // shared memory is released
-        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
-        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+        mbar_wait_bounded(mbar0, STAGES == 2 ? ((it >> 1) & 1) : (it & 1), a.status, kDevTimeoutMatchLoad);
+        if (STAGES == 2) mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
     }
 }
 
@@ -869,10 +875,11 @@ static cudaError_t launch_merge_tc(const MergeArgs& a, int sm_count, cudaStream_
 //     (row tile, token step) with ldmatrix.trans from the swizzled TMA stage (blocks come from the
 //     reordered copies).  Group sizes are counted with shared-memory atomics.
 // ------------------------------------------------------------------------------------
-__host__ __device__ constexpr int merge_multi_warps(int nmax) { return nmax <= 64 ? 12 : (nmax <= 128 ? 6 : 3); }   // as for the match kernel
+__host__ __device__ constexpr int merge_multi_warps(int nmax) { return nmax <= 64 ? 16 : (nmax <= 128 ? 12 : 6); }   // as for the match kernel
+__host__ __device__ constexpr int merge_multi_stages(int nmax) { return nmax <= 32 ? 2 : 1; }                          // (see match_stages)
 __host__ __device__ constexpr int merge_multi_aux(int nmax) { return nmax * 8 + 16; }   // counts, reciprocals, 2 mbarriers
 __host__ __device__ constexpr int merge_multi_smem(int nmax) {
-    return merge_multi_warps(nmax) * (2 * nmax * kRowBytes + merge_multi_aux(nmax)) + 1024 /*alignment slack*/;
+    return merge_multi_warps(nmax) * (merge_multi_stages(nmax) * nmax * kRowBytes + merge_multi_aux(nmax)) + 1024 /*alignment slack*/;
 }
 
 template <int PASSES, bool DIRECT>
@@ -882,14 +889,15 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                    const __grid_constant__ CUtensorMap map_sk, const __grid_constant__ CUtensorMap map_sv, const MergeArgs a) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = merge_multi_warps(NMAX);
+    constexpr int STAGES = merge_multi_stages(NMAX);
     constexpr int KS = NMAX / 16;   // token steps
     constexpr uint32_t STAGE_BYTES = NMAX * kRowBytes;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;   // accumulator layout: rows g, g + 8; columns 2 tq, 2 tq + 1
-    unsigned char* stage = smem + (size_t)warp * 2 * STAGE_BYTES;                       // [2][NMAX][128], 1024-aligned, swizzled
-    unsigned char* aux = smem + (size_t)WARPS * 2 * STAGE_BYTES + (size_t)warp * merge_multi_aux(NMAX);
+    unsigned char* stage = smem + (size_t)warp * STAGES * STAGE_BYTES;                  // [STAGES][NMAX][128], 1024-aligned, swizzled
+    unsigned char* aux = smem + (size_t)WARPS * STAGES * STAGE_BYTES + (size_t)warp * merge_multi_aux(NMAX);
     int* cnt = reinterpret_cast<int*>(aux);                                             // [NMAX] group size of kept row
     float* rcnt = reinterpret_cast<float*>(aux + NMAX * 4);                             // [NMAX] its reciprocal
     const uint32_t mbar0 = smem_u32(aux + NMAX * 8), stage0 = smem_u32(stage);
@@ -956,15 +964,17 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     };
     if (first < n_tasks && lane == 0) issue(nxt, 0);
     nxt.advance();
-    if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
-    nxt.advance();
+    if (STAGES == 2) {
+        if (first + stride < n_tasks && lane == 0) issue(nxt, 1);
+        nxt.advance();
+    }
 
     int it = 0;
     bool failed = false;
     for (int64_t task = first; task < n_tasks; task += stride, ++it, cur.advance(), nxt.advance()) {
-        const int buf = it & 1;
-        const uint32_t parity = (it >> 1) & 1;
-        const bool more = task + 2 * stride < n_tasks;
+        const int buf = STAGES == 2 ? (it & 1) : 0;
+        const uint32_t parity = STAGES == 2 ? ((it >> 1) & 1) : (it & 1);
+        const bool more = task + STAGES * stride < n_tasks;
         const int t = cur.t, h = cur.h;
         const bool special = cur.u >= a.n_blocks;
         int start, n, r, moff;
@@ -1102,8 +1112,8 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (more && lane == 0) issue(nxt, buf);
     }
     if (failed) {
-        mbar_wait_bounded(mbar0, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
-        mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
+        mbar_wait_bounded(mbar0, STAGES == 2 ? ((it >> 1) & 1) : (it & 1), a.status, kDevTimeoutMatchLoad);
+        if (STAGES == 2) mbar_wait_bounded(mbar0 + 8, (it >> 1) & 1, a.status, kDevTimeoutMatchLoad);
     }
 }
 
@@ -1111,6 +1121,7 @@ template <int PASSES>
 static cudaError_t launch_merge_multi(const MergeArgs& a, int sm_count, cudaStream_t stream) {
     constexpr int NMAX = 32 * PASSES;
     constexpr int WARPS = merge_multi_warps(NMAX);
+    constexpr int STAGES = merge_multi_stages(NMAX);
     CUtensorMap m[3], sp[3];
     const int64_t N = a.n_tokens;
     const bool direct = a.geom != nullptr;
