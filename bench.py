@@ -360,7 +360,7 @@ def run_ours(args, wl):
             line["cpu_baseline"] = {"value": N / sec, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
                                     "sample": info["sample"], "seconds": info["seconds"], "ms_per_layer_extrapolated": sec * 1e3}
             line["parity_sample"] = parity_sample(ctx, hb, wl, kept, out)
-        if world == 1 and args.outlier_fraction > 0 and not big:
+        if world == 1 and args.outlier_fraction > 0:
             line["outlier_filter"] = filtered_variant(args, wl, hb, dq, dk, dv, local)
         print(json.dumps(line), flush=True)
     ctx.close()
@@ -373,8 +373,9 @@ def filtered_variant(args, wl, hb, dq, dk, dv, device_index):
     import torch
     ctx = hb.Httm(hb.HttmConfig.of(wl, device=device_index))
     try:
-        if ctx.query(hb.Q_MAX_BLOCK_TOKENS) > 32:
-            return {"skipped": "outlier filtering supports merging blocks of at most 32 tokens"}
+        max_block = ctx.query(hb.Q_MAX_BLOCK_TOKENS)
+        if 32 < max_block <= 256:
+            return {"skipped": "outlier filtering supports merging blocks of at most 32 tokens, or of more than 256"}
         ctx.set_outlier_fraction(args.outlier_fraction)
         out = ctx.new_output()
         stream = torch.cuda.current_stream()
@@ -390,7 +391,11 @@ def filtered_variant(args, wl, hb, dq, dk, dv, device_index):
         e1.record(stream)
         torch.cuda.synchronize()
         launches = (ctx.launch_count() - l0) // steps
-        order = [hb.STAGE_MATCH_DIRECT, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE_DIRECT, hb.STAGE_ATTENTION, hb.STAGE_UNMERGE]
+        if max_block > 256:
+            order = [hb.STAGE_REORDER, hb.STAGE_BIG_SCORES, hb.STAGE_BIG_SELECT, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE, hb.STAGE_ATTENTION,
+                     hb.STAGE_UNMERGE]
+        else:
+            order = [hb.STAGE_MATCH_DIRECT, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE_DIRECT, hb.STAGE_ATTENTION, hb.STAGE_UNMERGE]
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(order) + 1)] for _ in range(steps)]
         for s_ in range(steps):
             evs[s_][0].record(stream)

@@ -125,7 +125,8 @@ enum {
     HTTM_STAGE_UNMERGE = 4,
     HTTM_STAGE_MATCH_DIRECT = 5,
     HTTM_STAGE_MERGE_DIRECT = 6,
-    HTTM_STAGE_OUTLIER_FILTER = 7,/* between 5 and 6, only after httm_set_outlier_fraction(> 0): five small kernels */
+    HTTM_STAGE_OUTLIER_FILTER = 7,/* between 5 and 6, only after httm_set_outlier_fraction(> 0): five small kernels
+                                     (six between 9 and 2 for blocks of more than 256 tokens) */
     /* merging blocks of 257 .. 4096 tokens (the paper's runs of 128 tokens over 30 frames, Sec. 4.1): stages 1, 5, 6 are
      * UNSUPPORTED; the order is 0, 8, 9, 2, 3, 4.  8: cosine of every token with every dst token of its block on the
      * tensor cores + best dst per token; 9: the r best src of every block merge (map written) */
@@ -171,7 +172,8 @@ int httm_global_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tens
  * destination token continues under its remaining member with the lowest reordered position.  Only queries are
  * filtered; K and V are untouched.  The merged query length then differs from head to head (HTTM_X_MERGED_Q_HEAD).
  * The first call with fraction > 0 allocates the extra workspace (device allocation: call it outside timed regions).
- * Supported for merging blocks of at most 32 tokens and scenes of at most 32767 frames / patch rows / columns.
+ * Supported for merging blocks of at most 32 tokens (scenes of at most 32767 frames / patch rows / columns, at most 32
+ * special tokens per frame) and for blocks of more than 256 tokens (there six kernels, see HTTM_STAGE_OUTLIER_FILTER).
  * Errors: INVALID_ARG (fraction outside [0, 1]), UNSUPPORTED, NOMEM, CUDA.
  */
 int httm_set_outlier_fraction(httm_ctx* ctx, double fraction);

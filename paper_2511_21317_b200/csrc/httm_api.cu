@@ -359,6 +359,14 @@ int stage_outlier(httm_ctx* c, const httm_tensor& q, cudaStream_t s) {
     a.status = c->d_status;
     int rc;
     if ((rc = check_cuda(c, cudaMemsetAsync(c->d_sel, 0, kSelWords * sizeof(int32_t), s), "selection state reset"))) return rc;
+    if (c->big()) {   // large blocks: the blocks are runs of rows of the reordered copy; six kernels
+        a.src_q = view(c->d_qr, c->n_tokens);
+        if ((rc = check_cuda(c, launch_big_deviation(a, s), "large-block deviation launch"))) return rc;
+        if ((rc = check_cuda(c, launch_threshold0(a, c->sm_count, s), "threshold launch"))) return rc;
+        if ((rc = check_cuda(c, launch_big_filter(a, s), "large-block filter launch"))) return rc;
+        c->launches += 6;
+        return check_cuda(c, launch_offsets(a, s), "offsets launch");
+    }
     if ((rc = check_cuda(c, launch_deviation(a, c->sm_count, s), "deviation launch"))) return rc;
     if ((rc = check_cuda(c, launch_threshold(a, c->sm_count, s), "threshold launch"))) return rc;
     c->launches += 5;
@@ -390,6 +398,7 @@ int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const h
         if ((rc = stage_reorder(c, q, k, v, s))) return rc;
         if ((rc = stage_big_scores(c, s))) return rc;
         if ((rc = stage_big_select(c, s))) return rc;
+        if (c->filtering() && (rc = stage_outlier(c, q, s))) return rc;
         if ((rc = stage_merge(c, s))) return rc;
         if ((rc = stage_attention(c, s))) return rc;
         return stage_unmerge(c, out, s);
@@ -594,8 +603,9 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
         c->outlier_fraction = 0.0;
         return HTTM_OK;
     }
-    if (c->max_block > 32) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering supports merging blocks of at most 32 tokens");
-    if (!direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering needs a scene of at most 32767 frames / patch rows / patch columns and at most 32 special tokens per frame");
+    if (c->max_block > 32 && !c->big())
+        return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering supports merging blocks of at most 32 tokens, or of more than 256");
+    if (!c->big() && !direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering needs a scene of at most 32767 frames / patch rows / patch columns and at most 32 special tokens per frame");
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
     if (!c->d_eps) {

@@ -425,6 +425,108 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// The groups of one block from its map A (every thread of a 1024-thread CTA calls this): merged row of every kept token =
+// its rank among the kept tokens in position order (row_of; -1 for merged tokens); all tokens sorted by (merged row,
+// position) in keys[] = (row << 12) | position, so that the members of a row are one ascending run; seg[row] = first
+// sorted index of the row, seg[n_kept] = n.  rep_of_row (optional) gets the position of every row's kept token; rank_out
+// (optional) the merged row of every token plus moff.  Returns the number of kept tokens, at most `limit` (tokens whose
+// row would lie beyond it, or whose target is not a kept token, are recorded as a corrupt map and left out).
+__device__ int build_groups(const int32_t* A, int block_start, int n, int limit, uint32_t* keys, int16_t* row_of, int* seg, int* warp_sum,
+                            int16_t* rep_of_row, int32_t* status, int32_t* rank_out, int moff) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int rep[4];
+    int kept = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        rep[e] = -1;
+        if (j < n) {
+            rep[e] = A[j] - block_start;
+            if (rep[e] < 0 || rep[e] >= n) {   // corrupt map: record, treat as kept
+                atomicCAS(status, kDevOk, kDevBadIndex);
+                rep[e] = j;
+            }
+            kept += rep[e] == j ? 1 : 0;
+        }
+    }
+    int incl = kept;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+    }
+    __syncthreads();   // (the scratch arrays may still be in use by a previous call's readers)
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_sum[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, w, off);
+            if (lane >= off) w += o;
+        }
+        warp_sum[lane] = w;
+    }
+    __syncthreads();
+    const int n_kept = min(warp_sum[31], limit);
+    int next_row = (warp > 0 ? warp_sum[warp - 1] : 0) + incl - kept;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        if (j < n) {
+            const bool is_kept = rep[e] == j;
+            row_of[j] = is_kept ? (int16_t)next_row : (int16_t)-1;
+            if (is_kept) {
+                if (rep_of_row && next_row < n_kept) rep_of_row[next_row] = (int16_t)j;
+                ++next_row;
+            }
+        }
+    }
+    __syncthreads();
+    int P = 512;
+    while (P < n) P <<= 1;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int j = 4 * tid + e;
+        uint32_t key = 0xffffffffu;
+        if (j < n) {
+            int row = row_of[rep[e]];
+            if (row < 0 || row >= n_kept) {   // target is not a kept token, or more kept tokens than a valid map has
+                atomicCAS(status, kDevOk, kDevBadIndex);
+                row = 0xfffff;                // sorts behind every valid row, is never gathered
+            } else if (rank_out) {
+                rank_out[j] = moff + row;
+            }
+            key = ((uint32_t)row << 12) | (uint32_t)j;
+        }
+        if (j < P) keys[j] = key;
+    }
+    __syncthreads();
+    for (int k = 2; k <= P; k <<= 1) {   // bitonic sort: the keys are distinct, so the order is unique
+        for (int jj = k >> 1; jj > 0; jj >>= 1) {
+            for (int i = tid; i < P; i += MG_THREADS) {
+                const int ixj = i ^ jj;
+                if (ixj > i) {
+                    const uint32_t x = keys[i], y = keys[ixj];
+                    if ((x > y) == ((i & k) == 0)) {
+                        keys[i] = y;
+                        keys[ixj] = x;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = tid; i <= n; i += MG_THREADS) {
+        const int row = i < n ? (int)(keys[i] >> 12) : n_kept;
+        const int prev = i > 0 ? (int)(keys[i - 1] >> 12) : -1;
+        if (row != prev && prev < n_kept)   // every row from prev + 1 to row starts here (rows without members cannot occur in a valid map)
+            for (int q = prev + 1; q <= min(row, n_kept); ++q) seg[q] = i;
+    }
+    __syncthreads();
+    return n_kept;
+}
+
 __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArgs a, int sp_chunks) {
     extern __shared__ __align__(16) unsigned char mg_smem[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);                                     // [P] (merged row << 12) | position
@@ -450,94 +552,14 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArg
     const int per_map = a.heads * a.n_blocks;
     const int m = blockIdx.x / per_map, h = (blockIdx.x % per_map) / a.n_blocks, b = blockIdx.x % a.n_blocks;
     const BlockInfo bi = a.blocks[b];
-    const int n = bi.n, r = m == 0 ? bi.r_q : bi.r_k, moff = m == 0 ? bi.moff_q : bi.moff_k, m_len = m == 0 ? a.m_q : a.m_k;
-    const int n_kept = n - r;
+    const int n = bi.n, r = m == 0 ? bi.r_q : bi.r_k, m_len = m == 0 ? a.m_q : a.m_k;
+    const bool variable = m == 0 && a.moff_q_var != nullptr;   // after outlier filtering the kept count of a block varies by head
+    const int moff = m == 0 ? (variable ? __ldg(a.moff_q_var + (int64_t)h * a.n_blocks + b) : bi.moff_q) : bi.moff_k;
+    const int limit = variable ? n : n - r;                    // most kept tokens a valid map can have
     const int64_t base = (int64_t)h * a.n_tokens + bi.start;
     const int32_t* A = a.assign[m] + base;
 
-    // merged row of every kept token = its rank among the kept tokens, in position order
-    int rep[4];
-    int kept = 0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int j = 4 * tid + e;
-        rep[e] = -1;
-        if (j < n) {
-            rep[e] = A[j] - bi.start;
-            if (rep[e] < 0 || rep[e] >= n) {   // corrupt map: record, treat as kept
-                atomicCAS(a.status, kDevOk, kDevBadIndex);
-                rep[e] = j;
-            }
-            kept += rep[e] == j ? 1 : 0;
-        }
-    }
-    int incl = kept;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const int o = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += o;
-    }
-    if (lane == 31) warp_sum[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int w = warp_sum[lane];
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int o = __shfl_up_sync(0xffffffffu, w, off);
-            if (lane >= off) w += o;
-        }
-        warp_sum[lane] = w;
-    }
-    __syncthreads();
-    int next_row = (warp > 0 ? warp_sum[warp - 1] : 0) + incl - kept;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int j = 4 * tid + e;
-        if (j < n) row_of[j] = rep[e] == j ? (int16_t)next_row++ : (int16_t)-1;
-    }
-    __syncthreads();
-    // sort the tokens by (merged row, position): the members of every row become one ascending run
-    int P = 512;
-    while (P < n) P <<= 1;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int j = 4 * tid + e;
-        uint32_t key = 0xffffffffu;
-        if (j < n) {
-            int row = row_of[rep[e]];
-            if (row < 0 || row >= n_kept) {   // target is not a kept token, or more kept tokens than the budget allows: corrupt map
-                atomicCAS(a.status, kDevOk, kDevBadIndex);
-                row = 0xfffff;                // sorts behind every valid row, is never gathered
-            } else if (m == 0) {
-                a.rank_q[base + j] = moff + row;
-            }
-            key = ((uint32_t)row << 12) | (uint32_t)j;
-        }
-        if (j < P) keys[j] = key;
-    }
-    __syncthreads();
-    for (int k = 2; k <= P; k <<= 1) {
-        for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            for (int i = tid; i < P; i += MG_THREADS) {
-                const int ixj = i ^ jj;
-                if (ixj > i) {
-                    const uint32_t x = keys[i], y = keys[ixj];
-                    if ((x > y) == ((i & k) == 0)) {
-                        keys[i] = y;
-                        keys[ixj] = x;
-                    }
-                }
-            }
-            __syncthreads();
-        }
-    }
-    for (int i = tid; i <= n; i += MG_THREADS) {
-        const int row = i < n ? (int)(keys[i] >> 12) : n_kept;
-        const int prev = i > 0 ? (int)(keys[i - 1] >> 12) : -1;
-        if (row != prev && prev < n_kept)   // every row from prev + 1 to row starts here (rows without members cannot occur in a valid map)
-            for (int q = prev + 1; q <= min(row, n_kept); ++q) seg[q] = i;
-    }
-    __syncthreads();
+    const int n_kept = build_groups(A, bi.start, n, limit, keys, row_of, seg, warp_sum, nullptr, a.status, m == 0 ? a.rank_q + base : nullptr, moff);
     // eight lanes per merged row (a lane owns one 16-byte chunk of the row), four rows per warp at a time, four
     // members of a row in flight: the gather is bound by load latency, so it needs many loads in the air.  Member
     // i of a row goes to accumulator i mod 4; the four are added in a fixed order: the result does not depend on
@@ -583,12 +605,185 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArg
     }
 }
 
+// ------------------------------------------------------------------------------------------------ outlier filtering
+// Query outlier filtering (Sec. 3.4, Algorithm 2) for large blocks: the same steps as for small blocks - deviation of
+// every query token from the mean of its group, one threshold over all heads (the refinement kernels of the small-block
+// path, which work on the array of deviations), outliers leave their groups - on the sorted group structure of the merge
+// kernel.  One CTA per (head, block).
+constexpr int OF_SMEM = MG_SMEM + kMaxBigBlockTokens * 2 /*position of every row's kept token*/ + kMaxBigBlockTokens /*outlier flags*/ +
+                        kMaxBigBlockTokens * 2 /*new representative of every row*/;
+
+// eps[h][p] = || q_p - mean of the group p was merged into ||_2 in fp32; 0 for a token on its own
+__global__ void __launch_bounds__(MG_THREADS, 1) big_deviation_kernel(const OutlierArgs a) {
+    extern __shared__ __align__(16) unsigned char mg_smem[];
+    uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);
+    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + kMaxBigBlockTokens * 4);
+    int* seg = reinterpret_cast<int*>(mg_smem + kMaxBigBlockTokens * 6);
+    int* warp_sum = seg + kMaxBigBlockTokens + 4;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ch = lane & 7, sub = lane >> 3;
+    const int h = blockIdx.x / a.n_blocks, b = blockIdx.x % a.n_blocks;
+    const BlockInfo bi = a.blocks[b];
+    const int n = bi.n;
+    const int64_t base = (int64_t)h * a.n_tokens + bi.start;
+    float* eps = a.eps + base;
+    if (bi.r_q == 0) {   // nothing merged in this block (uniform)
+        for (int j = tid; j < n; j += MG_THREADS) eps[j] = 0.f;
+        return;
+    }
+    const int n_kept = build_groups(a.assign_q + base, bi.start, n, n, keys, row_of, seg, warp_sum, nullptr, a.status, nullptr, 0);
+    const __nv_bfloat16* x = a.src_q.ptr + (int64_t)h * a.src_q.stride_head + (int64_t)bi.start * a.src_q.stride_token;
+    const int64_t st = a.src_q.stride_token;
+    // eight lanes per group (a lane owns 8 of the 64 channels), four groups per warp at a time
+    for (int row = warp * 4 + sub; row < ((n_kept + 3) & ~3); row += (MG_THREADS / 32) * 4) {   // (whole sub-groups stay together for the shuffles)
+        const bool live = row < n_kept;
+        const int i0 = live ? seg[row] : 0, i1 = live ? seg[row + 1] : 0;
+        const int cnt = i1 - i0;
+        float mean[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mean[e] = 0.f;
+        if (cnt >= 2) {
+            float acc[4][8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[u][e] = 0.f;
+            for (int i = i0; i < i1; i += 4) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (i + u < i1) v[u] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)(keys[i + u] & 4095u) * st) + ch);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    float f[8];
+                    unpack8f(v[u], f);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[u][e] += f[e];
+                }
+            }
+            const float inv = 1.0f / (float)cnt;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) mean[e] = ((acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e])) * inv;   // kept in fp32
+        }
+        // (the eight lanes of a group walk its members together: the trip count is the same in all of them)
+        for (int i = i0; i < i1; ++i) {
+            const int pos = (int)(keys[i] & 4095u);
+            float d2 = 0.f;
+            if (cnt >= 2) {
+                float f[8];
+                unpack8f(__ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * st) + ch), f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float d = f[e] - mean[e];
+                    d2 = fmaf(d, d, d2);
+                }
+            }
+            const unsigned group_mask = 0xffu << (8 * sub);
+            d2 += __shfl_xor_sync(group_mask, d2, 1);
+            d2 += __shfl_xor_sync(group_mask, d2, 2);
+            d2 += __shfl_xor_sync(group_mask, d2, 4);
+            if (ch == 0) eps[pos] = cnt >= 2 ? sqrtf(d2) : 0.f;
+        }
+    }
+}
+
+// Outliers (eps > tau) leave their groups: an outlier maps to itself; the other tokens of a group stay together, under
+// their old representative if it is not an outlier, else under the remaining member with the lowest position.
+__global__ void __launch_bounds__(MG_THREADS, 1) big_filter_kernel(const OutlierArgs a) {
+    extern __shared__ __align__(16) unsigned char mg_smem[];
+    uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);
+    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + kMaxBigBlockTokens * 4);
+    int* seg = reinterpret_cast<int*>(mg_smem + kMaxBigBlockTokens * 6);
+    int* warp_sum = seg + kMaxBigBlockTokens + 4;
+    int16_t* rep_of_row = reinterpret_cast<int16_t*>(mg_smem + MG_SMEM);
+    unsigned char* outl = mg_smem + MG_SMEM + kMaxBigBlockTokens * 2;
+    int16_t* new_rep = reinterpret_cast<int16_t*>(mg_smem + MG_SMEM + kMaxBigBlockTokens * 3);
+    __shared__ int s_kept, s_out;
+    const int tid = threadIdx.x;
+    const int h = blockIdx.x / a.n_blocks, b = blockIdx.x % a.n_blocks;
+    const BlockInfo bi = a.blocks[b];
+    const int n = bi.n;
+    const int64_t base = (int64_t)h * a.n_tokens + bi.start;
+    const int32_t* A = a.assign_q + base;
+    int32_t* A_out = a.assign_q_out + base;
+    if (bi.r_q == 0) {   // nothing merged, every deviation is 0: nothing to filter unless everything is an outlier, which changes nothing here
+        for (int j = tid; j < n; j += MG_THREADS) A_out[j] = bi.start + j;
+        if (tid == 0) a.kept_cnt[(int64_t)h * a.n_blocks + b] = n;
+        return;
+    }
+    if (tid == 0) {
+        s_kept = 0;
+        s_out = 0;
+    }
+    const float tau = *a.tau;
+    const int n_kept = build_groups(A, bi.start, n, n, keys, row_of, seg, warp_sum, rep_of_row, a.status, nullptr, 0);
+    int n_out = 0;
+    for (int j = tid; j < n; j += MG_THREADS) {
+        const bool o = a.eps[base + j] > tau;
+        outl[j] = o ? 1 : 0;
+        n_out += o ? 1 : 0;
+    }
+    __syncthreads();
+    for (int row = tid; row < n_kept; row += MG_THREADS) {   // a thread per group: groups are short, the rare long one costs its thread a scan
+        const int rp = rep_of_row[row];
+        int nr = rp;
+        if (outl[rp]) {
+            nr = -1;
+            for (int i = seg[row]; i < seg[row + 1]; ++i) {
+                const int pos = (int)(keys[i] & 4095u);
+                if (!outl[pos]) {
+                    nr = pos;
+                    break;
+                }
+            }
+        }
+        new_rep[row] = (int16_t)nr;
+    }
+    __syncthreads();
+    int kept = 0;
+    for (int j = tid; j < n; j += MG_THREADS) {
+        int target = j;
+        if (!outl[j]) {
+            int rp = A[j] - bi.start;
+            if (rp < 0 || rp >= n) rp = j;                  // (recorded by build_groups)
+            const int row = row_of[rp];
+            if (row >= 0 && row < n_kept) target = new_rep[row];   // never -1 here: j itself is a remaining member
+            if (target < 0) target = j;
+        }
+        A_out[j] = bi.start + target;
+        kept += target == j ? 1 : 0;
+    }
+    atomicAdd(&s_kept, kept);
+    atomicAdd(&s_out, n_out);
+    __syncthreads();
+    if (tid == 0) {
+        a.kept_cnt[(int64_t)h * a.n_blocks + b] = s_kept;
+        if (s_out) atomicAdd(a.sel + kSelOutliers, s_out);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_big_deviation(const OutlierArgs& a, cudaStream_t stream) {
+    big_deviation_kernel<<<a.heads * a.n_blocks, MG_THREADS, MG_SMEM, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_big_filter(const OutlierArgs& a, cudaStream_t stream) {
+    big_filter_kernel<<<a.heads * a.n_blocks, MG_THREADS, OF_SMEM, stream>>>(a);
+    return cudaGetLastError();
+}
 
 cudaError_t configure_big_blocks() {
     cudaError_t e = cudaFuncSetAttribute(big_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(big_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM);
+    e = cudaFuncSetAttribute(big_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(big_deviation_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(big_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, OF_SMEM);
 }
 
 cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t stream) {

@@ -1428,16 +1428,17 @@ __device__ void finish_level(const OutlierArgs& a, int level, int* hist) {
 
 constexpr int kRefineThreads = 256;
 // LEVEL 1: histogram of bits 20-10 of the deviations whose bits 31-21 equal the level-0 choice; LEVEL 2: of bits 9-0
-// of those whose bits 31-10 equal the choice so far.
+// of those whose bits 31-10 equal the choice so far.  LEVEL 0 (only where the deviation kernel does not build it on the
+// fly: the large-block path): histogram of bits 31-21 of all deviations.
 template <int LEVEL>
 __global__ void __launch_bounds__(kRefineThreads) refine_kernel(const OutlierArgs a) {
     __shared__ int hist[2048];
     if (__ldcg(a.sel + kSelFinished)) return;   // (same answer in every thread of every CTA)
-    constexpr int NB = LEVEL == 1 ? 2048 : 1024, SHIFT = LEVEL == 1 ? 10 : 0;
-    constexpr uint32_t MASK = LEVEL == 1 ? 0xffe00000u : 0xfffffc00u;
+    constexpr int NB = LEVEL == 2 ? 1024 : 2048, SHIFT = LEVEL == 0 ? 21 : (LEVEL == 1 ? 10 : 0);
+    constexpr uint32_t MASK = LEVEL == 0 ? 0u : (LEVEL == 1 ? 0xffe00000u : 0xfffffc00u);
     for (int i = threadIdx.x; i < NB; i += kRefineThreads) hist[i] = 0;
     __syncthreads();
-    const uint32_t prefix = (uint32_t)__ldcg(a.sel + kSelPrefix + LEVEL - 1);
+    const uint32_t prefix = LEVEL == 0 ? 0u : (uint32_t)__ldcg(a.sel + kSelPrefix + (LEVEL > 0 ? LEVEL - 1 : 0));
     const int64_t count = (int64_t)a.heads * a.n_tokens, quads = count >> 2;
     const uint4* bits4 = reinterpret_cast<const uint4*>(a.eps);   // (the array comes from cudaMalloc: 16-byte aligned)
     auto tally = [&](uint32_t b) {
@@ -1568,13 +1569,26 @@ cudaError_t launch_threshold(const OutlierArgs& a, int sm_count, cudaStream_t st
     refine_kernel<2><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
+cudaError_t launch_threshold0(const OutlierArgs& a, int sm_count, cudaStream_t stream) {
+    const int64_t quads = ((int64_t)a.heads * a.n_tokens) >> 2;
+    int64_t grid = (quads + kRefineThreads * 4 - 1) / (kRefineThreads * 4);
+    if (grid > 2ll * sm_count) grid = 2ll * sm_count;
+    if (grid < 1) grid = 1;
+    refine_kernel<0><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_threshold(a, sm_count, stream);
+}
+cudaError_t launch_offsets(const OutlierArgs& a, cudaStream_t stream) {
+    offsets_kernel<<<(unsigned)a.heads, kOffsetsThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
 cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream) {
     const int64_t threads = (int64_t)a.heads * a.n_blocks * 32;
     filter_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    offsets_kernel<<<(unsigned)a.heads, kOffsetsThreads, 0, stream>>>(a);
-    return cudaGetLastError();
+    return launch_offsets(a, stream);
 }
 
 // ------------------------------------------------------------------------------------

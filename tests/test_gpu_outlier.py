@@ -17,7 +17,7 @@ NAMES = {"pi": hb.X_PI, "blk_start": hb.X_BLOCK_START, "assign_q0": hb.X_ASSIGN_
          "rank_q": hb.X_RANK_Q, "q_m": hb.X_Q_MERGED, "k_m": hb.X_K_MERGED, "v_m": hb.X_V_MERGED, "o_m": hb.X_O_MERGED}
 
 
-def run_filtered(wl, gamma, q=None, k=None, v=None, sample=None, peaky=False):
+def run_filtered(wl, gamma, q=None, k=None, v=None, sample=None, peaky=False, launches=9):
     if q is None:
         q, k, v = synth.make_qkv(wl)
     g = orc.Geometry.of(wl)
@@ -28,7 +28,7 @@ def run_filtered(wl, gamma, q=None, k=None, v=None, sample=None, peaky=False):
         before = ctx.launch_count()
         out = ctx.global_attention(dq, dk, dv)
         torch.cuda.synchronize()
-        assert ctx.launch_count() - before == 9
+        assert ctx.launch_count() - before == launches
         assert ctx.query(hb.Q_DEVICE_STATUS) == 0
         ex = {name: ctx.export(what) for name, what in NAMES.items()}
         stats = parity.filtered_check(g, wl.ratio_q, wl.ratio_kv, gamma, q, k, v, ex, hb.bits_from_bf16(out),
@@ -113,7 +113,7 @@ def test_switching_the_filter_off_restores_the_plain_path():
 
 
 def test_filter_argument_errors():
-    wl = synth.Workload("big_blocks", 4, 8, 8, 4, 4, 4, 0.5, 0.5, heads=2)          # 64-token blocks
+    wl = synth.Workload("mid_blocks", 4, 8, 8, 4, 4, 4, 0.5, 0.5, heads=2)          # 64-token blocks: neither path
     with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
         with pytest.raises(hb.HttmError) as e:
             ctx.set_outlier_fraction(0.1)
@@ -139,3 +139,33 @@ def test_medium_config_filtered_full_size_sampled():
     K = int(np.floor(0.01 * wl.heads * wl.n_tokens + 1e-9))
     assert K - 4 <= stats["outliers"] <= K          # (K unless fp32 deviations tie at the threshold)
     assert stats["out_err"] <= parity.OUT_TOL
+
+
+BIG = [
+    # name, frames, grid_h, grid_w, blk, ratio_q, ratio_kv, n_camera, n_register, heads, gamma
+    ("runs_ragged", 4, 1, 230, (4, 1, 100), 0.9, 0.7, 1, 0, 2, 0.1),
+    ("windows_512", 5, 17, 19, (4, 8, 16), 0.7, 0.5, 1, 4, 2, 0.05),
+    ("runs_3840", 30, 1, 300, (30, 1, 128), 0.9, 0.7, 1, 4, 2, 0.1),          # the paper's block and budgets: 90 % merged, 10 % outliers
+    ("ratio_zero_q", 4, 1, 300, (4, 1, 128), 0.0, 0.7, 1, 4, 2, 0.1),
+    ("everything", 4, 1, 300, (4, 1, 128), 0.8, 0.6, 1, 4, 2, 1.0),
+]
+
+
+@pytest.mark.parametrize("case", BIG, ids=[c[0] for c in BIG])
+def test_large_blocks_filtered(case):
+    """Outlier filtering on the large-block path (reorder, scores, select, deviation, three threshold kernels, filter,
+    offsets, merge, attention, unmerge)."""
+    name, S, h, w, blk, rq, rkv, ncam, nreg, H, gamma = case
+    wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, n_camera=ncam, n_register=nreg, heads=H, seed=9)
+    run_filtered(wl, gamma, peaky=True, launches=12)
+
+
+def test_paper_configuration_full_size_sampled():
+    """Sec. 4.1's configuration on the synthetic stand-in: runs of 128 tokens x 30 frames, 90 % of the queries merged with
+    10 % outliers, 70 % of the keys merged; four heads."""
+    wl = synth.WORKLOADS["paper_1d"].replace(heads=4)
+    rng = np.random.default_rng(4)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 48), [0, 4, 5, wl.n_tokens - 1]]))
+    stats = run_filtered(wl, 0.1, sample=toks, launches=12)
+    K = int(np.floor(0.1 * wl.heads * wl.n_tokens + 1e-9))
+    assert K - 4 <= stats["outliers"] <= K and stats["out_err"] <= parity.OUT_TOL
