@@ -374,8 +374,6 @@ def filtered_variant(args, wl, hb, dq, dk, dv, device_index):
     ctx = hb.Httm(hb.HttmConfig.of(wl, device=device_index))
     try:
         max_block = ctx.query(hb.Q_MAX_BLOCK_TOKENS)
-        if 32 < max_block <= 256:
-            return {"skipped": "outlier filtering supports merging blocks of at most 32 tokens, or of more than 256"}
         ctx.set_outlier_fraction(args.outlier_fraction)
         out = ctx.new_output()
         stream = torch.cuda.current_stream()
@@ -394,6 +392,8 @@ def filtered_variant(args, wl, hb, dq, dk, dv, device_index):
         if max_block > 256:
             order = [hb.STAGE_REORDER, hb.STAGE_BIG_SCORES, hb.STAGE_BIG_SELECT, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE, hb.STAGE_ATTENTION,
                      hb.STAGE_UNMERGE]
+        elif max_block > 32:   # (blocks of 33 .. 256 tokens are filtered over the reordered copies)
+            order = [hb.STAGE_REORDER, hb.STAGE_MATCH, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE, hb.STAGE_ATTENTION, hb.STAGE_UNMERGE]
         else:
             order = [hb.STAGE_MATCH_DIRECT, hb.STAGE_OUTLIER_FILTER, hb.STAGE_MERGE_DIRECT, hb.STAGE_ATTENTION, hb.STAGE_UNMERGE]
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(order) + 1)] for _ in range(steps)]

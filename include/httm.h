@@ -172,9 +172,10 @@ int httm_global_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tens
  * destination token continues under its remaining member with the lowest reordered position.  Only queries are
  * filtered; K and V are untouched.  The merged query length then differs from head to head (HTTM_X_MERGED_Q_HEAD).
  * The first call with fraction > 0 allocates the extra workspace (device allocation: call it outside timed regions).
- * Supported for merging blocks of at most 32 tokens (scenes of at most 32767 frames / patch rows / columns, at most 32
- * special tokens per frame) and for blocks of more than 256 tokens (there six kernels, see HTTM_STAGE_OUTLIER_FILTER).
- * Errors: INVALID_ARG (fraction outside [0, 1]), UNSUPPORTED, NOMEM, CUDA.
+ * Blocks of at most 32 tokens that are loaded straight from q, k, v take five small warp-per-block kernels; every
+ * other geometry (larger blocks, or scenes that go over the reordered copies) takes six kernels that work on the sorted
+ * groups of a block and merges from the reordered copies.
+ * Errors: INVALID_ARG (fraction outside [0, 1]), NOMEM, CUDA.
  */
 int httm_set_outlier_fraction(httm_ctx* ctx, double fraction);
 

@@ -212,6 +212,11 @@ bool direct_mode(const httm_ctx* c) {
     return c->cfg.frames <= 32767 && c->cfg.grid_h <= 32767 && c->cfg.grid_w <= 32767 && c->n_special <= 32;
 }
 
+// Outlier filtering runs on the warp-per-block kernels where blocks have at most 32 tokens and are loaded straight from
+// Q/K/V; everywhere else (larger blocks, or scenes that take the reordered copies) on the sorted-group kernels of the
+// large-block path, which handle any block size from the reordered copy.
+bool sorted_filter(const httm_ctx* c) { return c->filtering() && !(c->max_block <= 32 && direct_mode(c)); }
+
 BigMatchArgs big_match_args(httm_ctx* c) {
     BigMatchArgs a{};
     a.xr[0] = c->d_qr;
@@ -266,7 +271,8 @@ int stage_match(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
 }
 
 int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
-    if (c->big() && src) return c->fail(HTTM_ERR_UNSUPPORTED, "blocks of more than 256 tokens are merged from the reordered copies");
+    if ((c->big() || sorted_filter(c)) && src)
+        return c->fail(HTTM_ERR_UNSUPPORTED, "this context merges from the reordered copies (blocks of more than 256 tokens, or outlier filtering with blocks of more than 32)");
     MergeArgs a{};
     if (src) {
         a.geom = c->d_geom;
@@ -294,7 +300,7 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.m_k = c->m_k;
     a.status = c->d_status;
     c->launches++;
-    if (c->big()) return check_cuda(c, launch_big_merge(a, s), "large-block merge launch");
+    if (c->big() || sorted_filter(c)) return check_cuda(c, launch_big_merge(a, s), "sorted-group merge launch");
     return check_cuda(c, launch_merge(a, c->max_block, c->sm_count, s), "merge launch");
 }
 
@@ -359,7 +365,7 @@ int stage_outlier(httm_ctx* c, const httm_tensor& q, cudaStream_t s) {
     a.status = c->d_status;
     int rc;
     if ((rc = check_cuda(c, cudaMemsetAsync(c->d_sel, 0, kSelWords * sizeof(int32_t), s), "selection state reset"))) return rc;
-    if (c->big()) {   // large blocks: the blocks are runs of rows of the reordered copy; six kernels
+    if (sorted_filter(c)) {   // the blocks are runs of rows of the reordered copy; six kernels
         a.src_q = view(c->d_qr, c->n_tokens);
         if ((rc = check_cuda(c, launch_big_deviation(a, s), "large-block deviation launch"))) return rc;
         if ((rc = check_cuda(c, launch_threshold0(a, c->sm_count, s), "threshold launch"))) return rc;
@@ -399,6 +405,14 @@ int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const h
         if ((rc = stage_big_scores(c, s))) return rc;
         if ((rc = stage_big_select(c, s))) return rc;
         if (c->filtering() && (rc = stage_outlier(c, q, s))) return rc;
+        if ((rc = stage_merge(c, s))) return rc;
+        if ((rc = stage_attention(c, s))) return rc;
+        return stage_unmerge(c, out, s);
+    }
+    if (sorted_filter(c)) {   // outlier filtering with blocks of 33 .. 256 tokens: everything from the reordered copies
+        if ((rc = stage_reorder(c, q, k, v, s))) return rc;
+        if ((rc = stage_match(c, s))) return rc;
+        if ((rc = stage_outlier(c, q, s))) return rc;
         if ((rc = stage_merge(c, s))) return rc;
         if ((rc = stage_attention(c, s))) return rc;
         return stage_unmerge(c, out, s);
@@ -603,9 +617,6 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
         c->outlier_fraction = 0.0;
         return HTTM_OK;
     }
-    if (c->max_block > 32 && !c->big())
-        return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering supports merging blocks of at most 32 tokens, or of more than 256");
-    if (!c->big() && !direct_mode(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "outlier filtering needs a scene of at most 32767 frames / patch rows / patch columns and at most 32 special tokens per frame");
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
     if (!c->d_eps) {

@@ -113,12 +113,6 @@ def test_switching_the_filter_off_restores_the_plain_path():
 
 
 def test_filter_argument_errors():
-    wl = synth.Workload("mid_blocks", 4, 8, 8, 4, 4, 4, 0.5, 0.5, heads=2)          # 64-token blocks: neither path
-    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
-        with pytest.raises(hb.HttmError) as e:
-            ctx.set_outlier_fraction(0.1)
-        assert e.value.code == hb.ERR_UNSUPPORTED
-        ctx.set_outlier_fraction(0.0)
     wl = synth.Workload("ok", 2, 8, 8, 2, 4, 4, 0.5, 0.5, heads=2)
     with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
         for bad in (-0.1, 1.5, float("nan")):
@@ -127,6 +121,24 @@ def test_filter_argument_errors():
             assert e.value.code == hb.ERR_INVALID_ARG
         with pytest.raises(hb.HttmError):
             ctx.launch_stage(hb.STAGE_OUTLIER_FILTER, *(hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(wl)))
+
+
+MID = [
+    # name, frames, grid_h, grid_w, blk, ratio_q, ratio_kv, n_camera, n_register, heads, gamma
+    ("blocks_64", 9, 10, 10, (4, 4, 4), 0.5, 0.9, 1, 4, 2, 0.05),
+    ("blocks_128_clipped", 4, 17, 19, (2, 8, 8), 0.7, 0.9, 1, 4, 2, 0.1),
+    ("blocks_256", 5, 9, 8, (4, 8, 8), 0.8, 0.3, 1, 4, 1, 0.03),
+    ("many_specials_32", 3, 6, 6, (2, 4, 4), 0.5, 0.5, 1, 44, 2, 0.1),        # 32-token blocks over the reordered copies
+]
+
+
+@pytest.mark.parametrize("case", MID, ids=[c[0] for c in MID])
+def test_mid_blocks_filtered(case):
+    """Blocks of 33 .. 256 tokens (and scenes that go over the reordered copies): reorder, match, deviation, three threshold
+    kernels, filter, offsets, merge, attention, unmerge."""
+    name, S, h, w, blk, rq, rkv, ncam, nreg, H, gamma = case
+    wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, n_camera=ncam, n_register=nreg, heads=H, seed=13)
+    run_filtered(wl, gamma, peaky=True, launches=11)
 
 
 def test_medium_config_filtered_full_size_sampled():
