@@ -3,7 +3,8 @@
 // warp's stage, and its similarity step (Eq. 1) is a real dense contraction: n tokens x n_dst dst tokens x 64.
 //
 //   big_scores_kernel   cosine of every token of a block with every dst token of the block on the 5th-generation
-//                       tensor cores (tcgen05.mma, accumulators in tensor memory), fused with the row-wise
+//                       tensor cores (tcgen05.mma, accumulators in tensor memory; the dst tokens enter scaled by
+//                       their inverse norms, split exactly into three bf16 planes), fused with the row-wise
 //                       arg-max: per token the best dst and the best cosine
 //   big_select_kernel   the r src tokens with the best cosines merge (Sec. 3.2): exact radix select per block,
 //                       ties by position; writes the assignment map
@@ -31,32 +32,45 @@ __device__ __forceinline__ bool is_dst_position(int j, int n_rule, int nd) {
 }
 
 // ------------------------------------------------------------------------------------------------ scores
+// cos(i, d) |x_i| = sum_k x_ik (w_d x_dk) with w_d = 1 / max(|x_d|, 1e-12).  The dst rows are multiplied by their
+// inverse norms when they are gathered, and the fp32 products are split EXACTLY into three bf16 planes (8 + 8 + 8
+// significant bits), so that three accumulating MMAs per K step give the scaled scores straight in tensor memory: the
+// arg-max warps neither load weights nor multiply (the tensor cores are idle most of the time in this kernel, the
+// arg-max warps are what bounds it).  The dst tokens of a block are taken 256 at a time (three planes of 32 KB); the
+// token tiles of the slice are streamed once per such chunk, and every token's best so far waits in shared memory.
 constexpr int TILE = 128;                        // rows of an operand tile
 constexpr int TILE_BYTES = TILE * kRowBytes;     // 16 KB
-constexpr int kDstTiles = kMaxBigDst / TILE;     // 8 resident dst tiles
-constexpr int kSrcTilesPerItem = kBigSliceRows / TILE;   // 8
+constexpr int kChunkDst = 256;                   // dst tokens per chunk = columns of a score buffer
+constexpr int kPlaneBytes = kChunkDst * kRowBytes;       // 32 KB
+constexpr int kSrcTilesPerItem = kBigSliceRows / TILE;   // 32: a work item is a whole block
 constexpr int SC_THREADS = 320;                  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: arg-max (two column halves x four lane quadrants)
-constexpr int SC_TMEM_COLS = 512;                // two score buffers of 256 columns (one token tile x two dst tiles)
+constexpr int SC_TMEM_COLS = 512;                // two score buffers of 256 columns
+constexpr int SC_STAGES = 2;                     // ring of token tiles
 
 struct ScoreBars {
-    uint64_t a_full[2], a_empty[2];   // ring of token tiles
+    uint64_t a_full[SC_STAGES], a_empty[SC_STAGES];   // ring of token tiles
     uint64_t s_full[2], s_empty[2];   // score buffers
     uint64_t x_full[2], x_done[2];    // exchange of the two column halves' results, by token-tile parity
     uint32_t tmem_base;
     int abort_flag;
 };
-constexpr int SC_OFF_A = kDstTiles * TILE_BYTES;                 // token tiles behind the dst tiles
-constexpr int SC_OFF_INV = SC_OFF_A + 2 * TILE_BYTES;            // float [1024] inverse norms of the dst tokens
-constexpr int SC_OFF_XCH = SC_OFF_INV + kMaxBigDst * 4;          // [2][128] (best, arg) of column half 1
+constexpr int SC_OFF_A = 3 * kPlaneBytes;                        // token tiles behind the three planes
+constexpr int SC_OFF_BEST = SC_OFF_A + SC_STAGES * TILE_BYTES;   // float2 [2 halves][1024 tokens]: (best, arg) so far
+constexpr int SC_OFF_XCH = SC_OFF_BEST + 2 * kBigSliceRows * 8;  // [2][128] (best, arg) of column half 1
 constexpr int SC_OFF_BARS = SC_OFF_XCH + 2 * TILE * 8;
 constexpr int SC_SMEM = SC_OFF_BARS + 256 + 1024 /*alignment slack*/;
+
+__device__ __forceinline__ uint32_t bf16_bits_rn(float f) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(f);
+    return (uint32_t)*reinterpret_cast<const unsigned short*>(&h);
+}
 
 __global__ void __launch_bounds__(SC_THREADS, 1)
 big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const BigMatchArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t s_b = tc::smem_addr(smem), s_a = s_b + SC_OFF_A;
-    float* inv_d = reinterpret_cast<float*>(smem + SC_OFF_INV);
+    float2* best_s = reinterpret_cast<float2*>(smem + SC_OFF_BEST);
     float2* xch = reinterpret_cast<float2*>(smem + SC_OFF_XCH);
     ScoreBars* bars = reinterpret_cast<ScoreBars*>(smem + SC_OFF_BARS);
     volatile int* abort_flag = &bars->abort_flag;
@@ -64,9 +78,11 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
     if (tid == 0) {
         bars->abort_flag = 0;
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < SC_STAGES; ++i) {
             tc::mbar_init(tc::smem_addr(&bars->a_full[i]), 1);
             tc::mbar_init(tc::smem_addr(&bars->a_empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
             tc::mbar_init(tc::smem_addr(&bars->s_full[i]), 1);
             tc::mbar_init(tc::smem_addr(&bars->s_empty[i]), 256);
             tc::mbar_init(tc::smem_addr(&bars->x_full[i]), 128);
@@ -82,16 +98,16 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
 
-    // completions so far of every barrier (each role counts its own): they give the phase parities across work items
-    uint32_t n_a[2] = {0, 0}, n_s[2] = {0, 0};   // token tiles per ring stage, score tiles per buffer
-    uint32_t n_x[2] = {0, 0};                    // exchanges per parity slot
+    // completions so far of every barrier (each role counts its own): they give the phase parities across chunks and items
+    uint32_t n_tiles_done = 0;   // token tiles so far: tile k uses ring stage k % SC_STAGES and score buffer k & 1
+    uint32_t n_x[2] = {0, 0};    // exchanges per parity slot
     const int64_t total = 2ll * a.heads * a.n_items;
-    constexpr uint32_t idesc = tc::idesc_bf16(128, 256, false, false);
-    constexpr uint64_t kTileStep = TILE_BYTES >> 4;   // descriptor address field counts 16-byte units
+    constexpr uint32_t idesc = tc::idesc_bf16(128, kChunkDst, false, false);
+    constexpr uint64_t kTileStep = TILE_BYTES >> 4, kPlaneStep = kPlaneBytes >> 4;   // descriptor address fields count 16-byte units
 
     for (int64_t item = blockIdx.x;; item += gridDim.x) {
-        __syncthreads();   // every role is done with the previous item: dst tiles and tables may be rewritten
-        if (item >= total || bars->abort_flag) break;   // (the flag is only set between two of these barriers: same answer in every thread)
+        __syncthreads();
+        if (item >= total || bars->abort_flag) break;   // (the flag is only set between two barriers: same answer in every thread)
         const int t = (int)(item / ((int64_t)a.heads * a.n_items));
         const int64_t rem = item - (int64_t)t * a.heads * a.n_items;
         const int h = (int)(rem / a.n_items);
@@ -99,107 +115,129 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const BlockInfo bi = a.blocks[it.block];
         const int n = bi.n, r = t == 0 ? bi.r_q : bi.r_k, nd = t == 0 ? bi.nd_q : bi.nd_k;
         if (r == 0) continue;   // nothing merges in this block (uniform)
-        const int n_dd = (nd + 2 * TILE - 1) / (2 * TILE);                        // pairs of dst tiles
+        const int n_chunks = (nd + kChunkDst - 1) / kChunkDst;
         const int n_st = min(kSrcTilesPerItem, (n - it.row0 + TILE - 1) / TILE);  // token tiles of this slice
         const int64_t head_row0 = (int64_t)h * a.n_tokens + bi.start;             // row of the block's first token in [H][N]
 
-        // ---- dst tokens of the block -> resident tiles (128-byte swizzle, as a tiled bulk copy would leave them)
-        {
-            const __nv_bfloat16* x = a.xr[t] + head_row0 * kHeadDim;
-            const float* inv = a.inv_norm[t] + head_row0;
-            const int chunk = tid & 7;
-            for (int d = tid >> 3; d < n_dd * 2 * TILE; d += SC_THREADS / 8) {
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);   // rows past the last dst token: zeros (their scores are masked)
-                float w = 0.f;
-                if (d < nd) {
-                    const int pos = dst_position(d, bi.n_rule, nd);
-                    v = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * kHeadDim) + chunk);
-                    w = __ldg(inv + pos);
-                }
-                const int row = d & (TILE - 1);
-                *reinterpret_cast<uint4*>(smem + (d >> 7) * TILE_BYTES + row * kRowBytes + ((chunk ^ (row & 7)) << 4)) = v;
-                if (chunk == 0) inv_d[d] = w;
+        for (int chunk = 0; chunk < n_chunks; ++chunk) {
+            const int d_lo = chunk * kChunkDst, d_cnt = min(kChunkDst, nd - d_lo);   // this chunk's dst tokens
+            if (chunk > 0) {
+                __syncthreads();   // every role is done with the previous chunk's planes
+                if (bars->abort_flag) break;   // (uniform, as above)
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor cores read these tiles through the async proxy
-        }
-        __syncthreads();
-
-        if (warp == 0) {
-            // ------------------------------------------------------------------ producer: token tiles of the slice
-            if (tc::elect_one()) {
-                for (int i = 0; i < n_st; ++i) {
-                    const int st = i & 1;
-                    if (!tc::mbar_wait(tc::smem_addr(&bars->a_empty[st]), (n_a[st] & 1u) ^ 1u, abort_flag)) break;
-                    const uint32_t bar = tc::smem_addr(&bars->a_full[st]);
-                    tc::mbar_expect_tx(bar, TILE_BYTES);
-                    // rows past the block's end belong to the next block (finite, results dropped) or are zero filled past N
-                    tc::tma_load_3d(s_a + st * TILE_BYTES, t == 0 ? &map_q : &map_k, bar, 0, bi.start + it.row0 + i * TILE, h);
-                    ++n_a[st];
-                }
-            } else {
-                for (int i = 0; i < n_st; ++i) ++n_a[i & 1];
-            }
-            __syncwarp();
-        } else if (warp == 1) {
-            // ------------------------------------------------------------------ issuer: S = X_tile . X_dst^T
-            if (tc::elect_one()) {
-                const uint64_t da0 = tc::smem_desc_sw128(s_a), db0 = tc::smem_desc_sw128(s_b);
-                bool ok = true;
-                auto issue = [&](uint32_t t_s, uint64_t da, uint64_t db, uint32_t bar) {   // four K = 16 steps over the 64 channels
-                    tc::mma_ss_c<false>(t_s, da, db, idesc);
-                    tc::mma_ss_c<true>(t_s, da + 2, db + 2, idesc);
-                    tc::mma_ss_c<true>(t_s, da + 4, db + 4, idesc);
-                    tc::mma_ss_c<true>(t_s, da + 6, db + 6, idesc);
-                    tc::mma_commit(bar);
-                };
-                for (int i = 0; ok && i < n_st; ++i) {
-                    const int st = i & 1;
-                    ok = tc::mbar_wait(tc::smem_addr(&bars->a_full[st]), n_a[st] & 1u, abort_flag);
-                    if (!ok) break;
-                    tc::fence_after_sync();
+            // ---- dst tokens of the chunk, scaled and split, -> three resident planes (128-byte swizzle, as a tiled bulk
+            //      copy would leave them)
+            {
+                const __nv_bfloat16* x = a.xr[t] + head_row0 * kHeadDim;
+                const float* inv = a.inv_norm[t] + head_row0;
+                const int c16 = tid & 7;
+                constexpr int kRowsPerPass = SC_THREADS / 8, kPasses = (kChunkDst + kRowsPerPass - 1) / kRowsPerPass;
+                uint4 v[kPasses];   // all of this thread's loads are issued before the first is used
+                float w[kPasses];
 #pragma unroll
-                    for (int jj = 0; jj < kDstTiles / 2; ++jj) {   // buffer jj & 1: operands are bases plus constants
-                        if (jj < n_dd) {
-                            const int b = jj & 1;
-                            ok = ok && tc::mbar_wait(tc::smem_addr(&bars->s_empty[b]), (n_s[b] & 1u) ^ 1u, abort_flag);
-                            if (ok) {
-                                tc::fence_after_sync();
-                                issue(tmem + b * 256, da0 + (uint64_t)st * kTileStep, db0 + (uint64_t)(2 * jj) * kTileStep,
-                                      tc::smem_addr(&bars->s_full[b]));
-                                ++n_s[b];
-                            }
-                        }
+                for (int u = 0; u < kPasses; ++u) {
+                    const int dl = (tid >> 3) + u * kRowsPerPass;
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    w[u] = 0.f;
+                    if (dl < d_cnt) {
+                        const int pos = dst_position(d_lo + dl, bi.n_rule, nd);
+                        v[u] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * kHeadDim) + c16);
+                        w[u] = __ldg(inv + pos);
                     }
-                    if (ok) tc::mma_commit(tc::smem_addr(&bars->a_empty[st]));   // the tile may be refilled when these MMAs are done
-                    ++n_a[st];
                 }
-            } else {
-                for (int i = 0; i < n_st; ++i) {
-                    ++n_a[i & 1];
-                    for (int jj = 0; jj < n_dd; ++jj) ++n_s[jj & 1];
+#pragma unroll
+                for (int u = 0; u < kPasses; ++u) {
+                    const int dl = (tid >> 3) + u * kRowsPerPass;
+                    if (dl >= kChunkDst) continue;
+                    // rows past the last dst token come out as zeros (x = 0, w = 0); their columns are masked below
+                    const uint32_t in[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    uint32_t o0[4], o1[4], o2[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t b0[2], b1[2], b2[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float xv = __uint_as_float(e == 0 ? in[q] << 16 : in[q] & 0xffff0000u);
+                            const float p = xv * w[u];                                // one rounding to fp32 (24 bits)
+                            b0[e] = bf16_bits_rn(p);
+                            const float r1 = p - __uint_as_float(b0[e] << 16);        // exact
+                            b1[e] = bf16_bits_rn(r1);
+                            const float r2 = r1 - __uint_as_float(b1[e] << 16);       // exact, at most 8 significant bits
+                            b2[e] = bf16_bits_rn(r2);
+                        }
+                        o0[q] = b0[0] | (b0[1] << 16);
+                        o1[q] = b1[0] | (b1[1] << 16);
+                        o2[q] = b2[0] | (b2[1] << 16);
+                    }
+                    unsigned char* dst = smem + dl * kRowBytes + ((c16 ^ (dl & 7)) << 4);
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(o0[0], o0[1], o0[2], o0[3]);
+                    *reinterpret_cast<uint4*>(dst + kPlaneBytes) = make_uint4(o1[0], o1[1], o1[2], o1[3]);
+                    *reinterpret_cast<uint4*>(dst + 2 * kPlaneBytes) = make_uint4(o2[0], o2[1], o2[2], o2[3]);
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor cores read the planes through the async proxy
             }
-            __syncwarp();
-        } else {
-            // ------------------------------------------------------------------ arg-max over the dst tokens, one thread per token and column half
-            const int half = (warp - 2) >> 2;                  // 0: dst tile 2 jj, 1: dst tile 2 jj + 1
-            const int row = (warp & 3) * 32 + lane;            // row of the token tile = lane of tensor memory
-            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-            bool ok = true;
-            for (int i = 0; ok && i < n_st; ++i) {
-                float best = -INFINITY;
-                int arg = 0;
-                for (int jj = 0; ok && jj < n_dd; ++jj) {
-                    const int b = jj & 1;
-                    ok = tc::mbar_wait(tc::smem_addr(&bars->s_full[b]), n_s[b] & 1u, abort_flag);
+            __syncthreads();
+
+            if (warp == 0) {
+                // -------------------------------------------------------------- producer: the token tiles of the slice, once per chunk
+                if (tc::elect_one()) {
+                    for (int i = 0; i < n_st; ++i) {
+                        const uint32_t k = n_tiles_done + i, st = k % SC_STAGES, ph = (k / SC_STAGES) & 1u;
+                        if (!tc::mbar_wait(tc::smem_addr(&bars->a_empty[st]), ph ^ 1u, abort_flag)) break;
+                        const uint32_t bar = tc::smem_addr(&bars->a_full[st]);
+                        tc::mbar_expect_tx(bar, TILE_BYTES);
+                        // rows past the block's end belong to the next block (finite, results dropped) or are zero filled past N
+                        tc::tma_load_3d(s_a + st * TILE_BYTES, t == 0 ? &map_q : &map_k, bar, 0, bi.start + it.row0 + i * TILE, h);
+                    }
+                }
+                __syncwarp();
+            } else if (warp == 1) {
+                // -------------------------------------------------------------- issuer: S = X_tile . (hi + mid + lo)^T
+                if (tc::elect_one()) {
+                    const uint64_t da0 = tc::smem_desc_sw128(s_a), db0 = tc::smem_desc_sw128(s_b);
+                    bool ok = true;
+                    for (int i = 0; ok && i < n_st; ++i) {
+                        const uint32_t k = n_tiles_done + i, st = k % SC_STAGES, b = k & 1u;
+                        ok = tc::mbar_wait(tc::smem_addr(&bars->a_full[st]), (k / SC_STAGES) & 1u, abort_flag) &&
+                             tc::mbar_wait(tc::smem_addr(&bars->s_empty[b]), ((k >> 1) & 1u) ^ 1u, abort_flag);
+                        if (!ok) break;
+                        tc::fence_after_sync();
+                        const uint64_t da = da0 + (uint64_t)st * kTileStep;
+#pragma unroll
+                        for (int pl = 0; pl < 3; ++pl)
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)   // K = 16 steps over the 64 channels: 32 bytes = 2 descriptor units
+                                tc::mma_ss(tmem + b * kChunkDst, da + 2 * ks, db0 + (uint64_t)pl * kPlaneStep + 2 * ks, idesc, (pl | ks) ? 1u : 0u);
+                        tc::mma_commit(tc::smem_addr(&bars->a_empty[st]));   // the tile may be refilled when these MMAs are done
+                        tc::mma_commit(tc::smem_addr(&bars->s_full[b]));
+                    }
+                }
+                __syncwarp();
+            } else {
+                // -------------------------------------------------------------- arg-max over the chunk's dst tokens, one thread per
+                // token and column half; the scores arrive scaled
+                const int half = (warp - 2) >> 2;
+                const int row = (warp & 3) * 32 + lane;            // row of the token tile = lane of tensor memory
+                const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+                const bool last_chunk = chunk == n_chunks - 1;
+                bool ok = true;
+                for (int i = 0; ok && i < n_st; ++i) {
+                    const uint32_t k = n_tiles_done + i, b = k & 1u;
+                    float2* mine = best_s + half * kBigSliceRows + i * TILE + row;
+                    float best = -INFINITY;
+                    int arg = 0;
+                    if (chunk > 0) {
+                        const float2 prev = *mine;
+                        best = prev.x;
+                        arg = __float_as_int(prev.y);
+                    }
+                    ok = tc::mbar_wait(tc::smem_addr(&bars->s_full[b]), (k >> 1) & 1u, abort_flag);
                     if (!ok) break;
                     tc::fence_after_sync();
-                    ++n_s[b];
-                    const int col0 = (2 * jj + half) * TILE;   // first dst of this thread's 128 columns
 #pragma unroll
                     for (int part = 0; part < 2; ++part) {
                         uint32_t raw[64];
-                        const uint32_t taddr = tmem + b * 256 + half * TILE + part * 64 + lane_addr;
+                        const uint32_t taddr = tmem + b * kChunkDst + half * TILE + part * 64 + lane_addr;
                         tc::tmem_ld32(taddr, raw);
                         tc::tmem_ld32(taddr + 32, raw + 32);
                         tc::tmem_wait_ld();
@@ -207,64 +245,64 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             tc::fence_before_sync();
                             tc::mbar_arrive(tc::smem_addr(&bars->s_empty[b]));
                         }
-                        const int c0 = col0 + part * 64;
-                        if (c0 < nd) {     // (uniform in the warp)
-                            const float4* w4 = reinterpret_cast<const float4*>(inv_d + c0);
-                            float v[64];
-                            float m = -INFINITY;
-#pragma unroll
-                            for (int q = 0; q < 16; ++q) {
-                                const float4 w = w4[q];
-                                v[4 * q + 0] = __uint_as_float(raw[4 * q + 0]) * w.x;
-                                v[4 * q + 1] = __uint_as_float(raw[4 * q + 1]) * w.y;
-                                v[4 * q + 2] = __uint_as_float(raw[4 * q + 2]) * w.z;
-                                v[4 * q + 3] = __uint_as_float(raw[4 * q + 3]) * w.w;
-                            }
-                            if (c0 + 64 > nd) {   // the block's last dst tokens: mask the columns behind them
+                        const int c0 = half * TILE + part * 64;   // first column of these 64 inside the chunk
+                        if (c0 < d_cnt) {                         // (uniform in the warp)
+                            if (c0 + 64 > d_cnt) {                // the block's last dst tokens: mask the columns behind them
 #pragma unroll
                                 for (int c = 0; c < 64; ++c)
-                                    if (c0 + c >= nd) v[c] = -INFINITY;
+                                    if (c0 + c >= d_cnt) raw[c] = 0xff800000u;   // -inf
                             }
+                            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;   // four independent chains
 #pragma unroll
-                            for (int c = 0; c < 64; c += 2) m = tc::fmax3(m, v[c], v[c + 1]);
-                            if (m > best) {   // rare after the first tiles: find the first column holding the maximum
+                            for (int c = 0; c < 64; c += 8) {
+                                m0 = tc::fmax3(m0, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+                                m1 = tc::fmax3(m1, __uint_as_float(raw[c + 2]), __uint_as_float(raw[c + 3]));
+                                m2 = tc::fmax3(m2, __uint_as_float(raw[c + 4]), __uint_as_float(raw[c + 5]));
+                                m3 = tc::fmax3(m3, __uint_as_float(raw[c + 6]), __uint_as_float(raw[c + 7]));
+                            }
+                            const float m = fmaxf(tc::fmax3(m0, m1, m2), m3);
+                            if (m > best) {   // find the first column holding the maximum (ties: lowest dst)
                                 best = m;
                                 int first = 63;
 #pragma unroll
                                 for (int c = 62; c >= 0; --c)
-                                    if (v[c] == m) first = c;
-                                arg = c0 + first;
+                                    if (__uint_as_float(raw[c]) == m) first = c;
+                                arg = d_lo + c0 + first;
                             }
                         }
                     }
-                }
-                if (!ok) break;
-                // the two column halves of a token meet: half 1 hands (best, arg) over, half 0 decides (ties: lowest dst)
-                const int slot = i & 1;
-                if (half == 1) {
-                    ok = tc::mbar_wait(tc::smem_addr(&bars->x_done[slot]), (n_x[slot] & 1u) ^ 1u, abort_flag);
-                    if (!ok) break;
-                    xch[slot * TILE + row] = make_float2(best, __int_as_float(arg));
-                    tc::mbar_arrive(tc::smem_addr(&bars->x_full[slot]));
-                } else {
-                    ok = tc::mbar_wait(tc::smem_addr(&bars->x_full[slot]), n_x[slot] & 1u, abort_flag);
-                    if (!ok) break;
-                    const float2 o = xch[slot * TILE + row];
-                    tc::mbar_arrive(tc::smem_addr(&bars->x_done[slot]));
-                    const int oarg = __float_as_int(o.y);
-                    if (o.x > best || (o.x == best && oarg < arg)) {
-                        best = o.x;
-                        arg = oarg;
+                    if (!last_chunk) {
+                        *mine = make_float2(best, __int_as_float(arg));
+                        continue;
                     }
-                    const int p = it.row0 + i * TILE + row;   // token number inside the block
-                    if (p < n) {
-                        const float w = __ldg(a.inv_norm[t] + head_row0 + p);
-                        a.best_key[t][head_row0 + p] = score_key(best * w);
-                        a.best_pos[t][head_row0 + p] = dst_position(arg, bi.n_rule, nd);
+                    // the two column halves of a token meet: half 1 hands (best, arg) over, half 0 decides (ties: lowest dst)
+                    const int slot = i & 1;
+                    if (half == 1) {
+                        ok = tc::mbar_wait(tc::smem_addr(&bars->x_done[slot]), (n_x[slot] & 1u) ^ 1u, abort_flag);
+                        if (!ok) break;
+                        xch[slot * TILE + row] = make_float2(best, __int_as_float(arg));
+                        tc::mbar_arrive(tc::smem_addr(&bars->x_full[slot]));
+                    } else {
+                        ok = tc::mbar_wait(tc::smem_addr(&bars->x_full[slot]), n_x[slot] & 1u, abort_flag);
+                        if (!ok) break;
+                        const float2 o = xch[slot * TILE + row];
+                        tc::mbar_arrive(tc::smem_addr(&bars->x_done[slot]));
+                        const int oarg = __float_as_int(o.y);
+                        if (o.x > best || (o.x == best && oarg < arg)) {
+                            best = o.x;
+                            arg = oarg;
+                        }
+                        const int p = it.row0 + i * TILE + row;   // token number inside the block
+                        if (p < n) {
+                            const float w = __ldg(a.inv_norm[t] + head_row0 + p);
+                            a.best_key[t][head_row0 + p] = score_key(best * w);
+                            a.best_pos[t][head_row0 + p] = dst_position(arg, bi.n_rule, nd);
+                        }
                     }
+                    ++n_x[slot];
                 }
-                ++n_x[slot];
             }
+            n_tiles_done += n_st;   // (every thread keeps the count, whatever its role)
         }
     }
     tc::fence_before_sync();

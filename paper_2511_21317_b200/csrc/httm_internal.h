@@ -12,7 +12,7 @@ constexpr int kRowBytes = kHeadDim * 2;  // one token of one head, bf16
 constexpr int kMaxBlockTokens = 256;  // largest merging block the warp-per-block match / merge kernels stage
 constexpr int kMaxBigBlockTokens = 4096;   // largest merging block of the large-block path (Sec. 4.1: 128 tokens x 30 frames = 3840)
 constexpr int kMaxBigDst = 1024;           // its dst tokens (a quarter of the block) stay in shared memory
-constexpr int kBigSliceRows = 1024;        // rows of a block one work item of the score kernel handles
+constexpr int kBigSliceRows = 4096;        // rows of a block one work item of the score kernel handles (the whole block)
 
 // Device status word values (first error wins).
 enum : int {
