@@ -45,7 +45,7 @@ constexpr int kPlaneBytes = kChunkDst * kRowBytes;       // 32 KB
 constexpr int kSrcTilesPerItem = kBigSliceRows / TILE;   // 32: a work item is a whole block
 constexpr int SC_THREADS = 320;                  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: arg-max (two column halves x four lane quadrants)
 constexpr int SC_TMEM_COLS = 512;                // two score buffers of 256 columns
-constexpr int SC_STAGES = 2;                     // ring of token tiles
+constexpr int SC_STAGES = 4;                     // ring of token tiles: a tile's load takes longer than its MMAs and its arg-max
 
 struct ScoreBars {
     uint64_t a_full[SC_STAGES], a_empty[SC_STAGES];   // ring of token tiles
@@ -55,8 +55,9 @@ struct ScoreBars {
     int abort_flag;
 };
 constexpr int SC_OFF_A = 3 * kPlaneBytes;                        // token tiles behind the three planes
-constexpr int SC_OFF_BEST = SC_OFF_A + SC_STAGES * TILE_BYTES;   // float2 [2 halves][1024 tokens]: (best, arg) so far
-constexpr int SC_OFF_XCH = SC_OFF_BEST + 2 * kBigSliceRows * 8;  // [2][128] (best, arg) of column half 1
+constexpr int SC_OFF_BEST = SC_OFF_A + SC_STAGES * TILE_BYTES;   // float [2 halves][tokens of the item]: best score so far
+constexpr int SC_OFF_ARG = SC_OFF_BEST + 2 * kBigSliceRows * 4;  // uint16 [2][tokens]: its dst (n_dst <= 1024)
+constexpr int SC_OFF_XCH = SC_OFF_ARG + 2 * kBigSliceRows * 2;   // [2][128] (best, arg) of column half 1
 constexpr int SC_OFF_BARS = SC_OFF_XCH + 2 * TILE * 8;
 constexpr int SC_SMEM = SC_OFF_BARS + 256 + 1024 /*alignment slack*/;
 
@@ -70,7 +71,8 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t s_b = tc::smem_addr(smem), s_a = s_b + SC_OFF_A;
-    float2* best_s = reinterpret_cast<float2*>(smem + SC_OFF_BEST);
+    float* best_s = reinterpret_cast<float*>(smem + SC_OFF_BEST);
+    uint16_t* arg_s = reinterpret_cast<uint16_t*>(smem + SC_OFF_ARG);
     float2* xch = reinterpret_cast<float2*>(smem + SC_OFF_XCH);
     ScoreBars* bars = reinterpret_cast<ScoreBars*>(smem + SC_OFF_BARS);
     volatile int* abort_flag = &bars->abort_flag;
@@ -223,13 +225,12 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 bool ok = true;
                 for (int i = 0; ok && i < n_st; ++i) {
                     const uint32_t k = n_tiles_done + i, b = k & 1u;
-                    float2* mine = best_s + half * kBigSliceRows + i * TILE + row;
+                    const int mine = half * kBigSliceRows + i * TILE + row;
                     float best = -INFINITY;
                     int arg = 0;
                     if (chunk > 0) {
-                        const float2 prev = *mine;
-                        best = prev.x;
-                        arg = __float_as_int(prev.y);
+                        best = best_s[mine];
+                        arg = arg_s[mine];
                     }
                     ok = tc::mbar_wait(tc::smem_addr(&bars->s_full[b]), (k >> 1) & 1u, abort_flag);
                     if (!ok) break;
@@ -252,27 +253,33 @@ big_scores_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                 for (int c = 0; c < 64; ++c)
                                     if (c0 + c >= d_cnt) raw[c] = 0xff800000u;   // -inf
                             }
-                            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;   // four independent chains
+                            // maxima of the four groups of 16 columns (independent chains), then of the part
+                            float g0 = -INFINITY, g1 = -INFINITY, g2 = -INFINITY, g3 = -INFINITY;
 #pragma unroll
-                            for (int c = 0; c < 64; c += 8) {
-                                m0 = tc::fmax3(m0, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
-                                m1 = tc::fmax3(m1, __uint_as_float(raw[c + 2]), __uint_as_float(raw[c + 3]));
-                                m2 = tc::fmax3(m2, __uint_as_float(raw[c + 4]), __uint_as_float(raw[c + 5]));
-                                m3 = tc::fmax3(m3, __uint_as_float(raw[c + 6]), __uint_as_float(raw[c + 7]));
+                            for (int c = 0; c < 16; c += 2) {
+                                g0 = tc::fmax3(g0, __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+                                g1 = tc::fmax3(g1, __uint_as_float(raw[16 + c]), __uint_as_float(raw[17 + c]));
+                                g2 = tc::fmax3(g2, __uint_as_float(raw[32 + c]), __uint_as_float(raw[33 + c]));
+                                g3 = tc::fmax3(g3, __uint_as_float(raw[48 + c]), __uint_as_float(raw[49 + c]));
                             }
-                            const float m = fmaxf(tc::fmax3(m0, m1, m2), m3);
-                            if (m > best) {   // find the first column holding the maximum (ties: lowest dst)
-                                best = m;
-                                int first = 63;
+                            const float m = fmaxf(tc::fmax3(g0, g1, g2), g3);
+                            if (m > best) {   // find the first column holding the maximum (ties: lowest dst): first group, then
+                                best = m;     // the first of its 16 columns (the search runs whenever any row of the warp improves)
+                                const bool in0 = g0 == m, in1 = g1 == m, in2 = g2 == m;
+                                const int group = in0 ? 0 : (in1 ? 1 : (in2 ? 2 : 3));
+                                int first = 15;
 #pragma unroll
-                                for (int c = 62; c >= 0; --c)
-                                    if (__uint_as_float(raw[c]) == m) first = c;
-                                arg = d_lo + c0 + first;
+                                for (int c = 14; c >= 0; --c) {
+                                    const uint32_t v = in0 ? raw[c] : (in1 ? raw[16 + c] : (in2 ? raw[32 + c] : raw[48 + c]));
+                                    if (__uint_as_float(v) == m) first = c;
+                                }
+                                arg = d_lo + c0 + 16 * group + first;
                             }
                         }
                     }
                     if (!last_chunk) {
-                        *mine = make_float2(best, __int_as_float(arg));
+                        best_s[mine] = best;
+                        arg_s[mine] = (uint16_t)arg;
                         continue;
                     }
                     // the two column halves of a token meet: half 1 hands (best, arg) over, half 0 decides (ties: lowest dst)
