@@ -712,24 +712,33 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_deviation_kernel(const Outl
 #pragma unroll
             for (int e = 0; e < 8; ++e) mean[e] = ((acc[0][e] + acc[1][e]) + (acc[2][e] + acc[3][e])) * inv;   // kept in fp32
         }
-        // (the eight lanes of a group walk its members together: the trip count is the same in all of them)
-        for (int i = i0; i < i1; ++i) {
-            const int pos = (int)(keys[i] & 4095u);
-            float d2 = 0.f;
-            if (cnt >= 2) {
+        // (the eight lanes of a group walk its members together: the trip count is the same in all of them); four members
+        // at a time, so that four loads are in flight
+        const unsigned group_mask = 0xffu << (8 * sub);
+        for (int i = i0; i < i1; i += 4) {
+            uint4 v[4];
+            int pos[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                pos[u] = i + u < i1 ? (int)(keys[i + u] & 4095u) : -1;
+                v[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (cnt >= 2 && pos[u] >= 0) v[u] = __ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos[u] * st) + ch);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
                 float f[8];
-                unpack8f(__ldg(reinterpret_cast<const uint4*>(x + (int64_t)pos * st) + ch), f);
+                unpack8f(v[u], f);
+                float d2 = 0.f;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const float d = f[e] - mean[e];
                     d2 = fmaf(d, d, d2);
                 }
+                d2 += __shfl_xor_sync(group_mask, d2, 1);
+                d2 += __shfl_xor_sync(group_mask, d2, 2);
+                d2 += __shfl_xor_sync(group_mask, d2, 4);
+                if (ch == 0 && pos[u] >= 0) eps[pos[u]] = cnt >= 2 ? sqrtf(d2) : 0.f;
             }
-            const unsigned group_mask = 0xffu << (8 * sub);
-            d2 += __shfl_xor_sync(group_mask, d2, 1);
-            d2 += __shfl_xor_sync(group_mask, d2, 2);
-            d2 += __shfl_xor_sync(group_mask, d2, 4);
-            if (ch == 0) eps[pos] = cnt >= 2 ? sqrtf(d2) : 0.f;
         }
     }
 }
