@@ -300,7 +300,7 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.m_k = c->m_k;
     a.status = c->d_status;
     c->launches++;
-    if (c->big() || sorted_filter(c)) return check_cuda(c, launch_big_merge(a, s), "sorted-group merge launch");
+    if (c->big() || sorted_filter(c)) return check_cuda(c, launch_big_merge(a, c->max_block, s), "sorted-group merge launch");
     return check_cuda(c, launch_merge(a, c->max_block, c->sm_count, s), "merge launch");
 }
 
@@ -367,9 +367,9 @@ int stage_outlier(httm_ctx* c, const httm_tensor& q, cudaStream_t s) {
     if ((rc = check_cuda(c, cudaMemsetAsync(c->d_sel, 0, kSelWords * sizeof(int32_t), s), "selection state reset"))) return rc;
     if (sorted_filter(c)) {   // the blocks are runs of rows of the reordered copy; six kernels
         a.src_q = view(c->d_qr, c->n_tokens);
-        if ((rc = check_cuda(c, launch_big_deviation(a, s), "large-block deviation launch"))) return rc;
+        if ((rc = check_cuda(c, launch_big_deviation(a, c->max_block, s), "large-block deviation launch"))) return rc;
         if ((rc = check_cuda(c, launch_threshold0(a, c->sm_count, s), "threshold launch"))) return rc;
-        if ((rc = check_cuda(c, launch_big_filter(a, s), "large-block filter launch"))) return rc;
+        if ((rc = check_cuda(c, launch_big_filter(a, c->max_block, s), "large-block filter launch"))) return rc;
         c->launches += 6;
         return check_cuda(c, launch_offsets(a, s), "offsets launch");
     }

@@ -454,8 +454,11 @@ __global__ void __launch_bounds__(SEL_THREADS, 1) big_select_kernel(const BigMat
 
 // ------------------------------------------------------------------------------------------------ merging
 // One CTA per (map in {Q, K}, head, block) - the K map also merges V - plus CTAs that copy the special tokens.
-constexpr int MG_THREADS = 1024;
-constexpr int MG_SMEM = kMaxBigBlockTokens * 4 /*keys*/ + kMaxBigBlockTokens * 2 /*row of kept token*/ + (kMaxBigBlockTokens + 4) * 4 /*segments*/ + 256;
+// The sorted-group kernels are templated on T, the threads of a CTA; a CTA holds one block of up to 4 T tokens (thread i
+// owns tokens 4 i .. 4 i + 3).  T is chosen from the largest block of the context: 1024 for blocks of 4096 tokens, 64 for
+// blocks of up to 256, so that small blocks get many small CTAs per SM.
+__host__ __device__ constexpr int mg_smem_bytes(int T) { return 4 * T * 4 /*keys*/ + 4 * T * 2 /*row of kept token*/ + (4 * T + 4) * 4 /*segments*/ + 256; }
+__host__ __device__ constexpr int of_smem_bytes(int T) { return mg_smem_bytes(T) + 4 * T * 2 /*position of every row's kept token*/ + 4 * T /*outlier flags*/ + 4 * T * 2 /*new representative of every row*/; }
 
 __device__ __forceinline__ void unpack8f(const uint4& raw, float* f) {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -470,12 +473,13 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// The groups of one block from its map A (every thread of a 1024-thread CTA calls this): merged row of every kept token =
+// The groups of one block from its map A (every thread of the T-thread CTA calls this): merged row of every kept token =
 // its rank among the kept tokens in position order (row_of; -1 for merged tokens); all tokens sorted by (merged row,
 // position) in keys[] = (row << 12) | position, so that the members of a row are one ascending run; seg[row] = first
 // sorted index of the row, seg[n_kept] = n.  rep_of_row (optional) gets the position of every row's kept token; rank_out
 // (optional) the merged row of every token plus moff.  Returns the number of kept tokens, at most `limit` (tokens whose
 // row would lie beyond it, or whose target is not a kept token, are recorded as a corrupt map and left out).
+template <int T>
 __device__ int build_groups(const int32_t* A, int block_start, int n, int limit, uint32_t* keys, int16_t* row_of, int* seg, int* warp_sum,
                             int16_t* rep_of_row, int32_t* status, int32_t* rank_out, int moff) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -504,16 +508,16 @@ __device__ int build_groups(const int32_t* A, int block_start, int n, int limit,
     if (lane == 31) warp_sum[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-        int w = warp_sum[lane];
+        int w = lane < T / 32 ? warp_sum[lane] : 0;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const int o = __shfl_up_sync(0xffffffffu, w, off);
             if (lane >= off) w += o;
         }
-        warp_sum[lane] = w;
+        if (lane < T / 32) warp_sum[lane] = w;
     }
     __syncthreads();
-    const int n_kept = min(warp_sum[31], limit);
+    const int n_kept = min(warp_sum[T / 32 - 1], limit);
     int next_row = (warp > 0 ? warp_sum[warp - 1] : 0) + incl - kept;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -528,7 +532,7 @@ __device__ int build_groups(const int32_t* A, int block_start, int n, int limit,
         }
     }
     __syncthreads();
-    int P = 512;
+    int P = 32;
     while (P < n) P <<= 1;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -549,7 +553,7 @@ __device__ int build_groups(const int32_t* A, int block_start, int n, int limit,
     __syncthreads();
     for (int k = 2; k <= P; k <<= 1) {   // bitonic sort: the keys are distinct, so the order is unique
         for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            for (int i = tid; i < P; i += MG_THREADS) {
+            for (int i = tid; i < P; i += T) {
                 const int ixj = i ^ jj;
                 if (ixj > i) {
                     const uint32_t x = keys[i], y = keys[ixj];
@@ -562,7 +566,7 @@ __device__ int build_groups(const int32_t* A, int block_start, int n, int limit,
             __syncthreads();
         }
     }
-    for (int i = tid; i <= n; i += MG_THREADS) {
+    for (int i = tid; i <= n; i += T) {
         const int row = i < n ? (int)(keys[i] >> 12) : n_kept;
         const int prev = i > 0 ? (int)(keys[i - 1] >> 12) : -1;
         if (row != prev && prev < n_kept)   // every row from prev + 1 to row starts here (rows without members cannot occur in a valid map)
@@ -572,19 +576,20 @@ __device__ int build_groups(const int32_t* A, int block_start, int n, int limit,
     return n_kept;
 }
 
-__global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArgs a, int sp_chunks) {
+template <int T>
+__global__ void __launch_bounds__(T, 1) big_merge_kernel(const MergeArgs a, int sp_chunks) {
     extern __shared__ __align__(16) unsigned char mg_smem[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);                                     // [P] (merged row << 12) | position
-    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + kMaxBigBlockTokens * 4);            // [n] merged row of a kept token, -1
-    int* seg = reinterpret_cast<int*>(mg_smem + kMaxBigBlockTokens * 6);                       // [n_kept + 1] first sorted index of every merged row
-    int* warp_sum = seg + kMaxBigBlockTokens + 4;                                              // [32]
+    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + (4 * T) * 4);            // [n] merged row of a kept token, -1
+    int* seg = reinterpret_cast<int*>(mg_smem + (4 * T) * 6);                       // [n_kept + 1] first sorted index of every merged row
+    int* warp_sum = seg + (4 * T) + 4;                                              // [32]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_block_ctas = 2 * a.heads * a.n_blocks;
     const int ch = lane & 7, sub = lane >> 3;   // 16-byte chunk of a row; which of four rows in flight
 
     if ((int)blockIdx.x >= n_block_ctas) {
-        // special tokens: never merged, first in the merged order; 128 rows of one head per CTA, all three tensors
-        const int idx = blockIdx.x - n_block_ctas, h = idx / sp_chunks, row = (idx % sp_chunks) * 128 + (tid >> 3);
+        // special tokens: never merged, first in the merged order; T / 8 rows of one head per CTA, all three tensors
+        const int idx = blockIdx.x - n_block_ctas, h = idx / sp_chunks, row = (idx % sp_chunks) * (T / 8) + (tid >> 3);
         if (row < a.n_special_total) {
             for (int t = 0; t < 3; ++t) {
                 const int m_len = t == 0 ? a.m_q : a.m_k;
@@ -604,7 +609,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArg
     const int64_t base = (int64_t)h * a.n_tokens + bi.start;
     const int32_t* A = a.assign[m] + base;
 
-    const int n_kept = build_groups(A, bi.start, n, limit, keys, row_of, seg, warp_sum, nullptr, a.status, m == 0 ? a.rank_q + base : nullptr, moff);
+    const int n_kept = build_groups<T>(A, bi.start, n, limit, keys, row_of, seg, warp_sum, nullptr, a.status, m == 0 ? a.rank_q + base : nullptr, moff);
     // eight lanes per merged row (a lane owns one 16-byte chunk of the row), four rows per warp at a time, four
     // members of a row in flight: the gather is bound by load latency, so it needs many loads in the air.  Member
     // i of a row goes to accumulator i mod 4; the four are added in a fixed order: the result does not depend on
@@ -612,7 +617,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArg
     for (int t = (m == 0 ? 0 : 1); t <= (m == 0 ? 0 : 2); ++t) {
         const __nv_bfloat16* x = a.xr[t] + base * kHeadDim;
         __nv_bfloat16* out = a.merged[t] + ((int64_t)h * m_len + moff) * kHeadDim;
-        for (int row = warp * 4 + sub; row < n_kept; row += (MG_THREADS / 32) * 4) {
+        for (int row = warp * 4 + sub; row < n_kept; row += (T / 32) * 4) {
             const int i0 = seg[row], i1 = seg[row + 1];
             float acc[4][8];
 #pragma unroll
@@ -655,16 +660,15 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_merge_kernel(const MergeArg
 // every query token from the mean of its group, one threshold over all heads (the refinement kernels of the small-block
 // path, which work on the array of deviations), outliers leave their groups - on the sorted group structure of the merge
 // kernel.  One CTA per (head, block).
-constexpr int OF_SMEM = MG_SMEM + kMaxBigBlockTokens * 2 /*position of every row's kept token*/ + kMaxBigBlockTokens /*outlier flags*/ +
-                        kMaxBigBlockTokens * 2 /*new representative of every row*/;
 
 // eps[h][p] = || q_p - mean of the group p was merged into ||_2 in fp32; 0 for a token on its own
-__global__ void __launch_bounds__(MG_THREADS, 1) big_deviation_kernel(const OutlierArgs a) {
+template <int T>
+__global__ void __launch_bounds__(T, 1) big_deviation_kernel(const OutlierArgs a) {
     extern __shared__ __align__(16) unsigned char mg_smem[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);
-    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + kMaxBigBlockTokens * 4);
-    int* seg = reinterpret_cast<int*>(mg_smem + kMaxBigBlockTokens * 6);
-    int* warp_sum = seg + kMaxBigBlockTokens + 4;
+    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + (4 * T) * 4);
+    int* seg = reinterpret_cast<int*>(mg_smem + (4 * T) * 6);
+    int* warp_sum = seg + (4 * T) + 4;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ch = lane & 7, sub = lane >> 3;
     const int h = blockIdx.x / a.n_blocks, b = blockIdx.x % a.n_blocks;
@@ -673,14 +677,14 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_deviation_kernel(const Outl
     const int64_t base = (int64_t)h * a.n_tokens + bi.start;
     float* eps = a.eps + base;
     if (bi.r_q == 0) {   // nothing merged in this block (uniform)
-        for (int j = tid; j < n; j += MG_THREADS) eps[j] = 0.f;
+        for (int j = tid; j < n; j += T) eps[j] = 0.f;
         return;
     }
-    const int n_kept = build_groups(a.assign_q + base, bi.start, n, n, keys, row_of, seg, warp_sum, nullptr, a.status, nullptr, 0);
+    const int n_kept = build_groups<T>(a.assign_q + base, bi.start, n, n, keys, row_of, seg, warp_sum, nullptr, a.status, nullptr, 0);
     const __nv_bfloat16* x = a.src_q.ptr + (int64_t)h * a.src_q.stride_head + (int64_t)bi.start * a.src_q.stride_token;
     const int64_t st = a.src_q.stride_token;
     // eight lanes per group (a lane owns 8 of the 64 channels), four groups per warp at a time
-    for (int row = warp * 4 + sub; row < ((n_kept + 3) & ~3); row += (MG_THREADS / 32) * 4) {   // (whole sub-groups stay together for the shuffles)
+    for (int row = warp * 4 + sub; row < ((n_kept + 3) & ~3); row += (T / 32) * 4) {   // (whole sub-groups stay together for the shuffles)
         const bool live = row < n_kept;
         const int i0 = live ? seg[row] : 0, i1 = live ? seg[row + 1] : 0;
         const int cnt = i1 - i0;
@@ -745,15 +749,16 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_deviation_kernel(const Outl
 
 // Outliers (eps > tau) leave their groups: an outlier maps to itself; the other tokens of a group stay together, under
 // their old representative if it is not an outlier, else under the remaining member with the lowest position.
-__global__ void __launch_bounds__(MG_THREADS, 1) big_filter_kernel(const OutlierArgs a) {
+template <int T>
+__global__ void __launch_bounds__(T, 1) big_filter_kernel(const OutlierArgs a) {
     extern __shared__ __align__(16) unsigned char mg_smem[];
     uint32_t* keys = reinterpret_cast<uint32_t*>(mg_smem);
-    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + kMaxBigBlockTokens * 4);
-    int* seg = reinterpret_cast<int*>(mg_smem + kMaxBigBlockTokens * 6);
-    int* warp_sum = seg + kMaxBigBlockTokens + 4;
-    int16_t* rep_of_row = reinterpret_cast<int16_t*>(mg_smem + MG_SMEM);
-    unsigned char* outl = mg_smem + MG_SMEM + kMaxBigBlockTokens * 2;
-    int16_t* new_rep = reinterpret_cast<int16_t*>(mg_smem + MG_SMEM + kMaxBigBlockTokens * 3);
+    int16_t* row_of = reinterpret_cast<int16_t*>(mg_smem + (4 * T) * 4);
+    int* seg = reinterpret_cast<int*>(mg_smem + (4 * T) * 6);
+    int* warp_sum = seg + (4 * T) + 4;
+    int16_t* rep_of_row = reinterpret_cast<int16_t*>(mg_smem + mg_smem_bytes(T));
+    unsigned char* outl = mg_smem + mg_smem_bytes(T) + (4 * T) * 2;
+    int16_t* new_rep = reinterpret_cast<int16_t*>(mg_smem + mg_smem_bytes(T) + (4 * T) * 3);
     __shared__ int s_kept, s_out;
     const int tid = threadIdx.x;
     const int h = blockIdx.x / a.n_blocks, b = blockIdx.x % a.n_blocks;
@@ -763,7 +768,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_filter_kernel(const Outlier
     const int32_t* A = a.assign_q + base;
     int32_t* A_out = a.assign_q_out + base;
     if (bi.r_q == 0) {   // nothing merged, every deviation is 0: nothing to filter unless everything is an outlier, which changes nothing here
-        for (int j = tid; j < n; j += MG_THREADS) A_out[j] = bi.start + j;
+        for (int j = tid; j < n; j += T) A_out[j] = bi.start + j;
         if (tid == 0) a.kept_cnt[(int64_t)h * a.n_blocks + b] = n;
         return;
     }
@@ -772,15 +777,15 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_filter_kernel(const Outlier
         s_out = 0;
     }
     const float tau = *a.tau;
-    const int n_kept = build_groups(A, bi.start, n, n, keys, row_of, seg, warp_sum, rep_of_row, a.status, nullptr, 0);
+    const int n_kept = build_groups<T>(A, bi.start, n, n, keys, row_of, seg, warp_sum, rep_of_row, a.status, nullptr, 0);
     int n_out = 0;
-    for (int j = tid; j < n; j += MG_THREADS) {
+    for (int j = tid; j < n; j += T) {
         const bool o = a.eps[base + j] > tau;
         outl[j] = o ? 1 : 0;
         n_out += o ? 1 : 0;
     }
     __syncthreads();
-    for (int row = tid; row < n_kept; row += MG_THREADS) {   // a thread per group: groups are short, the rare long one costs its thread a scan
+    for (int row = tid; row < n_kept; row += T) {   // a thread per group: groups are short, the rare long one costs its thread a scan
         const int rp = rep_of_row[row];
         int nr = rp;
         if (outl[rp]) {
@@ -797,7 +802,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_filter_kernel(const Outlier
     }
     __syncthreads();
     int kept = 0;
-    for (int j = tid; j < n; j += MG_THREADS) {
+    for (int j = tid; j < n; j += T) {
         int target = j;
         if (!outl[j]) {
             int rp = A[j] - bi.start;
@@ -820,24 +825,49 @@ __global__ void __launch_bounds__(MG_THREADS, 1) big_filter_kernel(const Outlier
 
 }  // namespace
 
-cudaError_t launch_big_deviation(const OutlierArgs& a, cudaStream_t stream) {
-    big_deviation_kernel<<<a.heads * a.n_blocks, MG_THREADS, MG_SMEM, stream>>>(a);
-    return cudaGetLastError();
+// threads per CTA for blocks of up to max_block tokens
+template <typename F>
+cudaError_t with_cta_size(int max_block, F&& f) {
+    if (max_block <= 256) return f(std::integral_constant<int, 64>{});
+    if (max_block <= 512) return f(std::integral_constant<int, 128>{});
+    if (max_block <= 1024) return f(std::integral_constant<int, 256>{});
+    if (max_block <= 2048) return f(std::integral_constant<int, 512>{});
+    return f(std::integral_constant<int, 1024>{});
 }
 
-cudaError_t launch_big_filter(const OutlierArgs& a, cudaStream_t stream) {
-    big_filter_kernel<<<a.heads * a.n_blocks, MG_THREADS, OF_SMEM, stream>>>(a);
-    return cudaGetLastError();
+cudaError_t launch_big_deviation(const OutlierArgs& a, int max_block, cudaStream_t stream) {
+    return with_cta_size(max_block, [&](auto t) {
+        constexpr int T = decltype(t)::value;
+        big_deviation_kernel<T><<<a.heads * a.n_blocks, T, mg_smem_bytes(T), stream>>>(a);
+        return cudaGetLastError();
+    });
+}
+
+cudaError_t launch_big_filter(const OutlierArgs& a, int max_block, cudaStream_t stream) {
+    return with_cta_size(max_block, [&](auto t) {
+        constexpr int T = decltype(t)::value;
+        big_filter_kernel<T><<<a.heads * a.n_blocks, T, of_smem_bytes(T), stream>>>(a);
+        return cudaGetLastError();
+    });
+}
+
+template <int T>
+cudaError_t configure_sorted_group_kernels() {
+    cudaError_t e = cudaFuncSetAttribute(big_merge_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, mg_smem_bytes(T));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(big_deviation_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, mg_smem_bytes(T));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(big_filter_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, of_smem_bytes(T));
 }
 
 cudaError_t configure_big_blocks() {
     cudaError_t e = cudaFuncSetAttribute(big_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SC_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(big_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(big_deviation_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MG_SMEM);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(big_filter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, OF_SMEM);
+    if (e == cudaSuccess) e = configure_sorted_group_kernels<64>();
+    if (e == cudaSuccess) e = configure_sorted_group_kernels<128>();
+    if (e == cudaSuccess) e = configure_sorted_group_kernels<256>();
+    if (e == cudaSuccess) e = configure_sorted_group_kernels<512>();
+    if (e == cudaSuccess) e = configure_sorted_group_kernels<1024>();
+    return e;
 }
 
 cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t stream) {
@@ -858,10 +888,13 @@ cudaError_t launch_big_select(const BigMatchArgs& a, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_big_merge(const MergeArgs& a, cudaStream_t stream) {
-    const int sp_chunks = (a.n_special_total + 127) / 128;
-    big_merge_kernel<<<2 * a.heads * a.n_blocks + a.heads * sp_chunks, MG_THREADS, MG_SMEM, stream>>>(a, sp_chunks);
-    return cudaGetLastError();
+cudaError_t launch_big_merge(const MergeArgs& a, int max_block, cudaStream_t stream) {
+    return with_cta_size(max_block, [&](auto t) {
+        constexpr int T = decltype(t)::value;
+        const int sp_chunks = (a.n_special_total + T / 8 - 1) / (T / 8);
+        big_merge_kernel<T><<<2 * a.heads * a.n_blocks + a.heads * sp_chunks, T, mg_smem_bytes(T), stream>>>(a, sp_chunks);
+        return cudaGetLastError();
+    });
 }
 
 }  // namespace httm

@@ -179,11 +179,11 @@ cudaError_t launch_threshold(const OutlierArgs& a, int sm_count, cudaStream_t st
 cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream);   // map rewrite + per-head offsets (two kernels)
 cudaError_t launch_offsets(const OutlierArgs& a, cudaStream_t stream);  // per-head offsets alone
 cudaError_t launch_threshold0(const OutlierArgs& a, int sm_count, cudaStream_t stream);   // threshold with the level-0 histogram taken from the deviations (three kernels)
-cudaError_t launch_big_deviation(const OutlierArgs& a, cudaStream_t stream);   // large blocks: deviations
-cudaError_t launch_big_filter(const OutlierArgs& a, cudaStream_t stream);      // large blocks: map rewrite + kept counts
+cudaError_t launch_big_deviation(const OutlierArgs& a, int max_block_tokens, cudaStream_t stream);   // large blocks: deviations
+cudaError_t launch_big_filter(const OutlierArgs& a, int max_block_tokens, cudaStream_t stream);      // large blocks: map rewrite + kept counts
 cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 contraction + row argmax
 cudaError_t launch_big_select(const BigMatchArgs& a, cudaStream_t stream);                  // top-r per (tensor, head, block)
-cudaError_t launch_big_merge(const MergeArgs& a, cudaStream_t stream);                      // sort by merged row + gather means
+cudaError_t launch_big_merge(const MergeArgs& a, int max_block_tokens, cudaStream_t stream);                      // sort by merged row + gather means
 cudaError_t configure_big_blocks();
 cudaError_t launch_linear(const LinearArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 GEMM for the projections
 cudaError_t configure_linear();
