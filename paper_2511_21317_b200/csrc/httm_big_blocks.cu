@@ -553,14 +553,12 @@ __device__ int build_groups(const int32_t* A, int block_start, int n, int limit,
     __syncthreads();
     for (int k = 2; k <= P; k <<= 1) {   // bitonic sort: the keys are distinct, so the order is unique
         for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            for (int i = tid; i < P; i += T) {
-                const int ixj = i ^ jj;
-                if (ixj > i) {
-                    const uint32_t x = keys[i], y = keys[ixj];
-                    if ((x > y) == ((i & k) == 0)) {
-                        keys[i] = y;
-                        keys[ixj] = x;
-                    }
+            for (int c = tid; c < (P >> 1); c += T) {   // comparator c of this stage: elements i and i + jj (bit jj of i clear)
+                const int i = ((c & ~(jj - 1)) << 1) | (c & (jj - 1));
+                const uint32_t x = keys[i], y = keys[i + jj];
+                if ((x > y) == ((i & k) == 0)) {
+                    keys[i] = y;
+                    keys[i + jj] = x;
                 }
             }
             __syncthreads();
