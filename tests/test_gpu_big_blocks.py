@@ -88,10 +88,10 @@ def test_large_blocks_ties_and_zero_vectors():
 
 
 def test_paper_block_regime_full_size_sampled():
-    """Runs of 128 tokens x 30 frames on 60 frames of 37 x 37 patches, 90 % / 70 % merged (Sec. 4.1), four heads:
-    maps and merged tensors on all tokens, attention output on sampled tokens."""
-    wl = synth.WORKLOADS["paper_1d"].replace(heads=4)
+    """Runs of 128 tokens x 30 frames on 60 frames of 37 x 37 patches, 90 % / 70 % merged (Sec. 4.1), all 16 heads (the
+    configuration the benchmark times): maps and merged tensors on all tokens, attention output on sampled tokens."""
+    wl = synth.WORKLOADS["paper_1d"]
     rng = np.random.default_rng(2)
-    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 48), [0, 4, 5, wl.n_tokens - 1]]))
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 24), [0, 4, 5, wl.n_tokens - 1]]))
     stats = run_big(wl, sample=toks)
-    assert stats["out_err"] <= parity.OUT_TOL
+    assert stats["out_err"] <= parity.OUT_TOL and stats["peaky_needed"] == 0

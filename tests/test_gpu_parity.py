@@ -49,7 +49,14 @@ def run_case(wl, q=None, k=None, v=None, sample=None, peaky=False):
 
 def test_tiny_config_full_parity():
     stats = run_case(synth.WORKLOADS["tiny"])
-    assert stats["out_err"] <= parity.OUT_TOL
+    assert stats["out_err"] <= parity.OUT_TOL and stats["peaky_needed"] == 0
+
+
+def report_peaky(name, stats):
+    """The adversarial cases are checked with the extra bf16-representation term; say how many elements used it."""
+    print(f"[peaky] {name}: {stats['peaky_needed']} of {stats['out_elements']} output elements beyond "
+          f"{parity.OUT_TOL} x RMS (max err / RMS {stats['out_err']:.4f})")
+    assert stats["peaky_needed"] <= 0.01 * stats["out_elements"]
 
 
 GEOMS = [
@@ -75,14 +82,14 @@ GEOMS = [
 def test_adversarial_geometries(case):
     name, S, h, w, blk, rq, rkv, ncam, nreg, H = case
     wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, n_camera=ncam, n_register=nreg, heads=H, seed=3)
-    run_case(wl, peaky=True)
+    report_peaky(name, run_case(wl, peaky=True))
 
 
 def test_random_uncorrelated_inputs():
     wl = synth.Workload("gauss", 4, 11, 13, 2, 4, 4, 0.6, 0.6, heads=4)
     rng = np.random.default_rng(5)
     q, k, v = (synth.f32_to_bf16_bits(rng.standard_normal((wl.heads, wl.n_tokens, 64)).astype(np.float32)) for _ in range(3))
-    run_case(wl, q, k, v, peaky=True)
+    report_peaky("gauss", run_case(wl, q, k, v, peaky=True))
 
 
 def test_ties_and_zero_vectors():
@@ -91,9 +98,9 @@ def test_ties_and_zero_vectors():
     q, k, v = synth.make_qkv(wl)
     z = q.copy()
     z[:, 10:40, :] = 0                                         # zero vectors: norm clamp
-    run_case(wl, x, k, v, peaky=True)
-    run_case(wl, q, x, v, peaky=True)
-    run_case(wl, z, z, v, peaky=True)
+    report_peaky("ties q", run_case(wl, x, k, v, peaky=True))
+    report_peaky("ties k", run_case(wl, q, x, v, peaky=True))
+    report_peaky("zero vectors", run_case(wl, z, z, v, peaky=True))
 
 
 def test_ratio_zero_equals_dense_and_textbook():
@@ -214,7 +221,7 @@ def test_small_config_full_size_sampled():
     rng = np.random.default_rng(1)
     toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 64), np.arange(5), [wl.n_tokens - 1]]))
     stats = run_case(wl, sample=toks)
-    assert stats["merged_exactly_rounded"] > 0.99
+    assert stats["merged_exactly_rounded"] > 0.99 and stats["peaky_needed"] == 0
 
 
 def test_medium_config_full_size_sampled():
@@ -225,7 +232,31 @@ def test_medium_config_full_size_sampled():
     rng = np.random.default_rng(2)
     toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 48), np.arange(5), [wl.n_tokens - 1]]))
     stats = run_case(wl, sample=toks)
-    assert stats["merged_exactly_rounded"] > 0.99
+    assert stats["merged_exactly_rounded"] > 0.99 and stats["peaky_needed"] == 0
+
+
+SWEEP = [(ratio, blk) for blk in ((2, 4, 4), (4, 4, 4), (2, 8, 8)) for ratio in (0.5, 0.7, 0.9)]
+
+
+@pytest.mark.parametrize("ratio,blk", SWEEP, ids=[f"{b[0]}x{b[1]}x{b[2]}-{r}" for r, b in SWEEP])
+def test_medium_sweep_full_size_sampled(ratio, blk):
+    """Every point of the medium scene's sweep (merge ratio 0.5 / 0.7 / 0.9, blocks 2x4x4 / 4x4x4 / 2x8x8) at full size:
+    permutation, maps, ranks and merged tensors on all tokens, attention on sampled tokens, plain 2e-2 x RMS bound."""
+    wl = synth.WORKLOADS["medium"].replace(name=f"medium-{blk}-{ratio}", blk_frames=blk[0], blk_h=blk[1], blk_w=blk[2],
+                                           ratio_q=ratio, ratio_kv=ratio)
+    rng = np.random.default_rng(20)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 24), np.arange(5), [wl.n_tokens - 1]]))
+    stats = run_case(wl, sample=toks)
+    assert stats["merged_exactly_rounded"] > 0.99 and stats["peaky_needed"] == 0
+
+
+def test_stack_layer_full_size_sampled():
+    """One layer of the 24-layer configuration at full size (S = 48, 65 952 tokens, 2x4x4 blocks, ratio 0.7)."""
+    wl = synth.WORKLOADS["stack_layer"]
+    rng = np.random.default_rng(21)
+    toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 16), np.arange(5), [wl.n_tokens - 1]]))
+    stats = run_case(wl, sample=toks)
+    assert stats["merged_exactly_rounded"] > 0.99 and stats["peaky_needed"] == 0
 
 
 def test_dense_attention_medium_config_sampled():
@@ -285,4 +316,4 @@ def test_large_config_full_size_sampled():
     rng = np.random.default_rng(4)
     toks = np.unique(np.concatenate([rng.integers(0, wl.n_tokens, 16), np.arange(5), [wl.n_tokens - 1]]))
     stats = run_case(wl, sample=toks)
-    assert stats["merged_exactly_rounded"] > 0.99
+    assert stats["merged_exactly_rounded"] > 0.99 and stats["peaky_needed"] == 0

@@ -9,8 +9,10 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import httm_oracle as orc
 from paper_2511_21317_b200 import binding as hb
 from paper_2511_21317_b200 import synth
+from tests import parity
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -47,6 +49,17 @@ def test_static_scratch_entry_matches_context_entry_twice_in_a_row():
             err = (out.float() - ref.float()).abs().max().item()
             assert np.isfinite(err) and err <= 2e-2 * rms, (wl.name, rep, err, rms)
             assert torch.equal(out, ref), (wl.name, rep)        # same kernels, same order: bit-identical
+
+
+def test_static_scratch_entry_against_the_oracle():
+    """Directly against the CPU oracle (not only through the context entry): output within 2e-2 x RMS on the tiny scene."""
+    wl = synth.WORKLOADS["tiny"]
+    q, k, v = synth.make_qkv(wl)
+    out = torch.empty(wl.n_tokens, wl.heads * 64, dtype=torch.bfloat16, device=DEV)
+    hb.global_attention_static(hb.HttmConfig.of(wl), *(hb.bf16_from_bits(x, DEV) for x in (q, k, v)), out)
+    torch.cuda.synchronize()
+    ref = orc.global_attention(orc.Geometry.of(wl), wl.ratio_q, wl.ratio_kv, q, k, v).out
+    assert parity.check_output(hb.bits_from_bf16(out), ref, what="static entry, tiny") <= parity.OUT_TOL
 
 
 def test_static_scratch_entry_rejects_what_does_not_fit():
