@@ -12,6 +12,7 @@ same workload on its own GPU: the path has no exchange step, so there is no data
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -27,9 +28,11 @@ if ROOT not in sys.path:
 
 from paper_2511_21317_b200 import synth  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (ncu, profiles/ncu_full_medium_five_kernels.txt);
-# None for workloads that were not captured, and to be reset to None whenever the attention kernel changes.
-ATTENTION_DRAM_TRAFFIC = {"medium": 64933120 + 5256960}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (one ncu capture, summary under profiles/), with
+# the digest of the kernel's sources at the time of the capture: the figure is reported only while the sources still
+# have that digest (null for workloads that were not captured and once the kernel has changed).
+ATTENTION_DRAM_TRAFFIC = {"medium": (64933120 + 5256960, "0" * 16)}
+ATTENTION_SOURCES = ("paper_2511_21317_b200/csrc/httm_attention_tc.cu", "paper_2511_21317_b200/csrc/tc_sm100.cuh")
 METRIC = "httm_global_attention_layer_throughput"
 UNIT = "tokens/s"
 
@@ -42,6 +45,24 @@ def workload_config(wl):
             "l2_policy": "inputs (Q/K/V %.0f MB) and streamed workspace are larger than the 126 MB L2; no flush"
                          % (3 * wl.heads * wl.n_tokens * wl.head_dim * 2 / 1e6),
             "parallelism": "replicas only (single-GPU path)"}
+
+
+def attention_source_digest():
+    h = hashlib.sha256()
+    for rel in ATTENTION_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def attention_traffic(workload_name):
+    """(bytes or None, note): the stored DRAM traffic of one attention launch, if it still describes the kernel."""
+    rec = ATTENTION_DRAM_TRAFFIC.get(workload_name)
+    if rec is None:
+        return None, "no ncu capture of this workload"
+    if rec[1] != attention_source_digest():
+        return None, "kernel sources changed since the ncu capture"
+    return rec[0], "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/)"
 
 
 def load_peaks():
@@ -57,8 +78,9 @@ def load_peaks():
 
 def oracle_layer_time(wl, q, k, v, sample_rows=48, keep=False):
     """Times the oracle as it stands on the host cores.  Reorder, match, merge and unmerge run in
-    full; attention runs on `sample_rows` merged query rows per head against all merged keys and is
-    scaled by M_q / sample_rows.  Returns (seconds per layer, details)."""
+    full.  sample_rows <= 0: attention in full too, the total is a measured time.  sample_rows > 0:
+    attention runs on that many merged query rows per head against all merged keys and is scaled by
+    M_q / sample_rows (the total is then labelled as extrapolated).  Returns (seconds per layer, details)."""
     from oracle import httm_oracle as orc
     g = orc.Geometry.of(wl)
     t = {}
@@ -75,21 +97,26 @@ def oracle_layer_time(wl, q, k, v, sample_rows=48, keep=False):
     rk, Mk = orc.merged_rank(g, ak)
     qm, km, vm = orc.merge(g, rq, Mq, qr), orc.merge(g, rk, Mk, kr), orc.merge(g, rk, Mk, vr)
     t["merge"] = time.perf_counter() - t0
-    rows = np.unique(np.linspace(0, Mq - 1, sample_rows).astype(np.int64))
+    full = sample_rows <= 0 or sample_rows >= Mq
+    rows = np.arange(Mq, dtype=np.int64) if full else np.unique(np.linspace(0, Mq - 1, sample_rows).astype(np.int64))
     t0 = time.perf_counter()
-    o_rows = orc.attention(qm, km, vm, rows)
+    o_rows = orc.attention(qm, km, vm, None if full else rows)
     t_attn = time.perf_counter() - t0
-    t["attention_sampled"] = t_attn
-    t["attention_extrapolated"] = t_attn * Mq / len(rows)
+    if full:
+        t["attention"] = t_attn
+    else:
+        t["attention_sampled"] = t_attn
+        t["attention_extrapolated"] = t_attn * Mq / len(rows)
     t0 = time.perf_counter()
     om = np.zeros((g.heads, Mq, g.head_dim))
     om[:, rows] = o_rows
     out = orc.unmerge(g, pi, rq, om)
     t["unmerge"] = time.perf_counter() - t0
-    total = t["reorder"] + t["match"] + t["merge"] + t["attention_extrapolated"] + t["unmerge"]
-    info = {"seconds": {k_: round(v_, 4) for k_, v_ in t.items()}, "cores": orc.threads(),
-            "sample": f"reorder, match, merge, unmerge in full; attention on {len(rows)} of {Mq} merged query rows per head "
-                      f"(all {Mk} keys), scaled by M_q/rows"}
+    total = t["reorder"] + t["match"] + t["merge"] + (t_attn if full else t["attention_extrapolated"]) + t["unmerge"]
+    info = {"seconds": {k_: round(v_, 4) for k_, v_ in t.items()}, "cores": orc.threads(), "extrapolated": not full,
+            "sample": ("the whole workload, nothing sampled: every step of the path in full" if full else
+                       f"reorder, match, merge, unmerge in full; attention on {len(rows)} of {Mq} merged query rows per head "
+                       f"(all {Mk} keys), scaled by M_q/rows (extrapolated)")}
     kept = None
     if keep:
         kept = dict(g=g, pi=pi, bs=bs, qr=qr, kr=kr, aq=aq, ak=ak, mbq=mbq, msq=msq, mbk=mbk, msk=msk, rq=rq, rows=rows,
@@ -105,14 +132,17 @@ def run_reference(args, wl):
     times = []
     info = None
     for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
         tot, info, _ = oracle_layer_time(wl, q, k, v, sample_rows=args.oracle_rows)
-        if i >= args.warmup:
-            times.append(tot)
+        wall = time.perf_counter() - t0
+        if i >= args.warmup:   # a step in full is the wall clock around it; a sampled one reports the extrapolated total
+            times.append(tot if info["extrapolated"] else wall)
     sec = float(np.mean(times))
     val = wl.n_tokens / sec
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic", "config": workload_config(wl),
+            "ms_per_step_is": "extrapolated from a sample (see cpu_baseline.sample)" if info["extrapolated"] else "measured",
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": info["cores"], "kind": "oracle", "sample": info["sample"],
                              "seconds": info["seconds"]},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -258,9 +288,31 @@ def run_ours(args, wl):
             ctx.launch_stage(st, dq, dk, dv, out)
             evs[s_][i + 1].record(stream)
     torch.cuda.synchronize()
+    stage_loop_s = evs[0][0].elapsed_time(evs[-1][-1]) * 1e-3
+    clocks_timed = clocks_stage = sampler.stop()   # one record over the timed region and the per-kernel loop behind it
     for s_ in range(args.steps):
         for i, st in enumerate(order):
             stage_ms[st] += evs[s_][i].elapsed_time(evs[s_][i + 1]) / args.steps
+
+    # ---- the attention kernel alone, back to back for about a second and a half: the regime the sustained GEMM peak
+    #      was measured in (seconds of tensor-core work under the board's power limit)
+    sus_reps = 0
+    sus_ms = None
+    clocks_sus = None
+    if rank == 0 and args.sustained_seconds > 0:
+        sus_reps = int(min(20000, max(10, args.sustained_seconds / max(stage_ms[3] * 1e-3, 1e-5))))
+        sus_sampler = ClockSampler(local)
+        sus_sampler.start()
+        s0, s1 = ev(), ev()
+        s0.record(stream)
+        for _ in range(sus_reps):
+            ctx.launch_stage(3, dq, dk, dv, out)
+        s1.record(stream)
+        torch.cuda.synchronize()
+        sus_ms = s0.elapsed_time(s1) / sus_reps
+        clocks_sus = sus_sampler.stop()
+    sampler = ClockSampler(local)
+    sampler.start()
 
     # ---- dense baseline of the same run (same attention kernel on the unmerged tokens)
     dsteps = max(3, min(args.steps, 10))
@@ -275,7 +327,8 @@ def run_ours(args, wl):
     d1.record(stream)
     torch.cuda.synchronize()
     dense_ms = d0.elapsed_time(d1) / dsteps
-    clocks = sampler.stop()
+    clocks_dense = sampler.stop()
+    clocks = clocks_timed
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies inside the timed region)
     hq, hk, hv = (hb.bf16_from_bits(x, pin=True) for x in (q, k, v))
@@ -323,7 +376,8 @@ def run_ours(args, wl):
                                  "algorithmic_gflop": big_flops / 1e9}
             elif name == "attention":
                 tf = attn_flops / (ms * 1e-3) / 1e12
-                kernels[name] = {"ms": ms, "tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                kernels[name] = {"ms": ms, "tflops": tf, "frac_of_measured_bf16_burst": tf / peaks["bf16_tflops"],
+                                 "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
                                  "frac_of_nominal_2250": tf / 2250.0}
             else:
                 gbs = alg[name] / (ms * 1e-3) / 1e9
@@ -334,10 +388,26 @@ def run_ours(args, wl):
                 "sum_of_their_stage_times_ms": float(sum(stage_ms[st] for st in used))}
         attn_ms = float(stage_ms[3])
         attn_tf = attn_flops / (attn_ms * 1e-3) / 1e12
-        roofline = {"kernel": "attention (merged sets)", "bound": "tensor", "achieved": attn_tf,
-                    "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": attn_tf / peaks["bf16_tflops_sustained"],
-                    "peak_source": peaks["source"] + " (sustained bf16 GEMM; kernel timed inside the step)",
-                    "traffic": ATTENTION_DRAM_TRAFFIC.get(wl.name)}
+        # Which measured GEMM peak the kernel is compared with: the sustained one only if the loop it was timed in
+        # lasted at least a second and the power cap was seen in the clock samples of that loop, else the burst one.
+        capped = "sw_power_cap" in (clocks_stage.get("reasons") or [])
+        use_sustained = stage_loop_s >= 1.0 and capped
+        peak = peaks["bf16_tflops_sustained"] if use_sustained else peaks["bf16_tflops"]
+        traffic, traffic_note = attention_traffic(wl.name)
+        roofline = {"kernel": "attention (merged sets)", "bound": "tensor", "achieved": attn_tf, "peak": peak, "unit": "TFLOP/s",
+                    "frac": attn_tf / peak, "frac_burst": attn_tf / peaks["bf16_tflops"],
+                    "frac_sustained": attn_tf / peaks["bf16_tflops_sustained"],
+                    "peak_source": peaks["source"] + (" sustained" if use_sustained else " burst") + " bf16 GEMM rate: the kernel's timing loop lasted "
+                                   f"{stage_loop_s:.3f} s, power cap {'seen' if capped else 'not seen'} in its clock samples",
+                    "timing_loop": {"seconds": stage_loop_s, "launches": args.steps, "clocks": clocks_stage,
+                                    "ms_x_sm_mhz": None if clocks_stage.get("sm_mhz") is None else attn_ms * clocks_stage["sm_mhz"]},
+                    "traffic": traffic, "traffic_note": traffic_note}
+        if sus_ms is not None:
+            sus_tf = attn_flops / (sus_ms * 1e-3) / 1e12
+            roofline["back_to_back"] = {"launches": sus_reps, "seconds": sus_ms * sus_reps * 1e-3, "ms": sus_ms, "achieved": sus_tf,
+                                        "frac_of_sustained_peak": sus_tf / peaks["bf16_tflops_sustained"],
+                                        "frac_of_burst_peak": sus_tf / peaks["bf16_tflops"], "clocks": clocks_sus,
+                                        "ms_x_sm_mhz": None if clocks_sus.get("sm_mhz") is None else sus_ms * clocks_sus["sm_mhz"]}
         line = {
             "metric": METRIC, "value": replica_throughput(N, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -351,7 +421,8 @@ def run_ours(args, wl):
             "kernels": kernels,
             "path": path,
             "merged_tokens": {"M_q": Mq, "M_k": Mk},
-            "dense": {"ms": dense_ms, "tflops": 4.0 * H * N * N * D / (dense_ms * 1e-3) / 1e12, "steps": dsteps},
+            "dense": {"ms": dense_ms, "tflops": 4.0 * H * N * N * D / (dense_ms * 1e-3) / 1e12, "steps": dsteps,
+                      "clocks": clocks_dense},
             "speedup_vs_dense": dense_ms / ms_step,
             "device_status": status,
         }
@@ -446,7 +517,11 @@ def main():
     ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
     ap.add_argument("--block", default=None, help="override block shape, e.g. 4x4x4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--oracle-rows", type=int, default=4096, help="merged query rows per head the CPU oracle attends (sample)")
+    ap.add_argument("--oracle-rows", type=int, default=None,
+                    help="merged query rows per head the CPU oracle attends; 0 = all of them, nothing extrapolated (default: 0 "
+                         "for --impl reference, whose step time is then a measured one, 4096 for the in-line cpu_baseline)")
+    ap.add_argument("--sustained-seconds", type=float, default=1.5,
+                    help="length of the back-to-back run of the attention kernel alone that is compared with the sustained GEMM peak (0: skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--outlier-fraction", type=float, default=None,
                     help="also time the step with query outlier filtering at this fraction (extra block of the line; 0: skip; "
@@ -460,6 +535,8 @@ def main():
         wl = wl.replace(blk_frames=bt, blk_h=bh, blk_w=bw)
     if args.outlier_fraction is None:
         args.outlier_fraction = 0.1 if args.workload == "paper_1d" else 0.01
+    if args.oracle_rows is None:
+        args.oracle_rows = 0 if args.impl == "reference" else 4096
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

@@ -56,7 +56,7 @@ def report_peaky(name, stats):
     """The adversarial cases are checked with the extra bf16-representation term; say how many elements used it."""
     print(f"[peaky] {name}: {stats['peaky_needed']} of {stats['out_elements']} output elements beyond "
           f"{parity.OUT_TOL} x RMS (max err / RMS {stats['out_err']:.4f})")
-    assert stats["peaky_needed"] <= 0.01 * stats["out_elements"]
+    assert stats["peaky_needed"] <= 0.001 * stats["out_elements"]   # (at most 5 elements in any case when this was written)
 
 
 GEOMS = [
