@@ -2,11 +2,12 @@
  * httm.h - C ABI of the B200 (sm_100a) library for one VGGT-style global-attention
  * layer with head-wise temporal token merging (HTTM).
  *
- * The path behind these calls is Algorithm 1 of the HTTM paper without its
- * projections and without outlier filtering:
+ * The path behind these calls is Algorithm 1 of the HTTM paper between its projections:
  *   temporal reorder (Sec. 3.3) -> per-head, per-block cosine matching of Q and of K
- *   (Eq. 1) -> mean merge of Q, K, V (V follows K, Sec. 3.2) -> softmax attention on
- *   the merged sets (Eq. 3-4) -> head-wise unmerge (Eq. 5-7) + inverse reorder.
+ *   (Eq. 1) -> [optional: outlier filtering of the queries, Sec. 3.4 / Algorithm 2, see
+ *   httm_set_outlier_fraction] -> mean merge of Q, K, V (V follows K, Sec. 3.2) -> softmax
+ *   attention on the merged sets (Eq. 3-4) -> head-wise unmerge (Eq. 5-7) + inverse reorder.
+ * The projections themselves are offered as httm_linear.
  *
  * Conventions common to all calls
  *   - S frames; every frame has n_camera + n_register special tokens followed by a
@@ -131,7 +132,10 @@ enum {
      * UNSUPPORTED; the order is 0, 8, 9, 2, 3, 4.  8: cosine of every token with every dst token of its block on the
      * tensor cores + best dst per token; 9: the r best src of every block merge (map written) */
     HTTM_STAGE_BIG_SCORES = 8,
-    HTTM_STAGE_BIG_SELECT = 9
+    HTTM_STAGE_BIG_SELECT = 9,
+    HTTM_STAGE_ATTENTION_UNMERGE = 10 /* stages 3 and 4 as one kernel: the attention epilogue writes every merged query row to its
+                                         member tokens in `out` (contexts with blocks of at most 32 tokens, outlier filtering off;
+                                         UNSUPPORTED otherwise); needs the member lists the last merge stage (2 or 6) left */
 };
 
 /*
@@ -153,9 +157,12 @@ int httm_create(const httm_config* cfg, httm_ctx** out);
  *   (mean of constituents) -> attention on merged sets (Eq. 3-4) -> unmerge +
  *   inverse reorder + head concat (Eq. 5-7).
  * Match and merge load each block's patch window straight from q, k, v and no reordered
- * copy is written (four kernels; HTTM_X_*_REORDERED hold what the last HTTM_STAGE_REORDER
- * wrote).  Scenes of more than 32767 frames / patch rows / patch columns, or with more than 32 special
- * tokens per frame, take five.
+ * copy is written (HTTM_X_*_REORDERED hold what the last HTTM_STAGE_REORDER wrote); scenes of
+ * more than 32767 frames / patch rows / patch columns, or with more than 32 special tokens per
+ * frame, run the reorder kernel first.  With blocks of at most 32 tokens (and outlier filtering
+ * off) the unmerge runs in the attention kernel's epilogue: every merged query row is written
+ * straight to its member tokens in `out`, three kernels in all; the merged attention output
+ * (HTTM_X_O_MERGED) is then computed only when it is exported.  Larger blocks: four kernels.
  * With ratio_q = ratio_kv = 0 the result equals httm_dense_attention up to rounding.
  * Errors: INVALID_ARG, ALIGNMENT, CUDA (launch failure); device-side wait time-outs
  * are reported by the next httm_query(HTTM_Q_DEVICE_STATUS) / httm_export.
@@ -259,7 +266,13 @@ int64_t httm_launch_count(const httm_ctx* ctx);
  *     the tiny 1044-token, 16-head configuration needs about 11 MiB) are rejected with
  *     HTTM_ERR_UNSUPPORTED before anything is launched; use a context for those.
  *   - The first call on a device looks up the array's device address and sets kernel
- *     attributes; make that first call outside any stream capture.
+ *     attributes; make that first call before any stream capture begins.
+ *   - The array also holds the plan tables of one configuration per device (reorder index and
+ *     block table).  A call whose configuration differs from the one resident on that device
+ *     (the first call included) uploads them: three host-to-device copies from pageable memory
+ *     on `cuda_stream`, which the runtime stages on the host before it returns.  Calls that
+ *     repeat the resident configuration enqueue kernels only, and return without waiting for
+ *     earlier work on the stream.
  *   - All calls share the one array and it keeps the previous call's contents (the call
  *     resets what must start clean).  Two calls that overlap on the GPU, e.g. on different
  *     streams, race on it: serialise them.  Calls are serialised on the host by a lock.

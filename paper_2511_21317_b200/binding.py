@@ -22,9 +22,9 @@ LIB_PATH = os.path.join(_HERE, "libhttm.so")
 (X_PI, X_PI_INV, X_BLOCK_START, X_ASSIGN_Q, X_ASSIGN_K, X_RANK_Q, X_Q_REORDERED, X_K_REORDERED, X_V_REORDERED,
  X_Q_MERGED, X_K_MERGED, X_V_MERGED, X_O_MERGED, X_DEVIATION, X_THRESHOLD, X_MERGED_Q_HEAD, X_ASSIGN_Q_INITIAL) = range(17)
 (STAGE_REORDER, STAGE_MATCH, STAGE_MERGE, STAGE_ATTENTION, STAGE_UNMERGE, STAGE_MATCH_DIRECT, STAGE_MERGE_DIRECT,
- STAGE_OUTLIER_FILTER, STAGE_BIG_SCORES, STAGE_BIG_SELECT) = range(10)
+ STAGE_OUTLIER_FILTER, STAGE_BIG_SCORES, STAGE_BIG_SELECT, STAGE_ATTENTION_UNMERGE) = range(11)
 STAGE_NAMES = ("reorder", "match", "merge", "attention", "unmerge", "match_direct", "merge_direct", "outlier_filter",
-               "big_scores", "big_select")
+               "big_scores", "big_select", "attention_unmerge")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 _STATUS_NAMES = {0: "HTTM_OK", -1: "HTTM_ERR_INVALID_ARG", -2: "HTTM_ERR_UNSUPPORTED", -3: "HTTM_ERR_ALIGNMENT",

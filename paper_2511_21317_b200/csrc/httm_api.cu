@@ -10,6 +10,7 @@
 
 #include "../../include/httm.h"
 #include "httm_internal.h"
+#include "httm_plan.h"
 
 using namespace httm;
 
@@ -45,6 +46,11 @@ struct httm_ctx {
     BlockInfo* d_blocks = nullptr;
     __nv_bfloat16 *d_qr = nullptr, *d_kr = nullptr, *d_vr = nullptr;
     __nv_bfloat16 *d_qm = nullptr, *d_km = nullptr, *d_vm = nullptr, *d_om = nullptr;
+    // Members of every merged query row (blocks of at most 32 tokens): the attention epilogue writes each row straight to
+    // its tokens (unmerge + inverse reorder, Eq. 5-7, without the O_m round trip).  om_stale: the last call took that
+    // path, so O_m does not hold its attention output (httm_export recomputes it on request).
+    int32_t *d_group_start = nullptr, *d_group_member = nullptr;
+    bool om_stale = false;
     // query outlier filtering (Sec. 3.4): off while fraction == 0; its workspace is allocated when it is first switched on.
     // The merged query length then differs per head: Q_m and O_m get N rows per head.
     double outlier_fraction = 0.0;
@@ -101,7 +107,8 @@ struct httm_ctx {
         void* ptrs[] = {d_geom, d_pi, d_pi_inv, d_assign_q, d_assign_k, d_rank_q, d_status, d_blocks, d_qr, d_kr,
                         d_vr, d_qm,     d_km,       d_vm,       d_om,     hs[0].q,  hs[0].k,  hs[0].v, hs[0].out, hs[1].q, hs[1].k, hs[1].v, hs[1].out,
                         d_assign_qf, d_kept_cnt, d_moff_var, d_mq_head, d_tile_prefix, d_sel, d_eps, d_tau, d_qm_var, d_om_var,
-                        d_big_items, d_inv_norm_q, d_inv_norm_k, d_best_key_q, d_best_key_k, d_best_pos_q, d_best_pos_k};
+                        d_big_items, d_inv_norm_q, d_inv_norm_k, d_best_key_q, d_best_key_k, d_best_pos_q, d_best_pos_k,
+                        d_group_start, d_group_member};
         for (void* p : ptrs)
             if (p) cudaFree(p);
         for (HostSet& h : hs)
@@ -113,20 +120,6 @@ struct httm_ctx {
 };
 
 namespace {
-
-int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
-
-// Merge budget of a block of n tokens (Sec. 3.2, r = N - M): r src tokens are merged away,
-// n_dst evenly spaced tokens act as destinations.
-void block_budget(int n, double ratio, int32_t* r, int32_t* nd) {
-    int64_t rr = (int64_t)std::floor(ratio * (double)n + 1e-9);
-    if (rr > n - 1) rr = n - 1;
-    if (rr < 0) rr = 0;
-    int64_t d = ceil_div64(n, 4);
-    if (d > n - rr) d = n - rr;
-    *r = (int32_t)rr;
-    *nd = (int32_t)d;
-}
 
 int check_cuda(httm_ctx* c, cudaError_t e, const char* what) {
     if (e == cudaSuccess) return HTTM_OK;
@@ -144,15 +137,8 @@ int64_t span_bytes(const httm_ctx* c, const httm_tensor& t) {
 }
 
 int check_tensor(httm_ctx* c, const httm_tensor& t, const char* name) {
-    if (!t.ptr) return c->fail(HTTM_ERR_INVALID_ARG, "%s: null pointer", name);
-    if (((uintptr_t)t.ptr & 15u) != 0) return c->fail(HTTM_ERR_ALIGNMENT, "%s: pointer is not 16-byte aligned", name);
-    if (t.stride_head % 8 != 0 || t.stride_token % 8 != 0)
-        return c->fail(HTTM_ERR_ALIGNMENT, "%s: strides must be multiples of 8 elements", name);
-    if (t.stride_token < kHeadDim || t.stride_head < 0)
-        return c->fail(HTTM_ERR_INVALID_ARG, "%s: stride_token must be >= head_dim and stride_head >= 0", name);
-    if (c->cfg.heads > 1 && t.stride_head < kHeadDim)
-        return c->fail(HTTM_ERR_INVALID_ARG, "%s: stride_head must be >= head_dim", name);
-    return HTTM_OK;
+    const int rc = check_tensor_layout(t, c->cfg.heads, name, &c->error);
+    return rc;
 }
 
 int check_io(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out) {
@@ -216,6 +202,10 @@ bool direct_mode(const httm_ctx* c) {
 // Q/K/V; everywhere else (larger blocks, or scenes that take the reordered copies) on the sorted-group kernels of the
 // large-block path, which handle any block size from the reordered copy.
 bool sorted_filter(const httm_ctx* c) { return c->filtering() && !(c->max_block <= 32 && direct_mode(c)); }
+
+// The unmerge runs in the attention epilogue where the merge kernel leaves the member lists of the merged query rows:
+// blocks of at most 32 tokens, every head with the same merged length (no outlier filtering).
+bool fused_unmerge(const httm_ctx* c) { return c->d_group_start != nullptr && !c->filtering(); }
 
 BigMatchArgs big_match_args(httm_ctx* c) {
     BigMatchArgs a{};
@@ -291,6 +281,11 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.merged[1] = c->d_km;
     a.merged[2] = c->d_vm;
     a.rank_q = c->d_rank_q;
+    if (fused_unmerge(c)) {
+        a.group_start = c->d_group_start;
+        a.group_member = c->d_group_member;
+        a.pi = c->d_pi;
+    }
     a.blocks = c->d_blocks;
     a.n_blocks = c->n_blocks;
     a.n_tokens = c->n_tokens;
@@ -304,14 +299,27 @@ int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     return check_cuda(c, launch_merge(a, c->max_block, c->sm_count, s), "merge launch");
 }
 
-int stage_attention(httm_ctx* c, cudaStream_t s) {
+// final_out: null = the merged output O_m is written (unmerged by the next stage); else the epilogue writes every merged row
+// to its member tokens in the caller's output tensor (needs fused_unmerge)
+int stage_attention(httm_ctx* c, cudaStream_t s, const httm_tensor* final_out = nullptr) {
     AttentionArgs a{};
     a.q = view(c->filtering() ? c->d_qm_var : c->d_qm, c->q_rows());
     a.k = view(c->d_km, c->m_k);
     a.v = view(c->d_vm, c->m_k);
-    a.out = c->filtering() ? c->d_om_var : c->d_om;
-    a.out_stride_head = (int64_t)c->q_rows() * kHeadDim;
-    a.out_stride_token = kHeadDim;
+    if (final_out) {
+        if (!fused_unmerge(c)) return c->fail(HTTM_ERR_UNSUPPORTED, "unmerge in the attention epilogue needs blocks of at most 32 tokens and no outlier filtering");
+        a.out = reinterpret_cast<__nv_bfloat16*>(final_out->ptr);
+        a.out_stride_head = final_out->stride_head;
+        a.out_stride_token = final_out->stride_token;
+        a.group_start = c->d_group_start;
+        a.group_member = c->d_group_member;
+        a.n_tokens = c->n_tokens;
+    } else {
+        a.out = c->filtering() ? c->d_om_var : c->d_om;
+        a.out_stride_head = (int64_t)c->q_rows() * kHeadDim;
+        a.out_stride_token = kHeadDim;
+    }
+    c->om_stale = final_out != nullptr;
     a.m_q = c->q_rows();
     if (c->filtering()) {
         a.mq_head = c->d_mq_head;
@@ -326,6 +334,7 @@ int stage_attention(httm_ctx* c, cudaStream_t s) {
 }
 
 int stage_unmerge(httm_ctx* c, const httm_tensor& out, cudaStream_t s) {
+    if (c->om_stale) return c->fail(HTTM_ERR_INVALID_ARG, "the merged output is not there: the last attention launch unmerged in its epilogue (run HTTM_STAGE_ATTENTION first)");
     UnmergeArgs a{};
     a.o_m = c->filtering() ? c->d_om_var : c->d_om;
     a.rank_q = c->d_rank_q;
@@ -417,7 +426,7 @@ int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const h
         if ((rc = stage_attention(c, s))) return rc;
         return stage_unmerge(c, out, s);
     }
-    if (direct_mode(c)) {   // four kernels: the temporal reorder is folded into the block loads of match and merge
+    if (direct_mode(c)) {   // the temporal reorder is folded into the block loads of match and merge
         const httm_tensor src[3] = {q, k, v};
         if ((rc = stage_match(c, s, src))) return rc;
         if (c->filtering() && (rc = stage_outlier(c, q, s))) return rc;
@@ -427,6 +436,7 @@ int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const h
         if ((rc = stage_match(c, s))) return rc;
         if ((rc = stage_merge(c, s))) return rc;
     }
+    if (fused_unmerge(c)) return stage_attention(c, s, &out);   // ... and the unmerge into the attention epilogue: three kernels
     if ((rc = stage_attention(c, s))) return rc;
     return stage_unmerge(c, out, s);
 }
@@ -455,18 +465,11 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
         g_create_error = std::string("httm_create: ") + msg;
         return code;
     };
-    if (cfg->frames < 1 || cfg->n_camera < 0 || cfg->n_register < 0 || cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->heads < 1 ||
-        cfg->blk_frames < 1 || cfg->blk_h < 1 || cfg->blk_w < 1)
-        return bad(HTTM_ERR_INVALID_ARG, "sizes must be positive (special-token counts non-negative)");
-    if (!(cfg->ratio_q >= 0.0 && cfg->ratio_q < 1.0) || !(cfg->ratio_kv >= 0.0 && cfg->ratio_kv < 1.0))
-        return bad(HTTM_ERR_INVALID_ARG, "merge ratios must lie in [0, 1)");
-    if (cfg->anchor_first_frame != 0 && cfg->anchor_first_frame != 1) return bad(HTTM_ERR_INVALID_ARG, "anchor_first_frame must be 0 or 1");
-    if (cfg->head_dim != kHeadDim) return bad(HTTM_ERR_UNSUPPORTED, "head_dim must be 64");
-    if (cfg->heads > 65535) return bad(HTTM_ERR_UNSUPPORTED, "at most 65535 heads");
-    const int64_t per_frame = (int64_t)cfg->n_camera + cfg->n_register + (int64_t)cfg->grid_h * cfg->grid_w;
-    const int64_t n_tokens = per_frame * cfg->frames;
-    if (n_tokens > (1ll << 24) || n_tokens * cfg->heads > (1ll << 31) - 1)
-        return bad(HTTM_ERR_UNSUPPORTED, "too many tokens (N <= 2^24 and N*heads < 2^31)");
+    {
+        std::string why;
+        const int rc = check_config(*cfg, &why);
+        if (rc != HTTM_OK) return bad(rc, why.c_str());
+    }
     const int64_t bf = std::min<int64_t>(cfg->blk_frames, cfg->frames), bh = std::min<int64_t>(cfg->blk_h, cfg->grid_h),
                   bw = std::min<int64_t>(cfg->blk_w, cfg->grid_w);
     if (bf * bh * bw > kMaxBigBlockTokens) return bad(HTTM_ERR_UNSUPPORTED, "a merging block may hold at most 4096 tokens");
@@ -479,57 +482,26 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
     httm_ctx* c = new (std::nothrow) httm_ctx();
     if (!c) return bad(HTTM_ERR_NOMEM, "host allocation failed");
     c->cfg = *cfg;
-    c->n_special = cfg->n_camera + cfg->n_register;
-    c->tokens_per_frame = (int32_t)per_frame;
-    c->n_tokens = (int32_t)n_tokens;
-
-    // --- reorder index pi (Sec. 3.3): specials first (frame-major), then the blocks
-    //     (frame group, window row, window column), inside a block frame / y / x.
-    const int S = cfg->frames, h = cfg->grid_h, w = cfg->grid_w, nsp = c->n_special, P = c->tokens_per_frame;
-    c->pi.resize(n_tokens);
-    c->pi_inv.resize(n_tokens);
-    int32_t pos = 0;
-    for (int s = 0; s < S; ++s)
-        for (int j = 0; j < nsp; ++j) c->pi[pos++] = s * P + j;
-    int32_t moff_q = pos, moff_k = pos;
     int anchored_nd_max = 0;
-    for (int g0 = 0; g0 < S; g0 += cfg->blk_frames) {
-        const int f = std::min(cfg->blk_frames, S - g0);
-        for (int y0 = 0; y0 < h; y0 += cfg->blk_h) {
-            const int hh = std::min(cfg->blk_h, h - y0);
-            for (int x0 = 0; x0 < w; x0 += cfg->blk_w) {
-                const int ww = std::min(cfg->blk_w, w - x0);
-                BlockInfo bi{};
-                bi.start = pos;
-                bi.n = f * hh * ww;
-                bi.n_rule = bi.n;
-                block_budget(bi.n, cfg->ratio_q, &bi.r_q, &bi.nd_q);
-                block_budget(bi.n, cfg->ratio_kv, &bi.r_k, &bi.nd_k);
-                if (cfg->anchor_first_frame && g0 == 0) {   // the block's tokens of frame 0 are its dst tokens, all others src
-                    const int n0 = hh * ww;
-                    bi.n_rule = n0;
-                    bi.nd_q = bi.nd_k = n0;
-                    bi.r_q = std::min<int64_t>((int64_t)std::floor(cfg->ratio_q * (double)bi.n + 1e-9), bi.n - n0);
-                    bi.r_k = std::min<int64_t>((int64_t)std::floor(cfg->ratio_kv * (double)bi.n + 1e-9), bi.n - n0);
-                    anchored_nd_max = std::max(anchored_nd_max, n0);
-                }
-                bi.moff_q = moff_q;
-                bi.moff_k = moff_k;
-                moff_q += bi.n - bi.r_q;
-                moff_k += bi.n - bi.r_k;
-                c->max_block = std::max(c->max_block, bi.n);
-                for (int row0 = 0; row0 < bi.n; row0 += kBigSliceRows) c->big_items.push_back(BigItem{(int32_t)c->blocks.size(), row0});
-                c->blk_start.push_back(pos);
-                c->blocks.push_back(bi);
-                c->geom.push_back(BlockGeom{(int16_t)g0, (int16_t)y0, (int16_t)x0, (int16_t)f, (int16_t)hh, (int16_t)ww});
-                for (int tl = 0; tl < f; ++tl)
-                    for (int yl = 0; yl < hh; ++yl)
-                        for (int xl = 0; xl < ww; ++xl) c->pi[pos++] = (g0 + tl) * P + nsp + (y0 + yl) * w + (x0 + xl);
-            }
-        }
+    {   // reorder index, block table and merge budgets (Sec. 3.2 / 3.3)
+        HostPlan plan;
+        build_host_plan(*cfg, &plan);
+        c->n_special = plan.n_special;
+        c->tokens_per_frame = plan.tokens_per_frame;
+        c->n_tokens = plan.n_tokens;
+        c->n_blocks = plan.n_blocks;
+        c->max_block = plan.max_block;
+        c->m_q = plan.m_q;
+        c->m_k = plan.m_k;
+        anchored_nd_max = plan.anchored_dst_max;
+        c->pi = std::move(plan.pi);
+        c->pi_inv = std::move(plan.pi_inv);
+        c->blk_start = std::move(plan.blk_start);
+        c->blocks = std::move(plan.blocks);
+        c->geom = std::move(plan.geom);
+        for (int32_t b = 0; b < c->n_blocks; ++b)
+            for (int row0 = 0; row0 < c->blocks[b].n; row0 += kBigSliceRows) c->big_items.push_back(BigItem{b, row0});
     }
-    c->blk_start.push_back(pos);
-    c->n_blocks = (int32_t)c->blocks.size();
     {   // the match kernels hold a quarter of their largest block as dst tokens (the large-block path 1024)
         const int cap = c->max_block > kMaxBlockTokens ? kMaxBigDst : (c->max_block <= 32 ? 8 : (c->max_block <= 64 ? 16 : (c->max_block <= 128 ? 32 : 64)));
         if (anchored_nd_max > cap) {
@@ -537,10 +509,6 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
             return bad(HTTM_ERR_UNSUPPORTED, "first-frame anchoring: a block's tokens of frame 0 exceed a quarter of the largest block (use more frames per block)");
         }
     }
-    c->m_q = moff_q;
-    c->m_k = moff_k;
-    for (int32_t p = 0; p < c->n_tokens; ++p) c->pi_inv[c->pi[p]] = p;
-
     DeviceGuard guard(cfg->device);
     int rc = HTTM_OK;
     auto done = [&](int code) -> int {
@@ -572,6 +540,12 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
         (rc = c->alloc(&c->d_vm, H * c->m_k * kHeadDim)) || (rc = c->alloc(&c->d_om, H * c->m_q * kHeadDim)))
         return done(rc);
 
+    if (c->max_block <= 32) {   // member lists of the merged query rows; entry M_q of every head is the constant N
+        if ((rc = c->alloc(&c->d_group_start, H * (size_t)(c->m_q + 1))) || (rc = c->alloc(&c->d_group_member, H * N))) return done(rc);
+        std::vector<int32_t> gs(H * (size_t)(c->m_q + 1), 0);
+        for (size_t hd = 0; hd < H; ++hd) gs[hd * (size_t)(c->m_q + 1) + c->m_q] = c->n_tokens;
+        if ((rc = check_cuda(c, cudaMemcpy(c->d_group_start, gs.data(), gs.size() * 4, cudaMemcpyHostToDevice), "group table upload"))) return done(rc);
+    }
     if (c->big()) {
         if ((rc = c->alloc(&c->d_big_items, c->big_items.size())) || (rc = c->alloc(&c->d_inv_norm_q, H * N)) ||
             (rc = c->alloc(&c->d_inv_norm_k, H * N)) || (rc = c->alloc(&c->d_best_key_q, H * N)) || (rc = c->alloc(&c->d_best_key_k, H * N)) ||
@@ -755,6 +729,9 @@ int httm_launch_stage(httm_ctx* c, int stage, httm_tensor q, httm_tensor k, httm
         case HTTM_STAGE_UNMERGE:
             if ((rc = check_tensor(c, out, "out"))) return rc;
             return stage_unmerge(c, out, s);
+        case HTTM_STAGE_ATTENTION_UNMERGE:
+            if ((rc = check_tensor(c, out, "out"))) return rc;
+            return stage_attention(c, s, &out);
         case HTTM_STAGE_BIG_SCORES:
         case HTTM_STAGE_BIG_SELECT:
             if (!c->big()) return c->fail(HTTM_ERR_UNSUPPORTED, "the large-block stages need merging blocks of more than 256 tokens");
@@ -838,6 +815,12 @@ int httm_export(httm_ctx* c, int what, void* host_dst, size_t bytes, void* cuda_
     }
     if (!src) return c->fail(HTTM_ERR_INVALID_ARG, "export %d needs outlier filtering switched on", what);
     if (bytes != need) return c->fail(HTTM_ERR_INVALID_ARG, "export %d needs %zu bytes, got %zu", what, need, bytes);
+    if (what == HTTM_X_O_MERGED && c->om_stale) {
+        // the last call unmerged in the attention epilogue and left O_m alone: compute it now from the merged Q, K, V of that call
+        DeviceGuard guard(c->cfg.device);
+        const int rc = stage_attention(c, static_cast<cudaStream_t>(cuda_stream));
+        if (rc) return rc;
+    }
     if (host_src) {
         memcpy(host_dst, src, need);
         return HTTM_OK;

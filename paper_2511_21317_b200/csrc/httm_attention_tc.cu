@@ -31,8 +31,10 @@ constexpr int TILE_BYTES = BM * kRowBytes;   // 16 KB
 constexpr int NTHREADS = 320;   // producer warp, MMA warp, 2 x 4 softmax warps: registers are granted per four warps, so 168 per thread as with twelve
 constexpr int TMEM_COLS = 512;
 constexpr int kTableHeads = 256;   // head tables (per-head query lengths) of up to this many heads are kept in shared memory
+constexpr int kOutRowPitch = kRowBytes + 16;             // staged output rows: the pitch keeps 16-byte stores of a quarter warp on distinct banks
+constexpr int kOutStageBytes = 8 * 32 * kOutRowPitch;   // eight softmax warps x 32 output rows, staged for bulk stores
 constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row exchange*/ +
-                           (2 * kTableHeads + 4) * 4 /*head tables*/;
+                           (2 * kTableHeads + 4) * 4 /*head tables*/ + kOutStageBytes;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
 struct Barriers {
@@ -57,6 +59,9 @@ struct TcParams {
     const int32_t* mq_head;      // optional: per-head query length (then m_q is the row stride and tile_prefix the tile table)
     const int32_t* tile_prefix;
     int32_t heads;
+    const int32_t* group_start;  // optional (UNMERGE): members of every merged query row, see AttentionArgs
+    const int32_t* group_member;
+    int32_t n_tokens;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -90,10 +95,10 @@ __device__ __forceinline__ float2 exp2_poly2(float2 t) {
 // Of every eight pairs of scores, the pairs whose bit is set here take the polynomial (FMA pipe), the
 // others ex2.approx (special-function unit, 16 results per clock per SM: with every exponential there,
 // the softmax of two query tiles needs 2048 cycles against 1056 of tensor-core work).  The polynomial
-// costs about ten issue slots per pair against two, and the softmax warps are as short of issue slots as
-// of special-function throughput: measured at 10500 x 10500 x 16 heads, one pair in eight is the best
-// split (0/8: 574 us, 1/8: 540 us, 2/8: 557 us, 3/8: 587 us).
-constexpr uint32_t kPolyPairs = 0x10;   // pair 4 of 8
+// costs about ten issue slots per pair against two.  Measured at 10500 x 10500 x 16 heads with the
+// persistent kernel: 0/8: 545 us, 1/8: 510 us, 2/8: 481 us, 3/8: 497-504 us, 4/8: 570 us, 8/8: 790 us
+// (alternating 2/8 and 3/8 over the 16-column groups: 480 us).
+constexpr uint32_t kPolyPairs = 0x11;   // pairs 0 and 4 of 8
 
 // Work decomposition.  The query tiles of all heads form one list (head-major, T tiles).  With G CTAs
 // (one per SM), round r < R = T / (2 G) gives CTA c the two tiles 2 (r G + c), +1: a PAIR pass (tiles A and B
@@ -176,7 +181,59 @@ struct PassWalker {
 // once per score tile k with k mod 3 == b (2 n tiles in a pair pass, n in a single pass).
 __device__ __forceinline__ int count_mod3(int n, int r) { return (n - r + 2) / 3; }
 
-template <bool VAR>
+// Where the 32 output rows of a softmax warp go.  UNMERGE (Eq. 5-7 folded into the epilogue): row `grow` is the attention
+// output of a merged query and goes to every original token of its group, at the token's place in the final
+// [tokens][heads x 64] tensor; the first four members are fetched ahead of the epilogue, larger groups read the rest
+// of their list when they are stored.  Otherwise the row goes to row `grow` of the merged output.
+struct RowTargets {
+    int count;      // tokens this thread's row is written to (0: the row does not exist)
+    int token[4];   // the first four of them
+    int first;      // index of the group's first member in the member list
+};
+template <bool UNMERGE>
+__device__ __forceinline__ RowTargets row_targets(const TcParams& p, int head, int grow, bool valid) {
+    RowTargets t{};
+    if (!valid) return t;
+    if (!UNMERGE) {
+        t.count = 1;
+        t.token[0] = grow;
+        return t;
+    }
+    const int32_t* gs = p.group_start + (int64_t)head * (p.m_q + 1) + grow;
+    const int32_t* member = p.group_member + (int64_t)head * p.n_tokens;
+    t.first = __ldg(gs);
+    t.count = __ldg(gs + 1) - t.first;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) t.token[i] = i < t.count ? __ldg(member + t.first + i) : 0;
+    return t;
+}
+// Every lane hands in its row (eight 16-byte pieces) and its targets.  The row is staged in shared memory and leaves as
+// one 128-byte bulk copy per target token (whole lines, issued by the row's own thread: no loop over the warp's rows).
+// The copies are asynchronous: bulk_stores_done() must come before the stage is rewritten and before the kernel ends.
+__device__ __forceinline__ void bulk_stores_done() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+template <bool UNMERGE>
+__device__ __forceinline__ void store_rows(const TcParams& p, int head, const uint4 (&v)[8], const RowTargets& t, unsigned char* stage, int lane) {
+    bulk_stores_done();   // (the copies of the previous pass have long left)
+    unsigned char* row = stage + lane * kOutRowPitch;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(row + c * 16) = v[c];
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the staged row is visible to the bulk-copy engine
+    const uint32_t src = tc::smem_addr(row);
+    __nv_bfloat16* base = p.out + (int64_t)head * p.out_stride_head;
+    const int32_t* member = UNMERGE ? p.group_member + (int64_t)head * p.n_tokens + t.first : nullptr;
+    auto send = [&](int token) {
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(base + (int64_t)token * p.out_stride_token), "r"(src),
+                     "n"(kRowBytes)
+                     : "memory");
+    };
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        if (q < t.count) send(t.token[q]);
+    for (int q = 4; q < t.count; ++q) send(__ldg(member + q));
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+template <bool VAR, bool UNMERGE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const TcParams p) {
@@ -407,6 +464,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         uint32_t sp_base[3] = {0, 0, 0}, od_base = 0;   // completions before this pass: score buffers, this group's P V
         uint32_t n_single = 0;                          // single passes so far (phase of x_full / x_done)
         float2* xch = reinterpret_cast<float2*>(smem + (2 + 2 * KV_STAGES) * TILE_BYTES + 256);   // [128 rows] (max, sum) of group B
+        unsigned char* out_stage = smem + (2 + 2 * KV_STAGES) * TILE_BYTES + 256 + 1024 + (2 * kTableHeads + 4) * 4 +
+                                   (warp - 2) * 32 * kOutRowPitch;   // this warp's 32 output rows
         bool ok = true;
         for (int pass = 0; ok && walker.next(&ps); ++pass) {
             const int n_score = ps.pair ? 2 * n_tiles : n_tiles;
@@ -495,26 +554,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     tc::mbar_arrive(pbar);
                 }
                 if (ok && ps.pair) {
+                    const int grow = (ps.tile + x) * BM + row;
+                    const RowTargets targets = row_targets<UNMERGE>(p, ps.head, grow, grow < mq_rows);   // (in flight during the wait)
                     if ((ok = tc::mbar_wait(tc::smem_addr(&bars->o_final), (uint32_t)pass & 1u, abort_flag))) {
                         tc::fence_after_sync();
-                        const int grow = (ps.tile + x) * BM + row;
                         const float inv = 1.0f / l;
                         uint32_t o[64];
                         tc::tmem_ld32(t_o, o);
                         tc::tmem_ld32(t_o + 32, o + 32);
                         tc::tmem_wait_ld();
-                        if (grow < mq_rows) {
-                            uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)ps.head * p.out_stride_head + (int64_t)grow * p.out_stride_token);
+                        uint4 v[8];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                uint4 v;
-                                v.x = pack_bf16(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-                                dst[i] = v;
-                            }
+                        for (int i = 0; i < 8; ++i) {
+                            v[i].x = pack_bf16(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+                            v[i].y = pack_bf16(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+                            v[i].z = pack_bf16(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+                            v[i].w = pack_bf16(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
                         }
+                        store_rows<UNMERGE>(p, ps.head, v, targets, out_stage, lane);
                     }
                 } else if (ok && x == 1) {
                     // single pass, group B: publish this row's partial (max, sum); O_B stays in tensor memory for group A.
@@ -525,6 +582,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 } else if (ok) {
                     // single pass, group A: combine the two partial softmaxes over disjoint keys
                     //   out = (O_A 2^(m_A - m) + O_B 2^(m_B - m)) / (l_A 2^(m_A - m) + l_B 2^(m_B - m)),  m = max(m_A, m_B)
+                    const int grow = ps.tile * BM + row;
+                    const RowTargets targets = row_targets<UNMERGE>(p, ps.head, grow, grow < mq_rows);   // (in flight during the waits)
                     ok = tc::mbar_wait(tc::smem_addr(&bars->o_final), (uint32_t)pass & 1u, abort_flag) &&
                          tc::mbar_wait(tc::smem_addr(&bars->x_full), n_single & 1u, abort_flag);
                     if (ok) {
@@ -534,26 +593,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         const float fa = exp2f(m - mm), fb = exp2f(pb.x - mm);   // 2^(-inf) = 0 when group B had no key tile
                         const float inv = 1.0f / (l * fa + pb.y * fb);
                         const float wa = fa * inv, wb = fb * inv;
-                        const int grow = ps.tile * BM + row;
-                        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)ps.head * p.out_stride_head + (int64_t)grow * p.out_stride_token);
+                        uint4 v[8];
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             uint32_t oa[32], ob[32];
                             tc::tmem_ld32(t_o + half * 32, oa);
                             tc::tmem_ld32(t_o + kHeadDim + half * 32, ob);   // O_B sits right behind O_A; same TMEM lanes
                             tc::tmem_wait_ld();
-                            if (grow < mq_rows) {
 #pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    uint32_t w[4];
+                            for (int i = 0; i < 4; ++i) {
+                                uint32_t w[4];
 #pragma unroll
-                                    for (int e = 0; e < 4; ++e)
-                                        w[e] = pack_bf16(fmaf(__uint_as_float(oa[8 * i + 2 * e]), wa, __uint_as_float(ob[8 * i + 2 * e]) * wb),
-                                                         fmaf(__uint_as_float(oa[8 * i + 2 * e + 1]), wa, __uint_as_float(ob[8 * i + 2 * e + 1]) * wb));
-                                    dst[half * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
-                                }
+                                for (int e = 0; e < 4; ++e)
+                                    w[e] = pack_bf16(fmaf(__uint_as_float(oa[8 * i + 2 * e]), wa, __uint_as_float(ob[8 * i + 2 * e]) * wb),
+                                                     fmaf(__uint_as_float(oa[8 * i + 2 * e + 1]), wa, __uint_as_float(ob[8 * i + 2 * e + 1]) * wb));
+                                v[half * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
                             }
                         }
+                        store_rows<UNMERGE>(p, ps.head, v, targets, out_stage, lane);
                         tc::fence_before_sync();
                         tc::mbar_arrive(tc::smem_addr(&bars->x_done));
                     }
@@ -564,6 +621,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
             for (int b = 0; b < 3; ++b) sp_base[b] += (uint32_t)count_mod3(n_score, b);
         }
+        bulk_stores_done();
     }
     tc::fence_before_sync();
     __syncthreads();
@@ -574,9 +632,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 }  // namespace
 
 cudaError_t configure_attention() {
-    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    e = cudaFuncSetAttribute(attention_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attention_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
 }
 
 // Returns cudaErrorInvalidValue if a tensor map cannot be encoded.
@@ -591,12 +651,17 @@ cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t 
     int ctas = sm_count < 1 ? 1 : sm_count;
     if (ctas > total) ctas = total;
     const int rounds = total / (2 * ctas);
-    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, rounds, a.mq_head, a.tile_prefix, a.heads};
+    TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, rounds, a.mq_head, a.tile_prefix, a.heads,
+               a.group_start, a.group_member, a.n_tokens};
     if (a.mq_head) {   // the tile table lives in device memory: full grid, CTAs without tiles leave at once
-        attention_tc_kernel<true><<<sm_count < 1 ? 1 : sm_count, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
+        if (a.group_start) return cudaErrorInvalidValue;   // (the member lists are built for equal query lengths only)
+        attention_tc_kernel<true, false><<<sm_count < 1 ? 1 : sm_count, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
         return cudaGetLastError();
     }
-    attention_tc_kernel<false><<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
+    if (a.group_start)
+        attention_tc_kernel<false, true><<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
+    else
+        attention_tc_kernel<false, false><<<ctas, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
 

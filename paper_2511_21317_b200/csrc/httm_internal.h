@@ -102,6 +102,11 @@ struct MergeArgs {
     __nv_bfloat16* merged[3];     // Q_m [H][M_q][64], K_m, V_m [H][M_k][64]
     int32_t* rank_q;              // [H][N] merged row of every reordered token (written for Q)
     const int32_t* moff_q_var;    // optional [H][blocks]: per-head merged offsets of Q (outlier filtering); then m_q is the row stride of merged[0]
+    // optional (blocks of at most 32 tokens): the members of every merged query row, for the unmerge in the attention epilogue:
+    // group_start[h][m] .. group_start[h][m + 1] index group_member[h][], which holds ORIGINAL token numbers (pi: [N])
+    int32_t* group_start;         // [H][M_q + 1]; entry M_q (= N) is written once when the workspace is set up
+    int32_t* group_member;        // [H][N]
+    const int32_t* pi;
     const BlockInfo* blocks;
     int32_t n_blocks, n_tokens, heads, n_special_total, m_q, m_k;
     int32_t* status;
@@ -159,6 +164,11 @@ struct AttentionArgs {
     // then m_q is the row stride of q / out and an upper bound of every head's length
     const int32_t* mq_head;
     const int32_t* tile_prefix;
+    // optional (unmerge folded into the epilogue, Eq. 5-7): every merged query row is written to each of its member tokens
+    // at out + head * out_stride_head + token * out_stride_token instead of to its own row; see MergeArgs
+    const int32_t* group_start;
+    const int32_t* group_member;
+    int32_t n_tokens;
 };
 
 struct LinearArgs {   // y[n_rows][out] = x[n_rows][in] . w[out][in]^T, leading dimensions in elements

@@ -1,57 +1,30 @@
 // HBM-bound kernels of the HTTM path: temporal reorder (gather), per-(head, block)
 // cosine matching, mean merge, and unmerge + inverse reorder.  sm_100a only.
 #include "httm_internal.h"
-#include "tc_sm100.cuh"   // tensor-map encoder (host)
+#include "tc_sm100.cuh"   // mbarrier / TMA wrappers (device), tensor-map encoders (host)
 
 namespace httm {
 
 // ------------------------------------------------------------------------------------
-// small device helpers
+// small device helpers (mbarrier and address wrappers: tc_sm100.cuh)
 // ------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ uint64_t global_timer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(mbar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after about two seconds, records `code` in the status word and
-// returns false.  Never spins forever.
+using tc::mbar_expect_tx;
+using tc::mbar_init;
+using tc::mbar_try_wait;
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return tc::smem_addr(p); }
+// Bounded wait of the warp-per-block kernels: gives up after about two seconds, records `code` in the
+// status word and returns false.  Never spins forever.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity, int32_t* status, int code) {
     if (mbar_try_wait(mbar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
+    const uint64_t t0 = tc::timer_ns();
     for (;;) {
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(mbar, parity)) return true;
-        if (global_timer_ns() - t0 > 2000000000ull) {
+        if (tc::timer_ns() - t0 > 2000000000ull) {
             atomicCAS(status, kDevOk, code);
             return false;
         }
     }
-}
-// TMA bulk copy global -> this CTA's shared memory, completion on an mbarrier.
-__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t mbar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
-                 "l"(src), "r"(bytes), "r"(mbar)
-                 : "memory");
 }
 __device__ __forceinline__ void unpack8(const uint4& raw, float* f) {
     f[0] = __uint_as_float(raw.x << 16);
@@ -587,7 +560,7 @@ cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count,
 //     One warp per (tensor, head, block); kept tokens are compacted in reordered order.
 // ------------------------------------------------------------------------------------
 constexpr int kMergeTcWarps = 8;
-constexpr int kMergeTcAux = 32 * 4 + 16;   // reciprocal group sizes per kept row + 2 mbarriers
+constexpr int kMergeTcAux = 32 * 4 + 16 + 32 * 4;   // reciprocal group sizes per kept row + 2 mbarriers + group sizes / starts
 constexpr int kMergeTcSmem = kMergeTcWarps * (2 * 32 * kRowBytes + kMergeTcAux) + 1024 /*alignment slack*/;
 
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t saddr) {
@@ -613,6 +586,7 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     unsigned char* aux = smem + (size_t)kMergeTcWarps * 2 * STAGE_BYTES + (size_t)warp * kMergeTcAux;
     float* rcnt = reinterpret_cast<float*>(aux);                                        // [32] 1 / group size of kept row
     const uint32_t mbar0 = smem_u32(aux + 32 * 4), stage0 = smem_u32(stage);
+    int* gsz = reinterpret_cast<int*>(aux + 32 * 4 + 16);                               // [32] size, then first member, of kept row
 
     if (lane == 0) {
         mbar_init(mbar0, 1);
@@ -757,6 +731,10 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 o4[q] = *reinterpret_cast<const uint4*>(sb + row * kRowBytes + ((ch ^ (row & 7)) << 4));
             }
             if (t == 0 && !special && lane < n) a.rank_q[(int64_t)h * a.n_tokens + start + lane] = moff + lane;
+            if (t == 0 && a.group_start && lane < n) {   // every token is a group of its own
+                a.group_start[(int64_t)h * (a.m_q + 1) + moff + lane] = start + lane;
+                a.group_member[(int64_t)h * a.n_tokens + start + lane] = __ldg(a.pi + start + lane);
+            }
             if (has_next) target_next = load_target(meta_next);
         } else {
             // merged row of every token: rank of its representative among the kept tokens
@@ -766,6 +744,28 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (t == 0 && tok >= 0) a.rank_q[(int64_t)h * a.n_tokens + start + tok] = moff + row_of;
             const unsigned group = __match_any_sync(0xffffffffu, row_of);
             if (rep == lane) rcnt[row_of] = 1.0f / (float)__popc(group);
+            if (t == 0 && a.group_start) {
+                // member lists of the merged rows: the block's tokens group by group, kept rows in rank order
+                // (first member of row k = tokens of the rows before it: a warp scan over the group sizes)
+                if (rep == lane) gsz[row_of] = __popc(group);
+                __syncwarp();
+                const int sz = lane < n_kept ? gsz[lane] : 0;
+                int incl = sz;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, off);
+                    if (lane >= off) incl += v;
+                }
+                __syncwarp();   // every size has been read
+                if (lane < n_kept) {
+                    gsz[lane] = incl - sz;
+                    a.group_start[(int64_t)h * (a.m_q + 1) + moff + lane] = start + incl - sz;
+                }
+                __syncwarp();
+                if (tok >= 0)
+                    a.group_member[(int64_t)h * a.n_tokens + start + gsz[row_of] + __popc(group & ((1u << lane) - 1u))] =
+                        __ldg(a.pi + start + tok);
+            }
             // x fragments: for k step ks (16 tokens) and channel tile pair np, one ldmatrix.x4.trans gives
             // b0, b1 of channel tile 2 np and b0, b1 of channel tile 2 np + 1
             uint32_t bf[2][4][4];

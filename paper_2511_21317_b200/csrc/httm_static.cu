@@ -12,6 +12,7 @@
 
 #include "../../include/httm.h"
 #include "httm_internal.h"
+#include "httm_plan.h"
 
 namespace httm {
 void set_global_error(const std::string& msg);   // defined next to httm_last_error
@@ -28,6 +29,10 @@ struct DeviceSetup {
     bool ready = false;
     unsigned char* base = nullptr;   // device address of g_static_scratch on this device
     int sm_count = 0;
+    // the configuration whose plan tables (pi, pi_inv, block table) the array holds on this device: a call that
+    // repeats it uploads nothing
+    bool tables_resident = false;
+    httm_config resident{};
 };
 DeviceSetup g_setup[kMaxDevices];
 std::mutex g_mutex;
@@ -35,9 +40,7 @@ std::mutex g_mutex;
 struct StaticPlan {   // host copy of the plan of the last geometry (rebuilt when the config changes)
     httm_config cfg{};
     bool valid = false;
-    int32_t n_tokens = 0, n_special_total = 0, n_blocks = 0, max_block = 0, m_q = 0, m_k = 0;
-    std::vector<int32_t> pi, pi_inv;
-    std::vector<BlockInfo> blocks;
+    HostPlan plan;
 };
 StaticPlan g_plan;
 
@@ -46,59 +49,10 @@ int fail(int code, const std::string& msg) {
     return code;
 }
 
-void budget(int n, double ratio, int32_t* r, int32_t* nd) {
-    int64_t rr = (int64_t)std::floor(ratio * (double)n + 1e-9);
-    rr = std::max<int64_t>(0, std::min<int64_t>(rr, n - 1));
-    int64_t d = std::min<int64_t>((n + 3) / 4, n - rr);
-    *r = (int32_t)rr;
-    *nd = (int32_t)d;
-}
-
 bool same_config(const httm_config& a, const httm_config& b) {
     return a.frames == b.frames && a.n_camera == b.n_camera && a.n_register == b.n_register && a.grid_h == b.grid_h &&
            a.grid_w == b.grid_w && a.heads == b.heads && a.head_dim == b.head_dim && a.blk_frames == b.blk_frames &&
            a.blk_h == b.blk_h && a.blk_w == b.blk_w && a.ratio_q == b.ratio_q && a.ratio_kv == b.ratio_kv;
-}
-
-void build_plan(const httm_config& cfg, StaticPlan* p) {
-    p->cfg = cfg;
-    const int nsp = cfg.n_camera + cfg.n_register, S = cfg.frames, h = cfg.grid_h, w = cfg.grid_w;
-    const int P = nsp + h * w;
-    p->n_tokens = S * P;
-    p->n_special_total = S * nsp;
-    p->pi.assign(p->n_tokens, 0);
-    p->pi_inv.assign(p->n_tokens, 0);
-    p->blocks.clear();
-    p->max_block = 0;
-    int32_t pos = 0;
-    for (int s = 0; s < S; ++s)
-        for (int j = 0; j < nsp; ++j) p->pi[pos++] = s * P + j;
-    int32_t mq = pos, mk = pos;
-    for (int g0 = 0; g0 < S; g0 += cfg.blk_frames)
-        for (int y0 = 0; y0 < h; y0 += cfg.blk_h)
-            for (int x0 = 0; x0 < w; x0 += cfg.blk_w) {
-                const int f = std::min(cfg.blk_frames, S - g0), hh = std::min(cfg.blk_h, h - y0), ww = std::min(cfg.blk_w, w - x0);
-                BlockInfo bi{};
-                bi.start = pos;
-                bi.n = f * hh * ww;
-                bi.n_rule = bi.n;
-                budget(bi.n, cfg.ratio_q, &bi.r_q, &bi.nd_q);
-                budget(bi.n, cfg.ratio_kv, &bi.r_k, &bi.nd_k);
-                bi.moff_q = mq;
-                bi.moff_k = mk;
-                mq += bi.n - bi.r_q;
-                mk += bi.n - bi.r_k;
-                p->max_block = std::max(p->max_block, bi.n);
-                p->blocks.push_back(bi);
-                for (int tl = 0; tl < f; ++tl)
-                    for (int yl = 0; yl < hh; ++yl)
-                        for (int xl = 0; xl < ww; ++xl) p->pi[pos++] = (g0 + tl) * P + nsp + (y0 + yl) * w + (x0 + xl);
-            }
-    p->n_blocks = (int32_t)p->blocks.size();
-    p->m_q = mq;
-    p->m_k = mk;
-    for (int32_t i = 0; i < p->n_tokens; ++i) p->pi_inv[p->pi[i]] = i;
-    p->valid = true;
 }
 
 // The array keeps whatever the previous call left in it.  What the kernels do not rewrite on every
@@ -119,13 +73,9 @@ __global__ void static_reset_kernel(int32_t* status, int32_t* assign_q, int32_t*
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 int check_tensor(const httm_tensor& t, int heads, const char* name) {
-    if (!t.ptr) return fail(HTTM_ERR_INVALID_ARG, std::string(name) + ": null pointer");
-    if (((uintptr_t)t.ptr & 15u) != 0) return fail(HTTM_ERR_ALIGNMENT, std::string(name) + ": pointer is not 16-byte aligned");
-    if (t.stride_head % 8 != 0 || t.stride_token % 8 != 0)
-        return fail(HTTM_ERR_ALIGNMENT, std::string(name) + ": strides must be multiples of 8 elements");
-    if (t.stride_token < kHeadDim || t.stride_head < 0 || (heads > 1 && t.stride_head < kHeadDim))
-        return fail(HTTM_ERR_INVALID_ARG, std::string(name) + ": strides smaller than head_dim");
-    return HTTM_OK;
+    std::string why;
+    const int rc = check_tensor_layout(t, heads, name, &why);
+    return rc == HTTM_OK ? rc : fail(rc, why);
 }
 
 }  // namespace
@@ -133,12 +83,11 @@ int check_tensor(const httm_tensor& t, int heads, const char* name) {
 extern "C" int httm_global_attention_static(const httm_config* cfg, httm_tensor q, httm_tensor k, httm_tensor v,
                                             httm_tensor out, void* cuda_stream) {
     if (!cfg) return fail(HTTM_ERR_INVALID_ARG, "null config");
-    if (cfg->frames < 1 || cfg->n_camera < 0 || cfg->n_register < 0 || cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->heads < 1 ||
-        cfg->blk_frames < 1 || cfg->blk_h < 1 || cfg->blk_w < 1)
-        return fail(HTTM_ERR_INVALID_ARG, "sizes must be positive (special-token counts non-negative)");
-    if (!(cfg->ratio_q >= 0.0 && cfg->ratio_q < 1.0) || !(cfg->ratio_kv >= 0.0 && cfg->ratio_kv < 1.0))
-        return fail(HTTM_ERR_INVALID_ARG, "merge ratios must lie in [0, 1)");
-    if (cfg->head_dim != kHeadDim) return fail(HTTM_ERR_UNSUPPORTED, "head_dim must be 64");
+    {
+        std::string why;
+        const int rc = check_config(*cfg, &why);
+        if (rc != HTTM_OK) return fail(rc, why);
+    }
     if (cfg->device < 0 || cfg->device >= kMaxDevices) return fail(HTTM_ERR_INVALID_ARG, "device ordinal out of range");
     const int64_t bf = std::min(cfg->blk_frames, cfg->frames), bh = std::min(cfg->blk_h, cfg->grid_h),
                   bw = std::min(cfg->blk_w, cfg->grid_w);
@@ -187,8 +136,14 @@ extern "C" int httm_global_attention_static(const httm_config* cfg, httm_tensor 
         ds.sm_count = prop.multiProcessorCount;
         ds.ready = true;
     }
-    if (!g_plan.valid || !same_config(g_plan.cfg, *cfg)) build_plan(*cfg, &g_plan);
-    const StaticPlan& pl = g_plan;
+    if (!g_plan.valid || !same_config(g_plan.cfg, *cfg)) {
+        g_plan.valid = false;
+        build_host_plan(*cfg, &g_plan.plan);
+        g_plan.cfg = *cfg;
+        g_plan.valid = true;
+    }
+    const HostPlan& pl = g_plan.plan;
+    const int32_t n_special_total = cfg->frames * pl.n_special;
     const size_t N = pl.n_tokens, Hh = cfg->heads;
 
     // carve the array
@@ -217,15 +172,24 @@ extern "C" int httm_global_attention_static(const httm_config* cfg, httm_tensor 
                                               std::to_string(kStaticScratchBytes) + "; use httm_create + httm_global_attention");
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = cudaMemcpyAsync(d_pi, pl.pi.data(), N * 4, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(d_pi_inv, pl.pi_inv.data(), N * 4, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess && !pl.blocks.empty())
-        e = cudaMemcpyAsync(d_blocks, pl.blocks.data(), pl.blocks.size() * sizeof(BlockInfo), cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(e, "plan upload");
+    cudaError_t e = cudaSuccess;
+    if (!ds.tables_resident || !same_config(ds.resident, *cfg)) {
+        // The plan tables of another configuration (or none) are in the array: upload this one's, in stream order
+        // behind whatever earlier calls enqueued on this stream.  Calls that repeat the resident configuration skip
+        // this and enqueue kernels only.
+        ds.tables_resident = false;
+        e = cudaMemcpyAsync(d_pi, pl.pi.data(), N * 4, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d_pi_inv, pl.pi_inv.data(), N * 4, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess && !pl.blocks.empty())
+            e = cudaMemcpyAsync(d_blocks, pl.blocks.data(), pl.blocks.size() * sizeof(BlockInfo), cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(e, "plan upload");
+        ds.resident = *cfg;
+        ds.tables_resident = true;
+    }
     {
-        const int threads = 256, work = std::max<int>(1, (int)Hh * pl.n_special_total);
+        const int threads = 256, work = std::max<int>(1, (int)Hh * n_special_total);
         static_reset_kernel<<<(work + threads - 1) / threads, threads, 0, s>>>(d_status, d_aq, d_ak, d_rq, pl.n_tokens,
-                                                                             pl.n_special_total, (int)Hh);
+                                                                             n_special_total, (int)Hh);
         if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "reset launch");
     }
     auto tv = [](const httm_tensor& t) { return TensorView{reinterpret_cast<const __nv_bfloat16*>(t.ptr), t.stride_head, t.stride_token}; };
@@ -245,7 +209,7 @@ extern "C" int httm_global_attention_static(const httm_config* cfg, httm_tensor 
     ga.xr[0] = d_qr; ga.xr[1] = d_kr; ga.xr[2] = d_vr; ga.assign[0] = d_aq; ga.assign[1] = d_ak;
     ga.merged[0] = d_qm; ga.merged[1] = d_km; ga.merged[2] = d_vm; ga.rank_q = d_rq;
     ga.blocks = d_blocks; ga.n_blocks = pl.n_blocks; ga.n_tokens = pl.n_tokens; ga.heads = cfg->heads;
-    ga.n_special_total = pl.n_special_total; ga.m_q = pl.m_q; ga.m_k = pl.m_k; ga.status = d_status;
+    ga.n_special_total = n_special_total; ga.m_q = pl.m_q; ga.m_k = pl.m_k; ga.status = d_status;
     if ((e = launch_merge(ga, pl.max_block, ds.sm_count, s)) != cudaSuccess) return cuda_fail(e, "merge launch");
 
     AttentionArgs aa{};

@@ -3,8 +3,8 @@
     python -m paper_2511_21317_b200.run_layer --workload medium --calls 2 [--dense 1] [--stages 1] [--ratio 0.9] [--block 4x4x4]
                                               [--outlier-fraction 0.01]
 
-A profiler is pointed at this command: few launches, no timing loops, no CPU work besides
-the input generator.  It prints the merged lengths and the device status word, and exits
+A profiler is pointed at this command (the ncu summaries under profiles/ name it): few launches, no timing loops,
+no CPU work besides the input generator.  It is not needed to use the library.  It prints the merged lengths and the device status word, and exits
 non-zero if the status word is set.
 """
 from __future__ import annotations
@@ -24,8 +24,8 @@ def main() -> int:
     ap.add_argument("--calls", type=int, default=2, help="httm_global_attention calls")
     ap.add_argument("--dense", type=int, default=0, help="httm_dense_attention calls")
     ap.add_argument("--stages", type=int, default=0, help="rounds of every kernel launched on its own (reorder, match, merge, "
-                    "match and merge with direct block loads, attention, unmerge; for large blocks reorder, scores, select, "
-                    "merge, attention, unmerge)")
+                    "match and merge with direct block loads, attention, unmerge, and - blocks of at most 32 tokens - attention "
+                    "with the unmerge in its epilogue; for large blocks reorder, scores, select, merge, attention, unmerge)")
     ap.add_argument("--heads", type=int, default=None, help="override the number of heads")
     ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
     ap.add_argument("--block", default=None, help="override the block shape, e.g. 4x4x4")
@@ -52,9 +52,13 @@ def main() -> int:
         for _ in range(args.dense):
             ctx.dense_attention(dq, dk, dv, out)
         ctx.set_outlier_fraction(0.0)
-        big = ctx.query(hb.Q_MAX_BLOCK_TOKENS) > 256   # large blocks: reorder (+ norms), scores, select, merge, attention, unmerge
+        max_block = ctx.query(hb.Q_MAX_BLOCK_TOKENS)
+        big = max_block > 256   # large blocks: reorder (+ norms), scores, select, merge, attention, unmerge
+        order = [0, 8, 9, 2, 3, 4] if big else [0, 1, 2, 5, 6, 3, 4]
+        if max_block <= 32:
+            order.append(hb.STAGE_ATTENTION_UNMERGE)   # attention with the unmerge in its epilogue (what the public call runs)
         for _ in range(args.stages):
-            for st in ([0, 8, 9, 2, 3, 4] if big else [0, 1, 2, 5, 6, 3, 4]):
+            for st in order:
                 ctx.launch_stage(st, dq, dk, dv, out)
         torch.cuda.synchronize()
         status = ctx.query(hb.Q_DEVICE_STATUS)

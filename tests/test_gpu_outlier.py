@@ -107,7 +107,7 @@ def test_switching_the_filter_off_restores_the_plain_path():
         before = ctx.launch_count()
         again = ctx.global_attention(dq, dk, dv)
         torch.cuda.synchronize()
-        assert ctx.launch_count() - before == 4
+        assert ctx.launch_count() - before == 3          # match, merge, attention with the unmerge in its epilogue
         assert torch.equal(plain, again)
         assert ctx.export(hb.X_Q_MERGED).shape == (wl.heads, ctx.m_q, 64)
 

@@ -187,6 +187,50 @@ def test_stage_calls_equal_the_fused_call_and_host_entry_point():
         assert torch.equal(hout, dref.cpu())
 
 
+def test_unmerge_in_the_attention_epilogue_equals_the_separate_kernels():
+    """With blocks of at most 32 tokens the public call is three kernels: the attention epilogue writes every merged query
+    row to its member tokens (Eq. 5-7).  Same bits as attention -> O_m -> unmerge kernel, for clipped blocks, scenes that go
+    over the reordered copies (many special tokens), single-token blocks, ratio 0, and a head-major output."""
+    cases = [synth.WORKLOADS["tiny"].replace(heads=3),
+             synth.Workload("fused_clipped", 5, 9, 10, 2, 4, 4, 0.6, 0.7, heads=3, seed=7),
+             synth.Workload("fused_specials", 3, 6, 6, 2, 4, 4, 0.5, 0.5, heads=2, n_camera=1, n_register=44, seed=8),
+             synth.Workload("fused_single_tokens", 2, 3, 3, 1, 1, 1, 0.9, 0.9, heads=2, n_camera=1, n_register=0, seed=9),
+             synth.Workload("fused_ratio_zero", 3, 7, 9, 2, 4, 4, 0.0, 0.5, heads=2, seed=10),
+             synth.WORKLOADS["small"].replace(heads=2)]
+    for wl in cases:
+        q, k, v = synth.make_qkv(wl)
+        H, N = wl.heads, wl.n_tokens
+        with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+            dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+            direct = wl.n_camera + wl.n_register <= 32
+            n0 = ctx.launch_count()
+            fused = ctx.global_attention(dq, dk, dv)
+            torch.cuda.synchronize()
+            assert ctx.launch_count() - n0 == (3 if direct else 4), wl.name
+            with pytest.raises(hb.HttmError) as e:      # O_m of that call was never written
+                ctx.launch_stage(hb.STAGE_UNMERGE, dq, dk, dv, ctx.new_output())
+            assert e.value.code == hb.ERR_INVALID_ARG
+            o_m = ctx.export(hb.X_O_MERGED)              # ... and is computed on request
+            rank_q, pi_inv = ctx.export(hb.X_RANK_Q), ctx.export(hb.X_PI_INV)
+            bits = hb.bits_from_bf16(fused)
+            for hd in range(H):
+                assert np.array_equal(bits[:, hd * 64:(hd + 1) * 64], o_m[hd][rank_q[hd][pi_inv]]), f"{wl.name}: head {hd}"
+            sep = ctx.new_output().fill_(float("nan"))
+            stages = (hb.STAGE_MATCH_DIRECT, hb.STAGE_MERGE_DIRECT) if direct else (hb.STAGE_REORDER, hb.STAGE_MATCH, hb.STAGE_MERGE)
+            for st in stages + (hb.STAGE_ATTENTION, hb.STAGE_UNMERGE):
+                ctx.launch_stage(st, dq, dk, dv, sep)
+            again = ctx.new_output().fill_(float("nan"))
+            ctx.launch_stage(hb.STAGE_ATTENTION_UNMERGE, dq, dk, dv, again)
+            out_hm = torch.full((H, N, 64), float("nan"), dtype=torch.bfloat16, device=DEV)    # head-major output
+            rc = ctx._lib.httm_global_attention(ctx._h, ctx._tensor(dq, "q"), ctx._tensor(dk, "k"), ctx._tensor(dv, "v"),
+                                                hb._Tensor(out_hm.data_ptr(), N * 64, 64), ctx._stream(None))
+            assert rc == 0
+            torch.cuda.synchronize()
+            assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+            assert torch.equal(fused, sep) and torch.equal(fused, again), wl.name
+            assert torch.equal(out_hm.permute(1, 0, 2).reshape(N, H * 64), fused), wl.name
+
+
 def test_argument_errors_are_reported_before_any_launch():
     wl = synth.WORKLOADS["tiny"].replace(heads=2)
     with hb.Httm(hb.HttmConfig.of(wl)) as ctx:

@@ -51,6 +51,42 @@ def test_static_scratch_entry_matches_context_entry_twice_in_a_row():
             assert torch.equal(out, ref), (wl.name, rep)        # same kernels, same order: bit-identical
 
 
+def test_static_scratch_entry_with_larger_blocks_after_a_smaller_geometry():
+    """Blocks of 64 and 128 tokens (the kernels that take a block in several passes), each run right after the tiny
+    32-token case has left its data in the shared array, and clipped at the grid edge."""
+    tiny = synth.WORKLOADS["tiny"]
+    tq, tk, tv = (hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(tiny))
+    tout = torch.empty(tiny.n_tokens, tiny.heads * 64, dtype=torch.bfloat16, device=DEV)
+    for wl in (synth.Workload("static_64", 6, 9, 10, 4, 4, 4, 0.6, 0.8, heads=3, seed=11),
+               synth.Workload("static_128", 3, 17, 19, 2, 8, 8, 0.7, 0.5, heads=2, seed=12)):
+        q, k, v = (hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(wl))
+        ref = reference(wl, q, k, v)
+        out = torch.full((wl.n_tokens, wl.heads * 64), float("nan"), dtype=torch.bfloat16, device=DEV)
+        hb.global_attention_static(hb.HttmConfig.of(tiny), tq, tk, tv, tout)
+        hb.global_attention_static(hb.HttmConfig.of(wl), q, k, v, out)
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref), wl.name
+
+
+def test_static_scratch_entry_repeated_configuration_enqueues_kernels_only():
+    """A call that repeats the configuration resident in the array copies nothing from the host, so it returns while
+    earlier work on the stream is still running (a pageable host-to-device copy would wait for it)."""
+    wl = synth.Workload("static_b", 3, 9, 11, 2, 4, 4, 0.7, 0.5, heads=4, n_camera=1, n_register=2, seed=9)
+    q, k, v = (hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(wl))
+    ref = reference(wl, q, k, v)
+    out = torch.empty(wl.n_tokens, wl.heads * 64, dtype=torch.bfloat16, device=DEV)
+    cfg = hb.HttmConfig.of(wl)
+    hb.global_attention_static(cfg, q, k, v, out)          # makes this configuration the resident one
+    torch.cuda.synchronize()
+    out.fill_(float("nan"))
+    torch.cuda._sleep(400_000_000)                          # about 0.2 s of GPU time ahead of the call on the same stream
+    hb.global_attention_static(cfg, q, k, v, out)
+    still_busy = not torch.cuda.current_stream().query()
+    torch.cuda.synchronize()
+    assert still_busy, "the call waited for earlier work on the stream"
+    assert torch.equal(out, ref)
+
+
 def test_static_scratch_entry_against_the_oracle():
     """Directly against the CPU oracle (not only through the context entry): output within 2e-2 x RMS on the tiny scene."""
     wl = synth.WORKLOADS["tiny"]
@@ -69,4 +105,14 @@ def test_static_scratch_entry_rejects_what_does_not_fit():
     with pytest.raises(hb.HttmError) as e:
         hb.global_attention_static(hb.HttmConfig.of(wl), q, q.clone(), q.clone(), out)
     assert e.value.code == hb.ERR_UNSUPPORTED and "static scratch" in str(e.value)
+    assert torch.count_nonzero(out).item() == 0
+    # a problem that passes the first size estimate (Q, K, V alone would fit) but not the exact layout of the array
+    wl = synth.Workload("static_carve", 1, 200, 200, 1, 4, 4, 0.0, 0.0, heads=1)
+    assert wl.n_tokens * 384 < 16 << 20
+    q = torch.zeros(1, wl.n_tokens, 64, dtype=torch.bfloat16, device=DEV)
+    out = torch.zeros(wl.n_tokens, 64, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(hb.HttmError) as e:
+        hb.global_attention_static(hb.HttmConfig.of(wl), q, q.clone(), q.clone(), out)
+    assert e.value.code == hb.ERR_UNSUPPORTED and "bytes of scratch" in str(e.value)
+    torch.cuda.synchronize()
     assert torch.count_nonzero(out).item() == 0
