@@ -63,9 +63,10 @@ typedef struct {
                                      frame 0 and every other token of the block is a src token, so the reference frame is
                                      never merged away and similar tokens of later frames merge INTO it; there the budget
                                      is r = min(floor(ratio*n + 1e-9), n - n0) with n0 the block's tokens of frame 0.
-                                     UNSUPPORTED where n0 exceeds what the match kernels hold (a quarter of the largest
-                                     block: blocks of up to 256 tokens need at least 4 frames per block) and in
-                                     httm_global_attention_static.  (The field takes the struct's former padding.)  */
+                                     Any block shape of up to 256 tokens is accepted (blocks of one frame then merge
+                                     nothing in the first frame group); blocks of more than 256 tokens may hold at most
+                                     1024 tokens of frame 0 (UNSUPPORTED otherwise), and httm_global_attention_static
+                                     has no anchoring.  (The field takes the struct's former padding.)  */
 } httm_config;
 
 typedef struct {

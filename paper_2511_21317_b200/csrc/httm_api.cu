@@ -51,6 +51,9 @@ struct httm_ctx {
     // path, so O_m does not hold its attention output (httm_export recomputes it on request).
     int32_t *d_group_start = nullptr, *d_group_member = nullptr;
     bool om_stale = false;
+    // first-frame anchoring: blocks of the first frame group (the first n_anchor blocks) with more dst tokens than the
+    // match kernel holds (match_capacity) are matched by a kernel of their own, launched behind it
+    int32_t n_anchor = 0, match_capacity = 0;
     // query outlier filtering (Sec. 3.4): off while fraction == 0; its workspace is allocated when it is first switched on.
     // The merged query length then differs per head: Q_m and O_m get N rows per head.
     double outlier_fraction = 0.0;
@@ -257,7 +260,13 @@ int stage_match(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
     a.heads = c->cfg.heads;
     a.status = c->d_status;
     c->launches++;
-    return check_cuda(c, launch_match(a, c->max_block, c->sm_count, s), "match launch");
+    int rc = check_cuda(c, launch_match(a, c->max_block, c->sm_count, s), "match launch");
+    if (rc || c->n_anchor == 0) return rc;
+    c->launches++;
+    if (src)
+        return check_cuda(c, launch_match_anchor(a, view(src[0]), view(src[1]), c->d_pi, c->n_anchor, c->match_capacity, c->max_block, s), "anchor match launch");
+    return check_cuda(c, launch_match_anchor(a, view(c->d_qr, c->n_tokens), view(c->d_kr, c->n_tokens), nullptr, c->n_anchor, c->match_capacity, c->max_block, s),
+                      "anchor match launch");
 }
 
 int stage_merge(httm_ctx* c, cudaStream_t s, const httm_tensor* src = nullptr) {
@@ -502,11 +511,17 @@ int httm_create(const httm_config* cfg, httm_ctx** out) {
         for (int32_t b = 0; b < c->n_blocks; ++b)
             for (int row0 = 0; row0 < c->blocks[b].n; row0 += kBigSliceRows) c->big_items.push_back(BigItem{b, row0});
     }
-    {   // the match kernels hold a quarter of their largest block as dst tokens (the large-block path 1024)
+    {   // the match kernels hold a quarter of their largest block as dst tokens (the large-block path 1024); anchored blocks of
+        // up to 256 tokens with more (two or three frames per block) go to a kernel of their own
         const int cap = c->max_block > kMaxBlockTokens ? kMaxBigDst : (c->max_block <= 32 ? 8 : (c->max_block <= 64 ? 16 : (c->max_block <= 128 ? 32 : 64)));
+        c->match_capacity = cap;
         if (anchored_nd_max > cap) {
-            delete c;
-            return bad(HTTM_ERR_UNSUPPORTED, "first-frame anchoring: a block's tokens of frame 0 exceed a quarter of the largest block (use more frames per block)");
+            if (c->max_block > kMaxBlockTokens) {
+                delete c;
+                return bad(HTTM_ERR_UNSUPPORTED, "first-frame anchoring: blocks of more than 256 tokens may hold at most 1024 tokens of frame 0");
+            }
+            const int64_t groups = (cfg->frames + cfg->blk_frames - 1) / cfg->blk_frames;
+            c->n_anchor = (int32_t)(c->n_blocks / groups);   // the blocks of the first frame group come first
         }
     }
     DeviceGuard guard(cfg->device);

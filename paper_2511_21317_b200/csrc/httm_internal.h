@@ -182,6 +182,10 @@ struct LinearArgs {   // y[n_rows][out] = x[n_rows][in] . w[out][in]^T, leading 
 // Launchers (each enqueues exactly one kernel on `stream`; returns the CUDA error).
 cudaError_t launch_reorder(const ReorderArgs& a, cudaStream_t stream);
 cudaError_t launch_match(const MatchArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
+// first-frame anchoring: the blocks of the first frame group (the first n_anchor blocks) whose dst tokens exceed main_capacity,
+// from the original tensors through the reorder index pi
+cudaError_t launch_match_anchor(const MatchArgs& a, const TensorView& src_q, const TensorView& src_k, const int32_t* pi, int n_anchor,
+                                int main_capacity, int max_block_tokens, cudaStream_t stream);
 cudaError_t launch_merge(const MergeArgs& a, int max_block_tokens, int sm_count, cudaStream_t stream);
 cudaError_t launch_unmerge(const UnmergeArgs& a, cudaStream_t stream);
 cudaError_t launch_deviation(const OutlierArgs& a, int sm_count, cudaStream_t stream);

@@ -304,6 +304,11 @@ match_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ 
             if (more && lane == 0) issue(nxt, buf);
             continue;
         }
+        if (nd > NT * 8) {   // first-frame anchoring with more dst tokens than a quarter of the largest block: match_anchor_kernel
+            __syncwarp();
+            if (more && lane == 0) issue(nxt, buf);
+            continue;
+        }
         // floor(x / n) and floor(x / n_dst) by multiplication: exact for the operand ranges below (n <= 256, n_dst <= 64)
         const int n_rule = bi.n_rule;   // n (evenly spaced dst tokens) or n_dst (the first n_dst tokens: first-frame anchoring)
         if (n_rule != cached_n || nd != cached_nd) {
@@ -539,6 +544,99 @@ static cudaError_t launch_match_t(const MatchArgs& a, int sm_count, cudaStream_t
         match_kernel<PASSES, true><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
     else
         match_kernel<PASSES, false><<<(unsigned)grid, WARPS * 32, smem, stream>>>(mq, mk, a);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------
+// a2 under first-frame anchoring (the paper's appendix on error mitigation: all tokens of frame 0 are dst tokens), for the
+//     blocks of the first frame group whose dst tokens exceed what match_kernel holds (a quarter of the largest block:
+//     blocks of two or three frames).  Same rule, plain formulation: one CTA per (tensor, head, block), the block's rows
+//     gathered through the reorder index into shared memory, inverse norms, for every src token the dot products with
+//     the dst tokens (the block's first n_dst tokens) by fp32 FMAs on exact bf16 products, best dst (ties: lowest),
+//     then the r best src by rank counting (ties: lowest position).  These blocks are 1 / (frame groups) of the scene.
+// ------------------------------------------------------------------------------------
+constexpr int kAnchorThreads = 128;
+constexpr int kAnchorPitch = kRowBytes + 16;   // row pitch in shared memory: 16-byte accesses of neighbouring rows on distinct banks
+__host__ __device__ constexpr int anchor_smem_bytes(int nmax) { return nmax * (kAnchorPitch + 12); }   // rows, inverse norms, scores, best dst
+
+__global__ void __launch_bounds__(kAnchorThreads) match_anchor_kernel(const MatchArgs a, const TensorView src_q, const TensorView src_k,
+                                                                       const int32_t* __restrict__ pi, int n_anchor, int main_capacity, int nmax) {
+    extern __shared__ __align__(16) unsigned char sm_anchor[];
+    const int task = blockIdx.x;
+    const int b = task % n_anchor, h = (task / n_anchor) % a.heads, t = task / (n_anchor * a.heads);
+    const BlockInfo bi = a.blocks[b];
+    const int n = bi.n, nd = t == 0 ? bi.nd_q : bi.nd_k, r = t == 0 ? bi.r_q : bi.r_k;
+    if (bi.n_rule == n || nd <= main_capacity || r == 0 || n > nmax) return;   // match_kernel has written this block's map
+    unsigned char* rows = sm_anchor;
+    float* inv = reinterpret_cast<float*>(sm_anchor + (size_t)nmax * kAnchorPitch);
+    float* score = inv + nmax;
+    int* best = reinterpret_cast<int*>(score + nmax);
+    const TensorView& sv = t == 0 ? src_q : src_k;
+    const __nv_bfloat16* base = sv.ptr + (int64_t)h * sv.stride_head;
+    for (int q = threadIdx.x; q < n * 8; q += kAnchorThreads) {
+        const int row = q >> 3, c = q & 7;
+        const int64_t orig = pi ? __ldg(pi + bi.start + row) : bi.start + row;   // (no index: the tensors are the reordered copies)
+        *reinterpret_cast<uint4*>(rows + row * kAnchorPitch + c * 16) = __ldg(reinterpret_cast<const uint4*>(base + orig * sv.stride_token + c * 8));
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < n; j += kAnchorThreads) {
+        float ss = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            float x[8];
+            unpack8(*reinterpret_cast<const uint4*>(rows + j * kAnchorPitch + c * 16), x);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ss = fmaf(x[e], x[e], ss);
+        }
+        inv[j] = fminf(rsqrtf(ss), 1e12f);   // 1 / max(|x|, 1e-12)
+    }
+    __syncthreads();
+    for (int j = nd + threadIdx.x; j < n; j += kAnchorThreads) {   // src tokens: everything behind the block's tokens of frame 0
+        float xs[64];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) unpack8(*reinterpret_cast<const uint4*>(rows + j * kAnchorPitch + c * 16), xs + 8 * c);
+        float top = -INFINITY;
+        int arg = 0;
+        for (int d = 0; d < nd; ++d) {
+            float dot = 0.f;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                float xd[8];
+                unpack8(*reinterpret_cast<const uint4*>(rows + d * kAnchorPitch + c * 16), xd);   // (the same row for every thread: a broadcast)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) dot = fmaf(xs[8 * c + e], xd[e], dot);
+            }
+            const float sim = dot * inv[d];
+            if (sim > top) {
+                top = sim;
+                arg = d;
+            }
+        }
+        score[j] = top * inv[j];
+        best[j] = arg;
+    }
+    __syncthreads();
+    int32_t* A = a.assign[t] + (int64_t)h * a.n_tokens + bi.start;
+    for (int j = threadIdx.x; j < n; j += kAnchorThreads) {
+        if (j < nd) {
+            A[j] = bi.start + j;
+            continue;
+        }
+        const uint32_t key = score_key(score[j]);
+        int rank = 0;   // src tokens that come before this one: better score, or the same score at a lower position
+        for (int i = nd; i < n; ++i) {
+            const uint32_t ki = score_key(score[i]);
+            rank += (ki > key || (ki == key && i < j)) ? 1 : 0;
+        }
+        A[j] = bi.start + (rank < r ? best[j] : j);
+    }
+}
+
+cudaError_t launch_match_anchor(const MatchArgs& a, const TensorView& src_q, const TensorView& src_k, const int32_t* pi, int n_anchor,
+                                int main_capacity, int max_block_tokens, cudaStream_t stream) {
+    if (n_anchor <= 0) return cudaSuccess;
+    const int nmax = max_block_tokens < kMaxBlockTokens ? max_block_tokens : kMaxBlockTokens;
+    match_anchor_kernel<<<2 * a.heads * n_anchor, kAnchorThreads, anchor_smem_bytes(nmax), stream>>>(a, src_q, src_k, pi, n_anchor, main_capacity, nmax);
     return cudaGetLastError();
 }
 
@@ -929,7 +1027,7 @@ merge_multi_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (DIRECT) {   // stage rows that no block load writes enter the MMAs with weight 0: they must hold finite values
         for (int q = box_rows * 8 + lane; q < NMAX * 8; q += 32) {   // (a load of special tokens may overwrite some of them later)
             *reinterpret_cast<uint4*>(stage + q * 16) = make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(stage + STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+            if (STAGES == 2) *reinterpret_cast<uint4*>(stage + STAGE_BYTES + q * 16) = make_uint4(0u, 0u, 0u, 0u);   // (one stage: there is no second buffer)
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
