@@ -221,6 +221,14 @@ def rank_max(x, world, device="cpu"):
     return float(t.item())
 
 
+def head_shard(rank, world, heads):
+    """(first head, number of heads) of rank `rank` when the heads of one layer are dealt to `world` GPUs."""
+    if heads % world != 0:
+        raise SystemExit(f"bench.py --shard heads: {heads} heads do not divide over {world} GPUs")
+    per = heads // world
+    return rank * per, per
+
+
 def replica_throughput(tokens_per_replica, world, ms_step):
     """Whole-job tokens/s of `world` independent replicas timed at `ms_step` (the maximum over the replicas)."""
     return world * tokens_per_replica / (ms_step * 1e-3)
@@ -249,11 +257,22 @@ def run_ours(args, wl):
         return rank_max(x, world, dev)
 
     q, k, v = synth.make_qkv(wl)
+    # --shard heads: ONE layer over all GPUs, rank g owns heads [g H / G, (g + 1) H / G) through head-strided views and
+    # writes its column slice of the output; no kernel touches another rank's data and the layer exchanges nothing
+    # (with outlier filtering on: the three threshold histograms, see filtered_variant)
+    shard = args.shard == "heads" and world > 1
+    layer_heads = wl.heads
+    h0, hl = head_shard(rank, world, wl.heads) if shard else (0, wl.heads)
+    if shard:
+        q, k, v = (np.ascontiguousarray(x[h0:h0 + hl]) for x in (q, k, v))
+        wl = wl.replace(heads=hl)
     ctx = hb.Httm(hb.HttmConfig.of(wl, device=local))
     dq, dk, dv = (hb.bf16_from_bits(x, dev) for x in (q, k, v))
-    out = ctx.new_output()
+    out_layer = torch.empty(wl.n_tokens, layer_heads * wl.head_dim, dtype=torch.bfloat16, device=dev)
+    out = out_layer[:, h0 * wl.head_dim:(h0 + hl) * wl.head_dim]   # (the whole tensor unless sharded)
     stream = torch.cuda.current_stream()
     N, H, D, Mq, Mk = wl.n_tokens, wl.heads, wl.head_dim, ctx.m_q, ctx.m_k
+    jobs = 1 if shard else world   # layers in flight: one sharded layer, or one replica per GPU
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -319,7 +338,7 @@ def run_ours(args, wl):
 
     # ---- dense baseline of the same run (same attention kernel on the unmerged tokens)
     dsteps = max(3, min(args.steps, 10))
-    dout = ctx.new_output()
+    dout = torch.empty_like(out_layer)[:, h0 * D:(h0 + hl) * D]
     for _ in range(2):
         ctx.dense_attention(dq, dk, dv, dout)
     torch.cuda.synchronize()
@@ -349,6 +368,9 @@ def run_ours(args, wl):
     e2e_ms = max_over_ranks(t0.elapsed_time(t1) / esteps)
     status = ctx.query(hb.Q_DEVICE_STATUS)
     same = bool(torch.equal(hout, out.cpu()))
+    outlier_block = None
+    if (world == 1 or shard) and args.outlier_fraction > 0:   # (every rank of a sharded layer takes part in the exchange)
+        outlier_block = filtered_variant(args, wl, hb, dq, dk, dv, local, layer_heads if shard else 0)
 
     if rank == 0:
         peaks = load_peaks()
@@ -412,11 +434,11 @@ def run_ours(args, wl):
                                         "frac_of_burst_peak": sus_tf / peaks["bf16_tflops"], "clocks": clocks_sus,
                                         "ms_x_sm_mhz": None if clocks_sus.get("sm_mhz") is None else sus_ms * clocks_sus["sm_mhz"]}
         line = {
-            "metric": METRIC, "value": replica_throughput(N, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": replica_throughput(N, jobs, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong" if shard else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(wl),
             "clocks": clocks,
-            "e2e": {"value": replica_throughput(N, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": replica_throughput(N, jobs, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 3 * H * N * D * b, "d2h_bytes_per_step": H * N * D * b, "steps": esteps,
                     "matches_device_path": same},
             "gpu_launches": int(launches),
@@ -434,21 +456,30 @@ def run_ours(args, wl):
             line["cpu_baseline"] = {"value": N / sec, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
                                     "sample": info["sample"], "seconds": info["seconds"], "ms_per_layer_extrapolated": sec * 1e3}
             line["parity_sample"] = parity_sample(ctx, hb, wl, kept, out)
-        if world == 1 and args.outlier_fraction > 0:
-            line["outlier_filter"] = filtered_variant(args, wl, hb, dq, dk, dv, local)
+        if outlier_block is not None:
+            line["outlier_filter"] = outlier_block
+        if shard:
+            line["config"]["parallelism"] = (f"one layer of {layer_heads} heads sharded by head over {world} GPUs ({hl} heads each, head-strided "
+                                             "views, no exchange inside the layer; per-kernel figures are rank 0's shard)")
         print(json.dumps(line), flush=True)
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
 
 
-def filtered_variant(args, wl, hb, dq, dk, dv, device_index):
-    """The same step with query outlier filtering on (Sec. 3.4): public call and per-stage times, in a context of its own."""
+def filtered_variant(args, wl, hb, dq, dk, dv, device_index, layer_heads=0):
+    """The same step with query outlier filtering on (Sec. 3.4): public call and per-stage times, in a context of its own.
+    layer_heads > 0: this rank holds a head shard of a layer with that many heads; the outlier budget is one for all heads, so
+    the three histograms of the threshold selection are summed over the ranks (an NCCL all-reduce of 8 KB each, on the stream
+    of the call)."""
     import torch
     ctx = hb.Httm(hb.HttmConfig.of(wl, device=device_index))
     try:
         max_block = ctx.query(hb.Q_MAX_BLOCK_TOKENS)
         ctx.set_outlier_fraction(args.outlier_fraction)
+        if layer_heads:
+            import torch.distributed as dist
+            ctx.set_head_shard(layer_heads, lambda counts: dist.all_reduce(counts))
         out = ctx.new_output()
         stream = torch.cuda.current_stream()
         steps = max(3, min(args.steps, 100))
@@ -520,6 +551,8 @@ def main():
     ap.add_argument("--ratio", type=float, default=None, help="override both merge ratios")
     ap.add_argument("--block", default=None, help="override block shape, e.g. 4x4x4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="with several GPUs: independent replicas of the layer (default), or ONE layer with its heads dealt to the GPUs")
     ap.add_argument("--oracle-rows", type=int, default=None,
                     help="merged query rows per head the CPU oracle attends; 0 = all of them, nothing extrapolated (default: 0 "
                          "for --impl reference, whose step time is then a measured one, 4096 for the in-line cpu_baseline)")

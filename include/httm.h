@@ -188,6 +188,26 @@ int httm_global_attention(httm_ctx* ctx, httm_tensor q, httm_tensor k, httm_tens
 int httm_set_outlier_fraction(httm_ctx* ctx, double fraction);
 
 /*
+ * Head-sharded layers (Sec. 3.2: every head matches, merges, attends and unmerges on its own).  A context created
+ * with heads = H / G serves the heads one GPU owns: hand it head-strided views of Q, K, V and of the output (its
+ * column slice of [tokens][H x 64]); no kernel reads another shard's data and nothing is exchanged inside the layer.
+ * The one quantity that spans the heads is the outlier budget of Sec. 3.4 (item 3: the gamma-quantile is taken
+ * "across all heads"): with outlier filtering on, tell the context how many heads the whole layer has and give it a
+ * function that sums a vector of int32 counters over all shards.  The threshold selection then builds each of its
+ * three radix histograms (2048, 2048, 1024 counters) locally, calls
+ *     exchange(user, device_counts, n_counts, cuda_stream)
+ * and chooses the bin from the summed histogram, so that every shard arrives at the same threshold: exactly the
+ * one a single context with all the heads finds.  exchange must enqueue, on cuda_stream, an in-place sum of the
+ * n_counts int32 values at device_counts (device memory owned by the context) over all shards, e.g. an NCCL
+ * all-reduce, and return 0; every shard calls it three times per httm_global_attention, in the same order.
+ * total_heads = 0 and exchange = NULL switch sharding off.  Without outlier filtering the setting has no effect.
+ * Errors: INVALID_ARG (fewer heads than the context has; more without an exchange function), UNSUPPORTED (total
+ * heads x tokens >= 2^31); a non-zero return of exchange makes the attention call fail with HTTM_ERR_CUDA.
+ */
+typedef int (*httm_exchange_fn)(void* user, void* device_counts, int32_t n_counts, void* cuda_stream);
+int httm_set_head_shard(httm_ctx* ctx, int32_t total_heads, httm_exchange_fn exchange, void* user);
+
+/*
  * The projections around the path (Algorithm 1: Q, K, V = x W_qkv before it, out = Attn W_o after it) for callers
  * that want no library matmul next to the path:  y[n_rows][out_features] = x[n_rows][in_features] . w^T  with the
  * weight given as w[out_features][in_features] (the layout a linear layer stores), all bf16 on the context's device,

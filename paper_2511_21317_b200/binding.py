@@ -34,7 +34,9 @@ EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
     "httm_global_attention_static", "httm_selftest_tensor_core", "httm_set_outlier_fraction", "httm_linear",
+    "httm_set_head_shard",
 )
+_EXCHANGE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p)
 
 
 class HttmError(RuntimeError):
@@ -70,6 +72,7 @@ def load_library() -> ctypes.CDLL:
     L.httm_global_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_dense_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_set_outlier_fraction.argtypes = [vp, ctypes.c_double]
+    L.httm_set_head_shard.argtypes = [vp, ctypes.c_int32, _EXCHANGE_FN, vp]
     L.httm_linear.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, ctypes.c_int32, ctypes.c_int32, vp]
     L.httm_attention_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
     L.httm_launch_stage.argtypes = [vp, ctypes.c_int, _Tensor, _Tensor, _Tensor, _Tensor, vp]
@@ -214,6 +217,27 @@ class Httm:
         """Query outlier filtering (Sec. 3.4) for the later calls; 0 switches it off."""
         self._check(self._lib.httm_set_outlier_fraction(self._h, float(fraction)))
 
+    def set_head_shard(self, total_heads: int, exchange=None):
+        """This context holds some of the heads of a layer with `total_heads` heads (see httm_set_head_shard).
+        exchange(counts) gets a CUDA int32 tensor that aliases the library's histogram and must sum it in place over all
+        shards on the current stream (e.g. torch.distributed.all_reduce); None with total_heads = 0 switches sharding off."""
+        if exchange is None:
+            cb = ctypes.cast(None, _EXCHANGE_FN)
+        else:
+            device = f"cuda:{self.cfg.device}"
+
+            def trampoline(_user, ptr, n, _stream):
+                try:
+                    exchange(device_int32_view(int(ptr), int(n), device))
+                    return 0
+                except Exception:   # the C side turns this into HTTM_ERR_CUDA; keep the reason
+                    import traceback
+                    traceback.print_exc()
+                    return 1
+            cb = _EXCHANGE_FN(trampoline)
+        self._check(self._lib.httm_set_head_shard(self._h, int(total_heads), cb, None))
+        self._exchange_cb = cb   # the library keeps the pointer: keep the object alive
+
     def linear(self, x: torch.Tensor, w: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
         """y = x . w^T with x [n][in], w [out][in] (rows may be strided), bf16 CUDA tensors; returns y [n][out]."""
         for t, name in ((x, "x"), (w, "w")):
@@ -262,6 +286,16 @@ class Httm:
         self._check(self._lib.httm_export(self._h, what, arr.ctypes.data_as(ctypes.c_void_p), arr.nbytes,
                                           self._stream(stream)))
         return arr
+
+
+class _DeviceInt32:
+    def __init__(self, ptr: int, n: int):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (ptr, False), "version": 2}
+
+
+def device_int32_view(ptr: int, n: int, device) -> torch.Tensor:
+    """A CUDA int32 tensor over n counters at a raw device address (no copy)."""
+    return torch.as_tensor(_DeviceInt32(ptr, n), device=device)
 
 
 def selftest_tensor_core(q, k, v):

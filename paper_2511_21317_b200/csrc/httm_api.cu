@@ -54,6 +54,10 @@ struct httm_ctx {
     // first-frame anchoring: blocks of the first frame group (the first n_anchor blocks) with more dst tokens than the
     // match kernel holds (match_capacity) are matched by a kernel of their own, launched behind it
     int32_t n_anchor = 0, match_capacity = 0;
+    // head-sharded layer (httm_set_head_shard): heads of the whole layer, and the caller's sum over the shards
+    int32_t total_heads = 0;
+    httm_exchange_fn exchange = nullptr;
+    void* exchange_user = nullptr;
     // query outlier filtering (Sec. 3.4): off while fraction == 0; its workspace is allocated when it is first switched on.
     // The merged query length then differs per head: Q_m and O_m get N rows per head.
     double outlier_fraction = 0.0;
@@ -375,7 +379,10 @@ int stage_outlier(httm_ctx* c, const httm_tensor& q, cudaStream_t s) {
     a.mq_head = c->d_mq_head;
     a.tile_prefix = c->d_tile_prefix;
     a.sel = c->d_sel;
-    a.budget = (int64_t)std::floor(c->outlier_fraction * (double)c->cfg.heads * (double)c->n_tokens + 1e-9);
+    const int64_t all_heads = c->total_heads > 0 ? c->total_heads : c->cfg.heads;
+    a.budget = (int64_t)std::floor(c->outlier_fraction * (double)all_heads * (double)c->n_tokens + 1e-9);
+    a.total_count = all_heads * (int64_t)c->n_tokens;
+    a.defer_select = c->exchange != nullptr;
     a.n_blocks = c->n_blocks;
     a.n_tokens = c->n_tokens;
     a.heads = c->cfg.heads;
@@ -383,6 +390,36 @@ int stage_outlier(httm_ctx* c, const httm_tensor& q, cudaStream_t s) {
     a.status = c->d_status;
     int rc;
     if ((rc = check_cuda(c, cudaMemsetAsync(c->d_sel, 0, kSelWords * sizeof(int32_t), s), "selection state reset"))) return rc;
+    if (c->exchange) {
+        // Head-sharded layer: the threshold is one for all heads, so every level's histogram is summed over the shards
+        // (the caller's exchange, in stream order) before its bin is chosen.  Nine kernels (ten over the reordered copies).
+        const bool sorted = sorted_filter(c);
+        if (sorted) {
+            a.src_q = view(c->d_qr, c->n_tokens);
+            if ((rc = check_cuda(c, launch_big_deviation(a, c->max_block, s), "large-block deviation launch"))) return rc;
+            if ((rc = check_cuda(c, launch_refine_level(a, 0, c->sm_count, s), "threshold launch"))) return rc;
+            c->launches += 2;
+        } else {
+            if ((rc = check_cuda(c, launch_deviation(a, c->sm_count, s), "deviation launch"))) return rc;
+            c->launches += 1;
+        }
+        for (int level = 0; level < 3; ++level) {
+            if (level > 0) {
+                if ((rc = check_cuda(c, launch_refine_level(a, level, c->sm_count, s), "threshold launch"))) return rc;
+                c->launches += 1;
+            }
+            if (c->exchange(c->exchange_user, c->d_sel + kSelHist + level * 2048, level == 2 ? 1024 : 2048, s) != 0)
+                return c->fail(HTTM_ERR_CUDA, "the histogram exchange of level %d failed", level);
+            if ((rc = check_cuda(c, launch_select_level(a, level, s), "threshold selection launch"))) return rc;
+            c->launches += 1;
+        }
+        c->launches += 2;
+        if (sorted) {
+            if ((rc = check_cuda(c, launch_big_filter(a, c->max_block, s), "large-block filter launch"))) return rc;
+            return check_cuda(c, launch_offsets(a, s), "offsets launch");
+        }
+        return check_cuda(c, launch_filter(a, s), "filter launch");
+    }
     if (sorted_filter(c)) {   // the blocks are runs of rows of the reordered copy; six kernels
         a.src_q = view(c->d_qr, c->n_tokens);
         if ((rc = check_cuda(c, launch_big_deviation(a, c->max_block, s), "large-block deviation launch"))) return rc;
@@ -628,6 +665,23 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
         if ((rc = check_cuda(c, e, "outlier workspace setup"))) return rc;
     }
     c->outlier_fraction = fraction;
+    return HTTM_OK;
+}
+
+int httm_set_head_shard(httm_ctx* c, int32_t total_heads, httm_exchange_fn exchange, void* user) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (total_heads == 0 && !exchange) {   // back to a layer of its own
+        c->total_heads = 0;
+        c->exchange = nullptr;
+        c->exchange_user = nullptr;
+        return HTTM_OK;
+    }
+    if (total_heads < c->cfg.heads) return c->fail(HTTM_ERR_INVALID_ARG, "head shard: the layer cannot have fewer heads than this context");
+    if ((int64_t)total_heads * c->n_tokens > (1ll << 31) - 1) return c->fail(HTTM_ERR_UNSUPPORTED, "head shard: total heads x tokens must stay below 2^31");
+    if (total_heads > c->cfg.heads && !exchange) return c->fail(HTTM_ERR_INVALID_ARG, "head shard: an exchange function is needed when other shards hold heads");
+    c->total_heads = total_heads;
+    c->exchange = exchange;
+    c->exchange_user = user;
     return HTTM_OK;
 }
 

@@ -141,6 +141,11 @@ struct OutlierArgs {
     int64_t budget;               // K: number of tokens, over all heads, that may be outliers
     int32_t n_blocks, n_tokens, heads, n_special_total;
     int32_t* status;
+    // Head-sharded layers (this context holds some of the heads, the budget is one for ALL heads, Sec. 3.4 item 3):
+    // total_count = deviations of all shards (total heads x tokens); defer_select: the kernels only build their
+    // histograms, the bin is chosen by a kernel of its own once the histograms of all shards have been summed
+    int64_t total_count;
+    int32_t defer_select;
 };
 
 struct UnmergeArgs {
@@ -193,6 +198,8 @@ cudaError_t launch_threshold(const OutlierArgs& a, int sm_count, cudaStream_t st
 cudaError_t launch_filter(const OutlierArgs& a, cudaStream_t stream);   // map rewrite + per-head offsets (two kernels)
 cudaError_t launch_offsets(const OutlierArgs& a, cudaStream_t stream);  // per-head offsets alone
 cudaError_t launch_threshold0(const OutlierArgs& a, int sm_count, cudaStream_t stream);   // threshold with the level-0 histogram taken from the deviations (three kernels)
+cudaError_t launch_refine_level(const OutlierArgs& a, int level, int sm_count, cudaStream_t stream);   // histogram of one level alone (0, 1, 2)
+cudaError_t launch_select_level(const OutlierArgs& a, int level, cudaStream_t stream);                 // choose the bin of one level from its (summed) histogram
 cudaError_t launch_big_deviation(const OutlierArgs& a, int max_block_tokens, cudaStream_t stream);   // large blocks: deviations
 cudaError_t launch_big_filter(const OutlierArgs& a, int max_block_tokens, cudaStream_t stream);      // large blocks: map rewrite + kept counts
 cudaError_t launch_big_scores(const BigMatchArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 contraction + row argmax

@@ -1485,19 +1485,10 @@ __device__ __forceinline__ void select_bin(const int* h, int nb, int rank, int* 
     }
 }
 
-// End of a level, called by every thread of every CTA after the CTA's histogram has been added to the global one:
-// the CTA that arrives last selects the bin.  hist: 2048 ints of shared memory.
-__device__ void finish_level(const OutlierArgs& a, int level, int* hist) {
-    __shared__ int s_last, s_bin, s_rank;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        s_last = atomicAdd(a.sel + kSelDone + level, 1) == (int)gridDim.x - 1;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const int64_t count = (int64_t)a.heads * a.n_tokens;
+// The bin of one level from its complete histogram (one CTA; hist: 2048 ints of shared memory).
+__device__ void select_level(const OutlierArgs& a, int level, int* hist) {
+    __shared__ int s_bin, s_rank;
+    const int64_t count = a.total_count;
     if (level == 0 && (a.budget <= 0 || a.budget >= count)) {   // nothing is an outlier (tau = +inf) / everything is (tau = -1)
         if (threadIdx.x == 0) {
             *a.tau = a.budget <= 0 ? INFINITY : -1.0f;
@@ -1505,6 +1496,7 @@ __device__ void finish_level(const OutlierArgs& a, int level, int* hist) {
         }
         return;
     }
+    if (level > 0 && __ldcg(a.sel + kSelFinished)) return;
     const int nb = level == 2 ? 1024 : 2048, shift = level == 0 ? 21 : (level == 1 ? 10 : 0);
     for (int i = threadIdx.x; i < nb; i += blockDim.x) hist[i] = __ldcg(a.sel + kSelHist + level * 2048 + i);
     __syncthreads();
@@ -1522,6 +1514,27 @@ __device__ void finish_level(const OutlierArgs& a, int level, int* hist) {
             }
         }
     }
+}
+
+// End of a level, called by every thread of every CTA after the CTA's histogram has been added to the global one:
+// the CTA that arrives last selects the bin - unless the selection is deferred (head-sharded layers: the histograms
+// of the other shards are still to be added; select_level_kernel runs behind the exchange).
+__device__ void finish_level(const OutlierArgs& a, int level, int* hist) {
+    __shared__ int s_last;
+    if (a.defer_select) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(a.sel + kSelDone + level, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    select_level(a, level, hist);
+}
+__global__ void __launch_bounds__(256) select_level_kernel(const OutlierArgs a, int level) {
+    __shared__ int hist[2048];
+    select_level(a, level, hist);
 }
 
 constexpr int kRefineThreads = 256;
@@ -1676,6 +1689,23 @@ cudaError_t launch_threshold0(const OutlierArgs& a, int sm_count, cudaStream_t s
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return launch_threshold(a, sm_count, stream);
+}
+cudaError_t launch_refine_level(const OutlierArgs& a, int level, int sm_count, cudaStream_t stream) {
+    const int64_t quads = ((int64_t)a.heads * a.n_tokens) >> 2;
+    int64_t grid = (quads + kRefineThreads * 4 - 1) / (kRefineThreads * 4);
+    if (grid > 2ll * sm_count) grid = 2ll * sm_count;
+    if (grid < 1) grid = 1;
+    if (level == 0)
+        refine_kernel<0><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
+    else if (level == 1)
+        refine_kernel<1><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
+    else
+        refine_kernel<2><<<(unsigned)grid, kRefineThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+cudaError_t launch_select_level(const OutlierArgs& a, int level, cudaStream_t stream) {
+    select_level_kernel<<<1, 256, 0, stream>>>(a, level);
+    return cudaGetLastError();
 }
 cudaError_t launch_offsets(const OutlierArgs& a, cudaStream_t stream) {
     offsets_kernel<<<(unsigned)a.heads, kOffsetsThreads, 0, stream>>>(a);
