@@ -305,6 +305,20 @@ int httm_global_attention_static(const httm_config* cfg, httm_tensor q, httm_ten
                                  httm_tensor out, void* cuda_stream);
 
 /*
+ * Aids for testing the error paths (host-side injection; nothing here faults or hangs the device).
+ *   httm_fail_nth_allocation(n): the n-th device allocation the library makes from now on (in this process) fails as if
+ *     the device were out of memory: the call that needed it returns HTTM_ERR_NOMEM and releases what it had taken.
+ *     n = 0 switches it off.
+ *   httm_expire_a_wait(ctx, stream): enqueues a one-tile kernel whose producer issues two of the three loads its
+ *     barrier expects, so that the kernel's bounded wait runs out (about two seconds): it records the time-out in the
+ *     context's status word, releases its tensor memory and returns.  The next httm_query(HTTM_Q_DEVICE_STATUS) /
+ *     httm_export then reports HTTM_ERR_TIMEOUT; the context stays usable (the status word keeps the first error).
+ * Errors: INVALID_ARG, UNSUPPORTED (a context with fewer than 384 token-heads), CUDA.
+ */
+int httm_fail_nth_allocation(int32_t n);
+int httm_expire_a_wait(httm_ctx* ctx, void* cuda_stream);
+
+/*
  * Diagnostic: one 128-row tile through the tensor-core building blocks of the attention kernel
  * (Eq. 3-4 on a single tile): s_out[128][128] = Q K^T and o_out[128][64] = bf16(s_out) V in fp32,
  * with q, k, v contiguous bf16 [128][64] DEVICE arrays (16-byte aligned), s_out / o_out / status_dev

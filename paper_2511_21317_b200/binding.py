@@ -34,7 +34,7 @@ EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
     "httm_global_attention_static", "httm_selftest_tensor_core", "httm_set_outlier_fraction", "httm_linear",
-    "httm_set_head_shard",
+    "httm_set_head_shard", "httm_fail_nth_allocation", "httm_expire_a_wait",
 )
 _EXCHANGE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p)
 
@@ -73,6 +73,8 @@ def load_library() -> ctypes.CDLL:
     L.httm_dense_attention.argtypes = [vp, _Tensor, _Tensor, _Tensor, _Tensor, vp]
     L.httm_set_outlier_fraction.argtypes = [vp, ctypes.c_double]
     L.httm_set_head_shard.argtypes = [vp, ctypes.c_int32, _EXCHANGE_FN, vp]
+    L.httm_fail_nth_allocation.argtypes = [ctypes.c_int32]
+    L.httm_expire_a_wait.argtypes = [vp, vp]
     L.httm_linear.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, ctypes.c_int32, ctypes.c_int32, vp]
     L.httm_attention_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
     L.httm_launch_stage.argtypes = [vp, ctypes.c_int, _Tensor, _Tensor, _Tensor, _Tensor, vp]
@@ -217,6 +219,10 @@ class Httm:
         """Query outlier filtering (Sec. 3.4) for the later calls; 0 switches it off."""
         self._check(self._lib.httm_set_outlier_fraction(self._h, float(fraction)))
 
+    def expire_a_wait(self, stream=None):
+        """Error-path test aid: a kernel whose bounded wait runs out (see httm_expire_a_wait)."""
+        self._check(self._lib.httm_expire_a_wait(self._h, self._stream(stream)))
+
     def set_head_shard(self, total_heads: int, exchange=None):
         """This context holds some of the heads of a layer with `total_heads` heads (see httm_set_head_shard).
         exchange(counts) gets a CUDA int32 tensor that aliases the library's histogram and must sum it in place over all
@@ -296,6 +302,11 @@ class _DeviceInt32:
 def device_int32_view(ptr: int, n: int, device) -> torch.Tensor:
     """A CUDA int32 tensor over n counters at a raw device address (no copy)."""
     return torch.as_tensor(_DeviceInt32(ptr, n), device=device)
+
+
+def fail_nth_allocation(n: int):
+    """Error-path test aid: the n-th device allocation of the library from now on fails (0: off)."""
+    load_library().httm_fail_nth_allocation(int(n))
 
 
 def selftest_tensor_core(q, k, v):

@@ -16,6 +16,7 @@ using namespace httm;
 
 namespace {
 thread_local std::string g_create_error;
+int g_fail_allocation = 0;   // httm_fail_nth_allocation: counts down to the device allocation that is made to fail
 
 struct DeviceGuard {
     int prev = -1;
@@ -100,7 +101,8 @@ struct httm_ctx {
     template <typename T>
     int alloc(T** p, size_t count) {
         const size_t bytes = (count ? count : 1) * sizeof(T);
-        cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
+        cudaError_t e = g_fail_allocation > 0 && --g_fail_allocation == 0 ? cudaErrorMemoryAllocation
+                                                                          : cudaMalloc(reinterpret_cast<void**>(p), bytes);
         if (e != cudaSuccess) {
             *p = nullptr;
             cudaGetLastError();
@@ -648,11 +650,21 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
     if (!c->d_eps) {
         const size_t H = c->cfg.heads, N = c->n_tokens, B = c->n_blocks;
         int rc;
+        const int64_t before = c->workspace_bytes;
         if ((rc = c->alloc(&c->d_assign_qf, H * N)) || (rc = c->alloc(&c->d_kept_cnt, H * B)) || (rc = c->alloc(&c->d_moff_var, H * B)) ||
             (rc = c->alloc(&c->d_mq_head, H)) || (rc = c->alloc(&c->d_tile_prefix, H + 1)) || (rc = c->alloc(&c->d_sel, kSelWords)) ||
             (rc = c->alloc(&c->d_tau, 1)) || (rc = c->alloc(&c->d_qm_var, H * N * kHeadDim)) || (rc = c->alloc(&c->d_om_var, H * N * kHeadDim)) ||
-            (rc = c->alloc(&c->d_eps, H * N)))
+            (rc = c->alloc(&c->d_eps, H * N))) {
+            // give back what this attempt took: a later call starts from nothing again
+            void** taken[] = {(void**)&c->d_assign_qf, (void**)&c->d_kept_cnt, (void**)&c->d_moff_var, (void**)&c->d_mq_head, (void**)&c->d_tile_prefix,
+                              (void**)&c->d_sel, (void**)&c->d_tau, (void**)&c->d_qm_var, (void**)&c->d_om_var, (void**)&c->d_eps};
+            for (void** p : taken) {
+                if (*p) cudaFree(*p);
+                *p = nullptr;
+            }
+            c->workspace_bytes = before;
             return rc;
+        }
         // special tokens: never merged (identity map entries, deviation 0), written here once; rows of Q_m past a head's
         // merged length are read by the last query tile of the head (their results are discarded): give them a value
         std::vector<int32_t> ident(H * N);
@@ -666,6 +678,21 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
     }
     c->outlier_fraction = fraction;
     return HTTM_OK;
+}
+
+int httm_fail_nth_allocation(int32_t n) {
+    g_fail_allocation = n > 0 ? n : 0;
+    return HTTM_OK;
+}
+
+int httm_expire_a_wait(httm_ctx* c, void* cuda_stream) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if ((int64_t)c->cfg.heads * c->n_tokens < 3 * 128) return c->fail(HTTM_ERR_UNSUPPORTED, "the context's workspace is smaller than three 128-token tiles");
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    c->launches++;
+    return check_cuda(c, launch_wait_expiry(c->d_qr, reinterpret_cast<float*>(c->d_kr), c->d_status, static_cast<cudaStream_t>(cuda_stream)),
+                      "wait-expiry launch");
 }
 
 int httm_set_head_shard(httm_ctx* c, int32_t total_heads, httm_exchange_fn exchange, void* user) {

@@ -211,5 +211,6 @@ cudaError_t configure_linear();
 cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t stream);   // tcgen05 / TMEM kernel
 cudaError_t configure_attention();
 cudaError_t configure_kernels();   // one-time function attributes (dynamic shared memory sizes)
+cudaError_t launch_wait_expiry(const void* tiles, float* scratch, int32_t* status, cudaStream_t stream);   // time-out path test, see httm_umma_selftest.cu
 
 }  // namespace httm

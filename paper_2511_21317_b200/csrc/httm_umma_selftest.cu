@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "../../include/httm.h"
+#include "httm_internal.h"
 #include "tc_sm100.cuh"
 
 namespace httm {
@@ -80,7 +81,7 @@ namespace {
 __global__ void __launch_bounds__(128) umma_selftest_kernel(const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             const __grid_constant__ CUtensorMap map_v, float* s_out, float* o_out,
-                                                            int* status) {
+                                                            int* status, int status_code, int drop_one_load) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* sq = smem;             // 128 x 128 B
@@ -109,7 +110,10 @@ __global__ void __launch_bounds__(128) umma_selftest_kernel(const __grid_constan
         tc::mbar_expect_tx(bar_tma, 3 * 16384);
         tc::tma_load_3d(tc::smem_addr(sq), &map_q, bar_tma, 0, 0, 0);
         tc::tma_load_3d(tc::smem_addr(sk), &map_k, bar_tma, 0, 0, 0);
-        tc::tma_load_3d(tc::smem_addr(sv), &map_v, bar_tma, 0, 0, 0);
+        // drop_one_load (the test of the time-out path): the barrier expects the bytes of three tiles but only two loads
+        // are issued, so the wait below runs into its limit; every thread then leaves through the ok == false path, the
+        // status word is set, tensor memory is released and the kernel returns normally
+        if (!drop_one_load) tc::tma_load_3d(tc::smem_addr(sv), &map_v, bar_tma, 0, 0, 0);
     }
     bool ok = tc::mbar_wait(bar_tma, 0, &abort_flag);
     if (ok && tid == 0) {
@@ -165,7 +169,7 @@ __global__ void __launch_bounds__(128) umma_selftest_kernel(const __grid_constan
             for (int i = 0; i < 32; ++i) o_out[tid * 64 + c * 32 + i] = __uint_as_float(r[i]);
         }
     }
-    if (!ok && tid == 0) atomicCAS(status, 0, 2);
+    if (!ok && tid == 0) atomicCAS(status, 0, status_code);
     tc::fence_before_sync();
     __syncthreads();
     if (warp == 0) tc::tmem_dealloc(tmem, 256);
@@ -187,6 +191,24 @@ extern "C" int httm_selftest_tensor_core(const void* q, const void* k, const voi
         cudaGetLastError();
         return HTTM_ERR_CUDA;
     }
-    umma_selftest_kernel<<<1, 128, smem, static_cast<cudaStream_t>(cuda_stream)>>>(mq, mk, mv, s_out, o_out, status_dev);
+    umma_selftest_kernel<<<1, 128, smem, static_cast<cudaStream_t>(cuda_stream)>>>(mq, mk, mv, s_out, o_out, status_dev, 2, 0);
     return cudaGetLastError() == cudaSuccess ? HTTM_OK : HTTM_ERR_CUDA;
 }
+
+namespace httm {
+// The one-tile kernel with one of its three loads left out: its bounded wait gives up after about two seconds and the
+// kernel records kDevTimeoutAttention in `status` (a context's status word).  tiles: 3 x 128 x 64 bf16 of readable
+// device memory (contents irrelevant), scratch: never written (the kernel only writes results when its waits succeed).
+cudaError_t launch_wait_expiry(const void* tiles, float* scratch, int32_t* status, cudaStream_t stream) {
+    CUtensorMap mq, mk, mv;
+    const __nv_bfloat16* t = static_cast<const __nv_bfloat16*>(tiles);
+    if (!encode_rows_tensor_map(&mq, t, 128, 1, 64, 0, 128) || !encode_rows_tensor_map(&mk, t + 8192, 128, 1, 64, 0, 128) ||
+        !encode_rows_tensor_map(&mv, t + 16384, 128, 1, 64, 0, 128))
+        return cudaErrorInvalidValue;
+    const int smem = 3 * 16384 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(umma_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    umma_selftest_kernel<<<1, 128, smem, stream>>>(mq, mk, mv, scratch, scratch, status, kDevTimeoutAttention, 1);
+    return cudaGetLastError();
+}
+}  // namespace httm
