@@ -31,7 +31,7 @@ from paper_2511_21317_b200 import synth  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (one ncu capture, summary under profiles/), with
 # the digest of the kernel's sources at the time of the capture: the figure is reported only while the sources still
 # have that digest (null for workloads that were not captured and once the kernel has changed).
-ATTENTION_DRAM_TRAFFIC = {"medium": (64933120 + 5256960, "0" * 16)}
+ATTENTION_DRAM_TRAFFIC = {"medium": (67586048 + 27885056, "c2398d696669b4f2")}   # profiles/ncu_full_medium_attention_kernels.txt, first launch
 ATTENTION_SOURCES = ("paper_2511_21317_b200/csrc/httm_attention_tc.cu", "paper_2511_21317_b200/csrc/tc_sm100.cuh")
 METRIC = "httm_global_attention_layer_throughput"
 UNIT = "tokens/s"

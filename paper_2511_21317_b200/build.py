@@ -21,7 +21,7 @@ SOURCES = ["httm_api.cu", "httm_mem_kernels.cu", "httm_attention_tc.cu", "httm_b
            "httm_umma_selftest.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "--use_fast_math=false" if False else "-Xcompiler", "-Wall",
+    "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall",
 ]
 
 

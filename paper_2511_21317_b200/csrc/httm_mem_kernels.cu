@@ -860,9 +860,11 @@ merge_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     a.group_start[(int64_t)h * (a.m_q + 1) + moff + lane] = start + incl - sz;
                 }
                 __syncwarp();
-                if (tok >= 0)
-                    a.group_member[(int64_t)h * a.n_tokens + start + gsz[row_of] + __popc(group & ((1u << lane) - 1u))] =
-                        __ldg(a.pi + start + tok);
+                if (tok >= 0) {   // the token's number in the original order: from the block's place in the scene, or through the reorder index
+                    const int orig = DIRECT ? (bg.s0 + own_t) * a.layout.tokens_per_frame + a.layout.n_special + (bg.y0 + own_y) * a.layout.grid_w + bg.x0 + own_x
+                                            : __ldg(a.pi + start + tok);
+                    a.group_member[(int64_t)h * a.n_tokens + start + gsz[row_of] + __popc(group & ((1u << lane) - 1u))] = orig;
+                }
             }
             // x fragments: for k step ks (16 tokens) and channel tile pair np, one ldmatrix.x4.trans gives
             // b0, b1 of channel tile 2 np and b0, b1 of channel tile 2 np + 1
