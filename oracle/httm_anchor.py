@@ -97,3 +97,22 @@ def global_attention(g: orc.Geometry, ratio_q: float, ratio_kv: float, q, k, v, 
         om = orc.attention(qm, km, vm)
         out = orc.unmerge(g, pi, rq, om)
     return orc.Result(pi, bs, aq, ak, mbq, msq, mbk, msk, rq, rk, Mq, Mk, qm, km, vm, om, out)
+
+
+def global_attention_filtered(g: orc.Geometry, ratio_q: float, ratio_kv: float, gamma: float, q, k, v, attend: bool = True,
+                              assign_q_filtered=None, assign_q_initial=None, assign_k=None):
+    """Algorithm 1 with first-frame anchoring in both matchings AND the query outlier filtering of Sec. 3.4.
+    The paper describes the two separately; the composition taken here: the filtering runs unchanged on the anchored
+    query map (deviation of every token from the mean of its group, one threshold over all heads, outliers leave
+    their groups).  A token of the reference frame that is an outlier leaves the group it anchors and stays on its
+    own row like every other outlier, so the reference frame remains unmerged; its former group continues under its
+    lowest remaining member.  The optional maps continue from maps under test, as in the plain filtered oracle."""
+    from . import httm_outlier as flt
+    pi, bs = orc.temporal_reorder(g)
+    if assign_q_initial is None:
+        assign_q_initial = match(g, bs, ratio_q, orc.reorder(g, pi, q))[0]
+    if assign_k is None:
+        assign_k = match(g, bs, ratio_kv, orc.reorder(g, pi, k))[0]
+    return flt.global_attention_filtered(g, ratio_q, ratio_kv, gamma, q, k, v, attend=attend,
+                                         assign_q_filtered=assign_q_filtered, assign_q_initial=assign_q_initial,
+                                         assign_k=assign_k)

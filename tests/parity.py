@@ -158,20 +158,28 @@ def full_check(g, rho_q, rho_kv, q, k, v, ex, out_bits, sample_tokens=None, what
 DEV_TOL = 1e-5   # deviations: |gpu - oracle| <= DEV_TOL x (largest |q| + the deviation): fp32 means, differences and sums of 64 squares
 
 
-def filtered_check(g, rho_q, rho_kv, gamma, q, k, v, ex, out_bits, n_outliers, sample_tokens=None, what="", peaky=False):
+def filtered_check(g, rho_q, rho_kv, gamma, q, k, v, ex, out_bits, n_outliers, sample_tokens=None, what="", peaky=False,
+                   anchor=False):
     """Query outlier filtering (Sec. 3.4, Algorithm 2) against its oracle.
     ex: exports pi, blk_start, assign_q0 (map of the initial merging), assign_q (after the outliers left), assign_k,
     eps, tau, mq_head, rank_q, q_m, k_m, v_m, o_m (q_m, o_m with N rows per head, head h's first mq_head[h] valid).
     Rules: the matching maps as in check_maps; deviations within DEV_TOL; the threshold is the (K+1)-th largest of
     the deviations under test, within DEV_TOL of the oracle's; the outlier decision agrees with the oracle's for
     every token whose deviation is further than 2 x DEV_TOL from the oracle's threshold; the filtered map is exactly
-    what the oracle's rule makes of the decisions under test; everything downstream continues from that map."""
+    what the oracle's rule makes of the decisions under test; everything downstream continues from that map.
+    anchor: the matching maps are those of first-frame anchoring (its oracle, its block rules in the margin check)."""
     from oracle import httm_outlier as flt
-    res0 = orc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
+    anchored = None
+    if anchor:
+        from oracle import httm_anchor as anc
+        res0 = anc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
+        anchored = {b: n0 for b, n, n0 in anc.anchored_blocks(g, res0.blk_start)}
+    else:
+        res0 = orc.global_attention(g, rho_q, rho_kv, q, k, v, attend=False)
     assert np.array_equal(ex["pi"].astype(np.int64), res0.pi), f"{what}: reorder permutation differs"
     qr, kr = orc.reorder(g, res0.pi, q), orc.reorder(g, res0.pi, k)
-    nq = check_maps(g, rho_q, res0.blk_start, qr, res0.assign_q, res0.margin_best_q, res0.margin_sel_q, ex["assign_q0"], what + " A_q (initial)")
-    nk = check_maps(g, rho_kv, res0.blk_start, kr, res0.assign_k, res0.margin_best_k, res0.margin_sel_k, ex["assign_k"], what + " A_k")
+    nq = check_maps(g, rho_q, res0.blk_start, qr, res0.assign_q, res0.margin_best_q, res0.margin_sel_q, ex["assign_q0"], what + " A_q (initial)", anchored)
+    nk = check_maps(g, rho_kv, res0.blk_start, kr, res0.assign_k, res0.margin_best_k, res0.margin_sel_k, ex["assign_k"], what + " A_k", anchored)
     aq0 = ex["assign_q0"].astype(np.int64)
     eps = flt.deviations(aq0, qr)
     eps_gpu = ex["eps"].astype(np.float64)
@@ -196,7 +204,7 @@ def filtered_check(g, rho_q, rho_kv, gamma, q, k, v, ex, out_bits, n_outliers, s
     assert n_outliers == in_blocks, f"{what}: outlier counter {n_outliers} != {in_blocks}"
     aq = flt.filter_map(aq0, outl_gpu)
     assert np.array_equal(ex["assign_q"].astype(np.int64), aq), f"{what}: filtered map differs from the rule applied to the decisions"
-    res = flt.global_attention_filtered(g, rho_q, rho_kv, gamma, q, k, v, attend=False, assign_q_filtered=aq,
+    res = (anc if anchor else flt).global_attention_filtered(g, rho_q, rho_kv, gamma, q, k, v, attend=False, assign_q_filtered=aq,
                                         assign_q_initial=aq0, assign_k=ex["assign_k"].astype(np.int64))
     assert ex["mq_head"].tolist() == res.M_q, f"{what}: merged query lengths {ex['mq_head'].tolist()} != {res.M_q}"
     stats = {"ambiguous_blocks_q": nq, "ambiguous_blocks_k": nk, "outliers": int(outl_gpu.sum()), "tau": tau_gpu,

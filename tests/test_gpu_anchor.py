@@ -101,18 +101,35 @@ def test_anchor_argument_errors():
     assert e.value.code == hb.ERR_UNSUPPORTED
 
 
-def test_anchoring_with_outlier_filtering_runs_and_keeps_the_reference_frame():
-    wl = synth.Workload("anchor_filter", 8, 8, 8, 4, 4, 2, 0.7, 0.7, heads=4)
+FILTERED = [
+    # name, frames, grid_h, grid_w, blk, ratio_q, ratio_kv, heads, gamma
+    ("four_frames_32", 8, 8, 8, (4, 4, 2), 0.7, 0.7, 4, 0.05),             # warp-per-block kernels with direct loads
+    ("two_frames_32_clipped", 5, 9, 10, (2, 4, 4), 0.5, 0.9, 2, 0.1),      # the first frame group's own match kernel
+    ("blocks_128", 8, 8, 16, (4, 4, 8), 0.5, 0.75, 2, 0.03),               # sorted-group kernels on the reordered copies
+    ("runs_large_blocks", 12, 1, 200, (12, 1, 64), 0.9, 0.7, 2, 0.1),      # large-block path
+]
+
+
+@pytest.mark.parametrize("case", FILTERED, ids=[c[0] for c in FILTERED])
+def test_anchoring_with_outlier_filtering(case):
+    """Both options together against the oracle's composition (filtering runs on the anchored query map): maps,
+    deviations, threshold, filtered map, per-head lengths, merged tensors and output; the reference frame stays unmerged."""
+    from tests.test_gpu_outlier import NAMES
+    name, S, h, w, blk, rq, rkv, H, gamma = case
+    wl = synth.Workload(name, S, h, w, blk[0], blk[1], blk[2], rq, rkv, heads=H, seed=6)
     q, k, v = synth.make_qkv(wl)
     with hb.Httm(dataclasses.replace(hb.HttmConfig.of(wl), anchor_first_frame=1)) as ctx:
-        ctx.set_outlier_fraction(0.05)
+        ctx.set_outlier_fraction(gamma)
         out = ctx.global_attention(*(hb.bf16_from_bits(x, DEV) for x in (q, k, v)))
         torch.cuda.synchronize()
-        assert ctx.query(hb.Q_DEVICE_STATUS) == 0 and torch.isfinite(out.float()).all()
-        A = ctx.export(hb.X_ASSIGN_Q)
-        frame = ctx.export(hb.X_PI) // wl.tokens_per_frame
-        assert (A[:, frame == 0] == np.arange(wl.n_tokens)[frame == 0]).all()
-        assert ctx.query(hb.Q_OUTLIERS) == int(np.floor(0.05 * wl.heads * wl.n_tokens + 1e-9))
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        ex = {n: ctx.export(what) for n, what in NAMES.items()}
+        stats = parity.filtered_check(orc.Geometry.of(wl), rq, rkv, gamma, q, k, v, ex, hb.bits_from_bf16(out),
+                                      ctx.query(hb.Q_OUTLIERS), None, name, peaky=True, anchor=True)
+        assert stats["outliers"] == int(np.floor(gamma * wl.heads * wl.n_tokens + 1e-9))
+        assert stats["peaky_needed"] <= 1e-3 * stats["out_elements"]
+        frame = ex["pi"] // wl.tokens_per_frame
+        assert (ex["assign_q"][:, frame == 0] == np.arange(wl.n_tokens)[frame == 0]).all()
 
 
 @pytest.mark.parametrize("name", ["tiny", "small", "medium"])

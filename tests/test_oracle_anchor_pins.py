@@ -108,3 +108,51 @@ def test_margins_follow_the_plain_convention():
     best = np.sort(sim.max(axis=1))[::-1]
     r = min(int(np.floor(0.5 * n + 1e-9)), n - n0)
     assert ms[0, b] == pytest.approx(best[r - 1] - best[r])
+
+
+def test_anchoring_with_outlier_filtering_against_plain_loops():
+    """The composition (filtering on the anchored query map) restated with loops: deviations from the group means,
+    the K largest over all heads leave, an orphaned group continues under its lowest remaining member."""
+    wl, g, (q, k, v) = case(seed=11, S=6, h=4, w=6, blk=(3, 2, 3), heads=2)
+    gamma = 0.08
+    res = anc.global_attention_filtered(g, 0.7, 0.6, gamma, q, k, v, attend=False)
+    base = anc.global_attention(g, 0.7, 0.6, q, k, v, attend=False)
+    assert np.array_equal(res.assign_q0, base.assign_q) and np.array_equal(res.assign_k, base.assign_k)
+    x = orc.bf16_to_double(orc.reorder(g, res.pi, q))
+    H, N = base.assign_q.shape
+    eps = np.zeros((H, N))
+    for hd in range(H):
+        for i in range(N):
+            members = [j for j in range(N) if base.assign_q[hd, j] == base.assign_q[hd, i]]
+            mean = sum(x[hd, j] for j in members) / len(members)
+            eps[hd, i] = float(np.sqrt(((x[hd, i] - mean) ** 2).sum())) if len(members) > 1 else 0.0
+    assert np.allclose(res.eps, eps, rtol=1e-12, atol=1e-14)
+    K = int(np.floor(gamma * H * N + 1e-9))
+    order = sorted(((-eps[hd, i], hd, i) for hd in range(H) for i in range(N)))
+    assert -order[K][0] < -order[K - 1][0]                       # no tie at the threshold in this case
+    out = {(hd, i) for _, hd, i in order[:K]}
+    assert {(int(a), int(b)) for a, b in zip(*np.nonzero(res.outlier))} == out
+    for hd in range(H):
+        for i in range(N):
+            if (hd, i) in out:
+                expect = i
+            else:
+                rest = [j for j in range(N) if base.assign_q[hd, j] == base.assign_q[hd, i] and (hd, j) not in out]
+                d = int(base.assign_q[hd, i])
+                expect = d if (hd, d) not in out else min(rest)
+            assert res.assign_q[hd, i] == expect
+    frame = frame_of_position(g, res.pi)
+    assert (res.assign_q[:, frame == 0] == np.arange(N)[frame == 0]).all()      # the reference frame stays unmerged
+    assert any((hd, i) in out for hd in range(H) for i in np.nonzero(frame == 0)[0])   # ... although some of it are outliers
+    assert res.M_q == [len(set(res.assign_q[hd].tolist())) for hd in range(H)] and min(res.M_q) > anc.merged_len(g, 0.7)
+
+
+def test_anchoring_with_an_outlier_budget_of_zero_or_all_tokens():
+    wl, g, (q, k, v) = case(seed=12)
+    plain = anc.global_attention(g, 0.7, 0.6, q, k, v)
+    res = anc.global_attention_filtered(g, 0.7, 0.6, 0.0, q, k, v)
+    assert np.array_equal(res.assign_q, plain.assign_q) and np.allclose(res.out, plain.out, rtol=1e-12, atol=1e-14)
+    res = anc.global_attention_filtered(g, 0.7, 0.6, 1.0, q, k, v)                  # every query on its own: K/V merging only
+    assert res.M_q == [res.pi.size] * g.heads
+    ref = orc.merged_attention_from_maps(g, res.pi, q, k, v, np.tile(np.arange(res.pi.size), (g.heads, 1)), plain.assign_k)
+    assert np.allclose(res.out, ref.out, rtol=1e-12, atol=1e-14)
