@@ -12,8 +12,9 @@
 // accumulators O_A, O_B take the remaining 2 x 64 columns.  S(k+3) is issued right after P(k) V, into
 // the buffer that P(k) V releases, so the scores of a softmax warp's next tile are ready before it
 // finishes the current one: the softmax warps never wait for the tensor core in steady state.
-// Running maxima are only raised when they grow by more than 2^8 (then the softmax threads rescale O
-// in place), so rescaling is rare after the first tiles.  Every wait is bounded; on expiry the kernel
+// A row's stabiliser is the maximum of its first score tile; later tiles take their exponentials without
+// looking for the maximum first and are redone (with O rescaled in place) only if their weights would
+// overflow, which bounded scores never do.  Every wait is bounded; on expiry the kernel
 // records kDevTimeoutAttention in the status word, releases its tensor memory and returns.
 #include "httm_internal.h"
 #include "tc_sm100.cuh"
@@ -35,7 +36,8 @@ constexpr int kOutRowPitch = kRowBytes + 16;             // staged output rows: 
 constexpr int kOutStageBytes = 8 * 32 * kOutRowPitch;   // eight softmax warps x 32 output rows, staged for bulk stores
 constexpr int SMEM_BYTES = (2 + 2 * KV_STAGES) * TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row exchange*/ +
                            (2 * kTableHeads + 4) * 4 /*head tables*/ + kOutStageBytes;
-constexpr float kRescaleThreshold = 8.0f;   // log2 units
+constexpr int kPColumn = 64;                  // P (bf16 pairs, 64 columns) lies over columns 64 .. 127 of its S
+constexpr float kSumLimit = 1.2676506e30f;   // 2^100: a tile whose row sum of weights reaches it is redone with a raised maximum
 
 struct Barriers {
     uint64_t q_full;
@@ -62,6 +64,8 @@ struct TcParams {
     const int32_t* group_start;  // optional (UNMERGE): members of every merged query row, see AttentionArgs
     const int32_t* group_member;
     int32_t n_tokens;
+    const __nv_bfloat16 *q, *k;  // the rows themselves, for the tile that is redone (element strides)
+    int64_t q_stride_head, q_stride_token, k_stride_head, k_stride_token;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -75,14 +79,15 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-// 2^t for two values without the special-function unit: round-to-nearest range reduction
-// t = n + f, f in [-0.5, 0.5] (the integer lands in the low mantissa bits of t + 1.5 * 2^23), a cubic
-// minimax polynomial for 2^f (relative error < 1e-4, far below the bf16 rounding of P) evaluated with
-// packed fp32 FMAs, and n added to the exponent field.  Arguments below -125 give 2^-125.
+// 2^t for two values without the special-function unit.  The arguments are clamped to [-125, 125] (an argument of
+// 125 or more gives 2^125, which the caller's test of the tile's row sum catches; without the clamps the exponent
+// arithmetic below would wrap).  Then round-to-nearest range reduction t = n + f, f in [-0.5, 0.5] (the integer lands
+// in the low mantissa bits of t + 1.5 * 2^23), a cubic minimax polynomial for 2^f (relative error < 1e-4, far below
+// the bf16 rounding of P) evaluated with packed fp32 FMAs, and n added to the exponent field.
 __device__ __forceinline__ float2 exp2_poly2(float2 t) {
     const float kMagic = 12582912.0f;
-    t.x = fmaxf(t.x, -125.0f);
-    t.y = fmaxf(t.y, -125.0f);
+    t.x = fminf(fmaxf(t.x, -125.0f), 125.0f);
+    t.y = fminf(fmaxf(t.y, -125.0f), 125.0f);
     const float2 tt = tc::fadd2(t, make_float2(kMagic, kMagic));
     const float2 n = tc::fadd2(tt, make_float2(-kMagic, -kMagic));
     const float2 f = tc::ffma2(n, make_float2(-1.0f, -1.0f), t);
@@ -99,6 +104,70 @@ __device__ __forceinline__ float2 exp2_poly2(float2 t) {
 // persistent kernel: 0/8: 545 us, 1/8: 510 us, 2/8: 481 us, 3/8: 497-504 us, 4/8: 570 us, 8/8: 790 us
 // (alternating 2/8 and 3/8 over the 16-column groups: 480 us).
 constexpr uint32_t kPolyPairs = 0x11;   // pairs 0 and 4 of 8
+
+// A score tile whose weights overflowed with the stabiliser at hand is done again here, for one query row per thread:
+// its 128 scores are recomputed from the rows in global memory by plain fp32 FMAs (the tile in tensor memory is
+// partly overwritten by the weights, the key tile in shared memory may have been replaced), first for their maximum,
+// then for the weights 2^(s c - m'), m' = max(m, c max s), written as bf16 pairs to the eight-column groups at
+// `t_p`.  Returns m' and the row's sum of weights.  Only inputs whose scores differ by more than 69 (100 in base 2)
+// between key tiles ever come here; it is kept out of line so that it costs the ordinary tiles no registers.
+struct RedoneTile {
+    float m, sum;
+};
+__device__ __noinline__ RedoneTile redo_score_tile(const __nv_bfloat16* q_row, const __nv_bfloat16* k_rows, int64_t k_stride_token, int valid,
+                                                   float c, float m_old, uint32_t t_p) {
+    float qf[kHeadDim];
+    if (q_row) {
+#pragma unroll
+        for (int i = 0; i < kHeadDim / 8; ++i) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(q_row) + i);
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                qf[8 * i + 2 * e] = __uint_as_float(w[e] << 16);
+                qf[8 * i + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+        }
+    } else {   // a row past the end of the queries (zero-filled by the tile load)
+#pragma unroll
+        for (int i = 0; i < kHeadDim; ++i) qf[i] = 0.f;
+    }
+    auto score = [&](int key) {
+        const uint4* kr = reinterpret_cast<const uint4*>(k_rows + (int64_t)key * k_stride_token);
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < kHeadDim / 8; ++i) {
+            const uint4 u = __ldg(kr + i);
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                a0 = fmaf(qf[8 * i + 2 * e], __uint_as_float(w[e] << 16), a0);
+                a1 = fmaf(qf[8 * i + 2 * e + 1], __uint_as_float(w[e] & 0xffff0000u), a1);
+            }
+        }
+        return a0 + a1;
+    };
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int key = 0; key < valid; ++key) mx = fmaxf(mx, score(key));
+    RedoneTile r;
+    r.m = fmaxf(m_old, mx * c);
+    r.sum = 0.f;
+#pragma unroll 1
+    for (int cc = 0; cc < 8; ++cc) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int key = cc * 16 + 2 * i;
+            const float e0 = key < valid ? exp2f(fmaf(score(key), c, -r.m)) : 0.f;
+            const float e1 = key + 1 < valid ? exp2f(fmaf(score(key + 1), c, -r.m)) : 0.f;
+            r.sum += e0 + e1;
+            pk[i] = pack_bf16(e0, e1);
+        }
+        tc::tmem_st8(t_p + cc * 8, pk);
+    }
+    return r;
+}
 
 // Work decomposition.  The query tiles of all heads form one list (head-major, T tiles).  With G CTAs
 // (one per SM), round r < R = T / (2 G) gives CTA c the two tiles 2 (r G + c), +1: a PAIR pass (tiles A and B
@@ -287,7 +356,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     __syncthreads();
     tc::fence_after_sync();
     const uint32_t tmem = bars->tmem_base;
-    // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the first 64 columns of its S
+    // columns: score buffers [0,128) [128,256) [256,384); O_A [384,448)  O_B [448,512); P overlays the last 64 columns of its S
     const int32_t* mq_table = tables_on_chip ? s_mq : p.mq_head;
     PassWalker<VAR> walker(p.rounds, p.total_tiles, p.tiles_per_head, tables_on_chip ? s_prefix : p.tile_prefix, p.heads);
     Pass ps;
@@ -357,7 +426,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (X == 0 && !tc::mbar_wait(tc::smem_addr(&bars->v_full[ST]), (kv_base[ST] + round_par) & 1u, abort_flag)) return false;
                 if (!tc::mbar_wait(tc::smem_addr(&bars->p_full[B]), (sp_base[B] + (C / 3)) & 1u, abort_flag)) return false;
                 tc::fence_after_sync();
-                issue_pv(t_o, t_buf, dv0 + ST * kStageStep);
+                issue_pv(t_o, t_buf + kPColumn, dv0 + ST * kStageStep);
                 tc::mma_commit(tc::smem_addr(&bars->o_done[X]));
                 if (X == 1) tc::mma_commit(tc::smem_addr(&bars->v_empty[ST]));
                 if (k0 + C + 3 < n_score) {
@@ -380,7 +449,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (!tc::mbar_wait(tc::smem_addr(&bars->v_full[B]), (kv_base[B] + IDX) & 1u, abort_flag)) return false;
                 if (!tc::mbar_wait(tc::smem_addr(&bars->p_full[B]), (sp_base[B] + IDX) & 1u, abort_flag)) return false;
                 tc::fence_after_sync();
-                issue_pv(t_o, t_buf, dv0 + B * kStageStep);
+                issue_pv(t_o, t_buf + kPColumn, dv0 + B * kStageStep);
                 tc::mma_commit(tc::smem_addr(&bars->o_done[X]));
                 tc::mma_commit(tc::smem_addr(&bars->v_empty[B]));
                 if (k0 + C + 3 < n_tiles) {
@@ -472,6 +541,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const int mq_rows = VAR ? mq_table[ps.head] : p.m_q;   // valid query rows of this head
             // this group's score tiles are k = 2 i + x; in a pair pass they come from key tile i, in a single pass from key tile k
             const int n_own = ps.pair ? n_tiles : (n_tiles - x + 1) / 2;
+            const int own_row = (ps.tile + (ps.pair ? x : 0)) * BM + row;   // this thread's query row inside the head
+            const bool row_exists = own_row < mq_rows;
+            const __nv_bfloat16* q_row = row_exists ? p.q + (int64_t)ps.head * p.q_stride_head + (int64_t)own_row * p.q_stride_token : nullptr;
+            const __nv_bfloat16* k_head = p.k + (int64_t)ps.head * p.k_stride_head;
             {
                 float m = -INFINITY, l = 0.f;
                 {   // the accumulator O starts at zero: every PV step accumulates (ordered before the first p_full arrival)
@@ -495,32 +568,64 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     for (int cc = 0; cc < 4; ++cc) tc::tmem_ld32(t_s + cc * 32, s + cc * 32);
                     tc::tmem_wait_ld();
                     const int valid = p.m_k - key_tile * BN;
-                    if (valid < BN) {
+                    auto mask_tail = [&](auto first_c, auto last_c) {   // -inf for keys past the end
+                        if (valid < BN) {
 #pragma unroll
-                        for (int i = 0; i < BN; ++i)
-                            if (i >= valid) s[i] = 0xff800000u;   // -inf: keys past the end
-                    }
-                    // row maximum: four independent chains of three-input maxima
-                    float mx4[4];
+                            for (int i = decltype(first_c)::value; i < decltype(last_c)::value; ++i)
+                                if (i >= valid) s[i] = 0xff800000u;
+                        }
+                    };
+                    mask_tail(std::integral_constant<int, 0>{}, std::integral_constant<int, BN>{});
+                    // The stabiliser m of a row is the maximum of its FIRST score tile (times c) and is raised later only if
+                    // a tile would overflow: bf16 weights and the fp32 sums and accumulators do not care about a common
+                    // factor, so weights of up to 2^100 are as good as weights of at most 1.  Every later tile therefore goes
+                    // without a pass over its scores for the row maximum: the exponentials are taken with the m at hand,
+                    // and only if some row's sum of weights reaches 2^100 (or is not a number) the tile is done again, this
+                    // time with its own maximum (redo_score_tile). the sum and the accumulator O are
+                    // rescaled in place once the previous P V of this query tile has completed (the next one is issued
+                    // after this tile's P), and the weights are written anew.
+                    auto row_max = [&]() {   // four independent chains of three-input maxima
+                        float mx4[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        mx4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
+                        for (int q = 0; q < 4; ++q) {
+                            mx4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
 #pragma unroll
-                        for (int i = 2; i < 32; i += 2)
-                            mx4[q] = tc::fmax3(mx4[q], __uint_as_float(s[32 * q + i]), __uint_as_float(s[32 * q + i + 1]));
-                    }
-                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                    const float m_new = fmaxf(m, mx * c);
-                    if (j == 0) {
-                        m = m_new;
-                    } else if (__any_sync(0xffffffffu, m_new - m > kRescaleThreshold)) {
-                        // raise the running maximum: rescale the row sum and the accumulator O in place, once the
-                        // previous P V of this query tile has completed (the next one is issued after this tile's P)
+                            for (int i = 2; i < 32; i += 2)
+                                mx4[q] = tc::fmax3(mx4[q], __uint_as_float(s[32 * q + i]), __uint_as_float(s[32 * q + i + 1]));
+                        }
+                        return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    };
+                    auto weights = [&]() {   // P = 2^(s c - m) as bf16 pairs over the LAST 64 columns of S; returns the row sum
+                        const float2 c2 = make_float2(c, c), neg_m2 = make_float2(-m, -m);
+                        float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0;
+#pragma unroll
+                        for (int cc = 0; cc < 8; ++cc) {
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const float2 t = tc::ffma2(make_float2(__uint_as_float(s[cc * 16 + 2 * i]), __uint_as_float(s[cc * 16 + 2 * i + 1])), c2, neg_m2);
+                                const float2 e = ((kPolyPairs >> i) & 1u) ? exp2_poly2(t) : make_float2(fast_exp2(t.x), fast_exp2(t.y));
+                                if (i & 1)
+                                    sum1 = tc::fadd2(sum1, e);
+                                else
+                                    sum0 = tc::fadd2(sum0, e);
+                                pk[i] = pack_bf16(e.x, e.y);
+                            }
+                            tc::tmem_st8(t_s + kPColumn + cc * 8, pk);
+                        }
+                        return (sum0.x + sum0.y) + (sum1.x + sum1.y);
+                    };
+                    if (j == 0) m = row_max() * c;
+                    float tile_sum = weights();
+                    if (j > 0 && __any_sync(0xffffffffu, row_exists && !(tile_sum < kSumLimit))) {
                         if (!(ok = tc::mbar_wait(obar, (od_base + (uint32_t)(j - 1)) & 1u, abort_flag))) break;
                         tc::fence_after_sync();
-                        const float f = exp2f(m - m_new);
+                        const RedoneTile redone = redo_score_tile(q_row, k_head + (int64_t)key_tile * BN * p.k_stride_token, p.k_stride_token,
+                                                                  valid < BN ? valid : BN, c, m, t_s + kPColumn);
+                        const float f = exp2f(m - redone.m);
                         l *= f;
-                        m = m_new;
+                        m = redone.m;
+                        tile_sum = redone.sum;
 #pragma unroll 1
                         for (int cc = 0; cc < 8; ++cc) {   // eight columns at a time: this rare path must not cost registers
                             uint32_t o[8];
@@ -531,24 +636,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             tc::tmem_st8(t_o + cc * 8, o);
                         }
                     }
-                    const float2 c2 = make_float2(c, c), neg_m2 = make_float2(-m, -m);
-                    float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0;
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc) {
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float2 t = tc::ffma2(make_float2(__uint_as_float(s[cc * 16 + 2 * i]), __uint_as_float(s[cc * 16 + 2 * i + 1])), c2, neg_m2);
-                            const float2 e = ((kPolyPairs >> i) & 1u) ? exp2_poly2(t) : make_float2(fast_exp2(t.x), fast_exp2(t.y));
-                            if (i & 1)
-                                sum1 = tc::fadd2(sum1, e);
-                            else
-                                sum0 = tc::fadd2(sum0, e);
-                            pk[i] = pack_bf16(e.x, e.y);
-                        }
-                        tc::tmem_st8(t_s + cc * 8, pk);   // P: bf16 pairs over the first 64 columns of S
-                    }
-                    l += (sum0.x + sum0.y) + (sum1.x + sum1.y);
+                    l += tile_sum;
                     tc::tmem_wait_st();
                     tc::fence_before_sync();
                     tc::mbar_arrive(pbar);
@@ -652,7 +740,7 @@ cudaError_t launch_attention(const AttentionArgs& a, int sm_count, cudaStream_t 
     if (ctas > total) ctas = total;
     const int rounds = total / (2 * ctas);
     TcParams p{a.out, a.out_stride_head, a.out_stride_token, a.m_q, a.m_k, a.scale_log2, a.status, tiles_per_head, total, rounds, a.mq_head, a.tile_prefix, a.heads,
-               a.group_start, a.group_member, a.n_tokens};
+               a.group_start, a.group_member, a.n_tokens, a.q.ptr, a.k.ptr, a.q.stride_head, a.q.stride_token, a.k.stride_head, a.k.stride_token};
     if (a.mq_head) {   // the tile table lives in device memory: full grid, CTAs without tiles leave at once
         if (a.group_start) return cudaErrorInvalidValue;   // (the member lists are built for equal query lengths only)
         attention_tc_kernel<true, false><<<sm_count < 1 ? 1 : sm_count, NTHREADS, SMEM_BYTES, stream>>>(mq, mk, mv, p);

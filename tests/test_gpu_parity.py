@@ -121,6 +121,41 @@ def test_ratio_zero_equals_dense_and_textbook():
         assert d <= 2e-2 * float(np.sqrt(np.mean(ref ** 2)))
 
 
+@pytest.mark.parametrize("heads", [2, 26])
+def test_scores_far_above_those_of_the_first_key_tile(heads):
+    """Keys whose scores exceed everything in a row's first key tile by 2^80 .. 2^320: the kernel takes its stabiliser
+    from the first tile and redoes a tile whose weights would overflow (even heads: two such jumps; odd heads stay just
+    below the limit, with weights of up to 2^90); rows with the opposite sign see scores that only fall.  Two heads
+    are dealt as single passes (one query tile per CTA), 26 heads as pair passes."""
+    wl = synth.Workload("grow", 2, 18, 20, 2, 4, 4, 0.0, 0.0, heads=heads)
+    N = wl.n_tokens                                              # 730 tokens: six key tiles, pair passes and single passes
+    rng = np.random.default_rng(21)
+    w = rng.standard_normal(64)
+    w /= np.linalg.norm(w)
+    tile = np.arange(N) // 128
+    a = np.stack([np.where(tile == 0, 0.1, np.where(tile <= 2, 25.0, 60.0)),     # q.k/8*log2(e): 0.5, 135, 325
+                  np.where(tile == 0, 0.1, 15.0)] * (heads // 2))                 # 0.5, 81
+    b = np.where(rng.random(N) < 0.5, 30.0, -30.0)
+    b[::7] = 0.01                                                # rows that see almost flat scores
+    k = a[:, :, None] * w + 0.3 * rng.standard_normal((heads, N, 64))
+    q = b[None, :, None] * w + 0.05 * rng.standard_normal((heads, N, 64))
+    v = rng.standard_normal((heads, N, 64))
+    q, k, v = (synth.f32_to_bf16_bits(x.astype(np.float32)) for x in (q, k, v))
+    ref = orc.dense_attention(orc.Geometry.of(wl), q, k, v)
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        dq, dk, dv = (hb.bf16_from_bits(x, DEV) for x in (q, k, v))
+        o_d = ctx.dense_attention(dq, dk, dv)
+        o_h = ctx.global_attention(dq, dk, dv)                  # ratio 0: the same rows through the epilogue that unmerges
+        torch.cuda.synchronize()
+        assert ctx.query(hb.Q_DEVICE_STATUS) == 0
+        for name, o in (("dense", o_d), ("ratio 0", o_h)):
+            bits = hb.bits_from_bf16(o)
+            assert np.isfinite(parity.bits_to_f64(bits)).all(), name
+            stats = {}
+            stats["out_err"] = parity.check_output(bits, ref, what=f"growing scores, {name}", peaky=True, stats=stats)
+            report_peaky(f"growing scores, {name}", stats)
+
+
 def test_dense_attention_small_config_sampled():
     wl = synth.WORKLOADS["small"].replace(heads=4)
     q, k, v = synth.make_qkv(wl)
