@@ -305,6 +305,22 @@ int httm_global_attention_static(const httm_config* cfg, httm_tensor q, httm_ten
                                  httm_tensor out, void* cuda_stream);
 
 /*
+ * Times of the kernels INSIDE a call of httm_global_attention (the paper's Table 3 splits a layer the same way: attention,
+ * matching, aggregation).  httm_set_call_timing(ctx, 1) makes every later httm_global_attention on this context record
+ * a CUDA event on the caller's stream before its first kernel and after each part of the call (a part is one kernel;
+ * the five small kernels of the outlier filter count as one part); the events are created by this call, none per
+ * httm_global_attention.  httm_call_times waits for the last call's final event and returns, for its parts in launch
+ * order, the time between consecutive events in milliseconds (ms[i]) and a name (names[i], static strings such as
+ * "match_direct", "merge_direct", "attention_unmerge"; names may be NULL); *count = number of parts of the last call,
+ * of which at most `capacity` are written.  Host pointers.  The times are those of the kernels as they run in the
+ * call, one behind the other (caches as the previous kernel left them), which the one-kernel launches of
+ * httm_launch_stage are not.  Off by default; enable = 0 switches it off again.
+ * Errors: INVALID_ARG (null arguments, timing off), CUDA.
+ */
+int httm_set_call_timing(httm_ctx* ctx, int32_t enable);
+int httm_call_times(httm_ctx* ctx, float* ms, const char** names, int32_t capacity, int32_t* count);
+
+/*
  * Aids for testing the error paths (host-side injection; nothing here faults or hangs the device).
  *   httm_fail_nth_allocation(n): the n-th device allocation the library makes from now on (in this process) fails as if
  *     the device were out of memory: the call that needed it returns HTTM_ERR_NOMEM and releases what it had taken.

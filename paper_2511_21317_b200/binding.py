@@ -34,7 +34,7 @@ EXPORTED_SYMBOLS = (
     "httm_create", "httm_global_attention", "httm_dense_attention", "httm_attention_host", "httm_launch_stage",
     "httm_query", "httm_export", "httm_last_error", "httm_launch_count", "httm_destroy",
     "httm_global_attention_static", "httm_selftest_tensor_core", "httm_set_outlier_fraction", "httm_linear",
-    "httm_set_head_shard", "httm_fail_nth_allocation", "httm_expire_a_wait",
+    "httm_set_head_shard", "httm_fail_nth_allocation", "httm_expire_a_wait", "httm_set_call_timing", "httm_call_times",
 )
 _EXCHANGE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p)
 
@@ -218,6 +218,19 @@ class Httm:
     def set_outlier_fraction(self, fraction: float):
         """Query outlier filtering (Sec. 3.4) for the later calls; 0 switches it off."""
         self._check(self._lib.httm_set_outlier_fraction(self._h, float(fraction)))
+
+    def set_call_timing(self, enable: bool):
+        """Events between the kernels of global_attention (see httm_set_call_timing)."""
+        self._check(self._lib.httm_set_call_timing(self._h, 1 if enable else 0))
+
+    def call_times(self):
+        """[(part name, milliseconds)] of the last global_attention call, in launch order (waits for the call to finish)."""
+        cap = 16
+        ms = (ctypes.c_float * cap)()
+        names = (ctypes.c_char_p * cap)()
+        n = ctypes.c_int32(0)
+        self._check(self._lib.httm_call_times(self._h, ms, names, cap, ctypes.byref(n)))
+        return [(names[i].decode(), float(ms[i])) for i in range(min(n.value, cap))]
 
     def expire_a_wait(self, stream=None):
         """Error-path test aid: a kernel whose bounded wait runs out (see httm_expire_a_wait)."""

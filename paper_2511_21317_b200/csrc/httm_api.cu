@@ -87,6 +87,12 @@ struct httm_ctx {
     int64_t host_calls = 0;
     int64_t workspace_bytes = 0;
     int64_t launches = 0;
+    // optional: events between the kernels of httm_global_attention (httm_set_call_timing)
+    static constexpr int kMaxCallParts = 12;
+    bool call_timing = false;
+    cudaEvent_t call_ev[kMaxCallParts + 1] = {};
+    const char* call_part[kMaxCallParts] = {};
+    int call_parts = 0;
     std::string error;
 
     int fail(int code, const char* fmt, ...) {
@@ -123,6 +129,10 @@ struct httm_ctx {
         for (HostSet& h : hs)
             for (cudaEvent_t e : {h.loaded, h.consumed, h.computed, h.returned})
                 if (e) cudaEventDestroy(e);
+        for (cudaEvent_t& e : call_ev) {
+            if (e) cudaEventDestroy(e);
+            e = nullptr;
+        }
         if (s_h2d) cudaStreamDestroy(s_h2d);
         if (s_d2h) cudaStreamDestroy(s_d2h);
     }
@@ -456,37 +466,49 @@ int dense_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const ht
 
 int global_impl(httm_ctx* c, const httm_tensor& q, const httm_tensor& k, const httm_tensor& v, const httm_tensor& out,
                 cudaStream_t s) {
+    // With call timing on, an event follows every part of the call (a part is one kernel, or the five small kernels of
+    // the outlier filter); part(rc, name) passes the stage's return code through.
+    c->call_parts = 0;
+    if (c->call_timing) cudaEventRecord(c->call_ev[0], s);
+    auto part = [&](int rc, const char* name) {
+        if (rc == HTTM_OK && c->call_timing && c->call_parts < httm_ctx::kMaxCallParts) {
+            c->call_part[c->call_parts++] = name;
+            cudaEventRecord(c->call_ev[c->call_parts], s);
+        }
+        return rc;
+    };
     int rc;
     if (c->big()) {   // six kernels: reorder (+ norms), scores, select, merge, attention, unmerge
-        if ((rc = stage_reorder(c, q, k, v, s))) return rc;
-        if ((rc = stage_big_scores(c, s))) return rc;
-        if ((rc = stage_big_select(c, s))) return rc;
-        if (c->filtering() && (rc = stage_outlier(c, q, s))) return rc;
-        if ((rc = stage_merge(c, s))) return rc;
-        if ((rc = stage_attention(c, s))) return rc;
-        return stage_unmerge(c, out, s);
+        if ((rc = part(stage_reorder(c, q, k, v, s), "reorder"))) return rc;
+        if ((rc = part(stage_big_scores(c, s), "big_scores"))) return rc;
+        if ((rc = part(stage_big_select(c, s), "big_select"))) return rc;
+        if (c->filtering() && (rc = part(stage_outlier(c, q, s), "outlier_filter"))) return rc;
+        if ((rc = part(stage_merge(c, s), "merge"))) return rc;
+        if ((rc = part(stage_attention(c, s), "attention"))) return rc;
+        return part(stage_unmerge(c, out, s), "unmerge");
     }
     if (sorted_filter(c)) {   // outlier filtering with blocks of 33 .. 256 tokens: everything from the reordered copies
-        if ((rc = stage_reorder(c, q, k, v, s))) return rc;
-        if ((rc = stage_match(c, s))) return rc;
-        if ((rc = stage_outlier(c, q, s))) return rc;
-        if ((rc = stage_merge(c, s))) return rc;
-        if ((rc = stage_attention(c, s))) return rc;
-        return stage_unmerge(c, out, s);
+        if ((rc = part(stage_reorder(c, q, k, v, s), "reorder"))) return rc;
+        if ((rc = part(stage_match(c, s), "match"))) return rc;
+        if ((rc = part(stage_outlier(c, q, s), "outlier_filter"))) return rc;
+        if ((rc = part(stage_merge(c, s), "merge"))) return rc;
+        if ((rc = part(stage_attention(c, s), "attention"))) return rc;
+        return part(stage_unmerge(c, out, s), "unmerge");
     }
     if (direct_mode(c)) {   // the temporal reorder is folded into the block loads of match and merge
         const httm_tensor src[3] = {q, k, v};
-        if ((rc = stage_match(c, s, src))) return rc;
-        if (c->filtering() && (rc = stage_outlier(c, q, s))) return rc;
-        if ((rc = stage_merge(c, s, src))) return rc;
+        if ((rc = part(stage_match(c, s, src), "match_direct"))) return rc;
+        if (c->filtering() && (rc = part(stage_outlier(c, q, s), "outlier_filter"))) return rc;
+        if ((rc = part(stage_merge(c, s, src), "merge_direct"))) return rc;
     } else {
-        if ((rc = stage_reorder(c, q, k, v, s))) return rc;
-        if ((rc = stage_match(c, s))) return rc;
-        if ((rc = stage_merge(c, s))) return rc;
+        if ((rc = part(stage_reorder(c, q, k, v, s), "reorder"))) return rc;
+        if ((rc = part(stage_match(c, s), "match"))) return rc;
+        if ((rc = part(stage_merge(c, s), "merge"))) return rc;
     }
-    if (fused_unmerge(c)) return stage_attention(c, s, &out);   // ... and the unmerge into the attention epilogue: three kernels
-    if ((rc = stage_attention(c, s))) return rc;
-    return stage_unmerge(c, out, s);
+    // ... and the unmerge into the attention epilogue: three kernels
+    if (fused_unmerge(c)) return part(stage_attention(c, s, &out), "attention_unmerge");
+    if ((rc = part(stage_attention(c, s), "attention"))) return rc;
+    return part(stage_unmerge(c, out, s), "unmerge");
 }
 
 int device_status(httm_ctx* c, int32_t* value) {
@@ -678,6 +700,38 @@ int httm_set_outlier_fraction(httm_ctx* c, double fraction) {
     }
     c->outlier_fraction = fraction;
     return HTTM_OK;
+}
+
+int httm_set_call_timing(httm_ctx* c, int32_t enable) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (enable != 0 && enable != 1) return c->fail(HTTM_ERR_INVALID_ARG, "enable must be 0 or 1");
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    if (enable && !c->call_ev[0]) {
+        for (cudaEvent_t& e : c->call_ev) {
+            const int rc = check_cuda(c, cudaEventCreate(&e), "cudaEventCreate");
+            if (rc) return rc;
+        }
+    }
+    c->call_timing = enable != 0;
+    c->call_parts = 0;
+    return HTTM_OK;
+}
+
+int httm_call_times(httm_ctx* c, float* ms, const char** names, int32_t capacity, int32_t* count) {
+    if (!c) return HTTM_ERR_INVALID_ARG;
+    if (!ms || !count || capacity < 0) return c->fail(HTTM_ERR_INVALID_ARG, "httm_call_times: null argument");
+    if (!c->call_timing) return c->fail(HTTM_ERR_INVALID_ARG, "call timing is off (httm_set_call_timing)");
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return c->fail(HTTM_ERR_CUDA, "cudaSetDevice failed");
+    *count = c->call_parts;
+    if (c->call_parts == 0) return HTTM_OK;
+    int rc = check_cuda(c, cudaEventSynchronize(c->call_ev[c->call_parts]), "cudaEventSynchronize");
+    for (int i = 0; rc == HTTM_OK && i < c->call_parts && i < capacity; ++i) {
+        rc = check_cuda(c, cudaEventElapsedTime(&ms[i], c->call_ev[i], c->call_ev[i + 1]), "cudaEventElapsedTime");
+        if (names) names[i] = c->call_part[i];
+    }
+    return rc;
 }
 
 int httm_fail_nth_allocation(int32_t n) {

@@ -46,6 +46,7 @@ struct Barriers {
     uint64_t s_full[3], p_full[3];   // per score buffer
     uint64_t o_done[2];              // per query tile: one completion per P V
     uint64_t o_final;
+    uint64_t q_free;                 // every S = Q K^T of the pass has been computed: the Q tiles may be replaced
     uint64_t x_full, x_done;         // single pass: tile B's (max, sum) published / tile A done reading O_B
     uint32_t tmem_base;
     int abort_flag;
@@ -334,6 +335,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc::mbar_init(tc::smem_addr(&bars->o_done[0]), 1);
         tc::mbar_init(tc::smem_addr(&bars->o_done[1]), 1);
         tc::mbar_init(tc::smem_addr(&bars->o_final), 1);
+        tc::mbar_init(tc::smem_addr(&bars->q_free), 1);
         tc::mbar_init(tc::smem_addr(&bars->x_full), 128);
         tc::mbar_init(tc::smem_addr(&bars->x_done), 128);
         tc::fence_barrier_init();
@@ -366,8 +368,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (tc::elect_one()) {
             uint32_t kv_base[3] = {0, 0, 0};   // completions of each ring stage before this pass (parity bit)
             for (int pass = 0; walker.next(&ps); ++pass) {
-                // the previous pass's MMAs read Q and the ring: all of them are complete at o_final
-                if (pass > 0 && !tc::mbar_wait(tc::smem_addr(&bars->o_final), (uint32_t)(pass - 1) & 1u, abort_flag)) break;
+                // The Q tiles are free once the previous pass's last S has been computed (a few key tiles before its end):
+                // the next pass's Q and first K / V tiles arrive while the previous pass finishes, the ring runs on.
+                if (pass > 0 && !tc::mbar_wait(tc::smem_addr(&bars->q_free), (uint32_t)(pass - 1) & 1u, abort_flag)) break;
                 const uint32_t qb = tc::smem_addr(&bars->q_full);
                 tc::mbar_expect_tx(qb, ps.pair ? 2 * TILE_BYTES : TILE_BYTES);
                 tc::tma_load_3d(s_q, &map_q, qb, 0, ps.tile * BM, ps.head);
@@ -375,12 +378,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 bool ok = true;
                 for (int j = 0; j < n_tiles; ++j) {
                     const int st = j % KV_STAGES;
-                    const uint32_t par = (kv_base[st] + (uint32_t)(j / KV_STAGES)) & 1u;   // completion index of tile j in stage st
-                    if (j >= KV_STAGES && !(ok = tc::mbar_wait(tc::smem_addr(&bars->k_empty[st]), par ^ 1u, abort_flag))) break;
+                    const uint32_t fill = kv_base[st] + (uint32_t)(j / KV_STAGES);         // completion index of tile j in stage st
+                    const uint32_t par = fill & 1u;
+                    if (fill > 0 && !(ok = tc::mbar_wait(tc::smem_addr(&bars->k_empty[st]), par ^ 1u, abort_flag))) break;
                     const uint32_t kb = tc::smem_addr(&bars->k_full[st]);
                     tc::mbar_expect_tx(kb, TILE_BYTES);
                     tc::tma_load_3d(s_k + st * TILE_BYTES, &map_k, kb, 0, j * BN, ps.head);
-                    if (j >= KV_STAGES && !(ok = tc::mbar_wait(tc::smem_addr(&bars->v_empty[st]), par ^ 1u, abort_flag))) break;
+                    if (fill > 0 && !(ok = tc::mbar_wait(tc::smem_addr(&bars->v_empty[st]), par ^ 1u, abort_flag))) break;
                     const uint32_t vb = tc::smem_addr(&bars->v_full[st]);
                     tc::mbar_expect_tx(vb, TILE_BYTES);
                     tc::tma_load_3d(s_v + st * TILE_BYTES, &map_v, vb, 0, j * BN, ps.head);
@@ -436,6 +440,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     }
                     issue_qk(t_buf, dq0 + X3 * kStageStep, dk0 + ST3 * kStageStep, tc::smem_addr(&bars->s_full[B]));
                     if (X3 == 1) tc::mma_commit(tc::smem_addr(&bars->k_empty[ST3]));
+                    if (k0 + C + 4 == n_score) tc::mma_commit(tc::smem_addr(&bars->q_free));   // that was the last S of the pass
                 }
                 return true;
             };
@@ -457,6 +462,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     tc::fence_after_sync();
                     issue_qk(t_buf, dq0, dk0 + B * kStageStep, tc::smem_addr(&bars->s_full[B]));
                     tc::mma_commit(tc::smem_addr(&bars->k_empty[B]));
+                    if (k0 + C + 4 == n_tiles) tc::mma_commit(tc::smem_addr(&bars->q_free));   // that was the last S of the pass
                 }
                 return true;
             };
@@ -478,6 +484,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         tc::fence_after_sync();
                         issue_qk(tmem + 2 * BN, dq0, dk0 + kStageStep, tc::smem_addr(&bars->s_full[2]));
                     }
+                    if (n_score <= 3) tc::mma_commit(tc::smem_addr(&bars->q_free));
                     uint32_t round_par = 0;
                     for (int k0 = 0; ok && k0 < n_score; k0 += 6, round_par ^= 1u) {
                         ok = step_pair(std::integral_constant<int, 0>{}, k0, round_par, n_score);
@@ -505,6 +512,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         issue_qk(tmem + 2 * BN, dq0, dk0 + 2 * kStageStep, tc::smem_addr(&bars->s_full[2]));
                         tc::mma_commit(tc::smem_addr(&bars->k_empty[2]));
                     }
+                    if (n_tiles <= 3) tc::mma_commit(tc::smem_addr(&bars->q_free));
                     for (int k0 = 0; ok && k0 < n_tiles; k0 += 6) {
                         ok = step_single(std::integral_constant<int, 0>{}, k0);
                         if (ok && k0 + 1 < n_tiles) ok = step_single(std::integral_constant<int, 1>{}, k0);

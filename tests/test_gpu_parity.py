@@ -266,6 +266,42 @@ def test_unmerge_in_the_attention_epilogue_equals_the_separate_kernels():
             assert torch.equal(out_hm.permute(1, 0, 2).reshape(N, H * 64), fused), wl.name
 
 
+def test_call_timing_names_the_kernels_of_the_public_call():
+    """Events between the kernels of httm_global_attention: the parts are the kernels the call runs, in order, their
+    times are positive and add up to no more than the whole call, and the results do not change."""
+    wl = synth.WORKLOADS["tiny"]
+    q, k, v = (hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(wl))
+    with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
+        ref = ctx.global_attention(q, k, v).clone()
+        with pytest.raises(hb.HttmError) as e:
+            ctx.call_times()
+        assert e.value.code == hb.ERR_INVALID_ARG
+        ctx.set_call_timing(True)
+        assert ctx.call_times() == []                                  # no call yet
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        before = ctx.launch_count()
+        e0.record()
+        out = ctx.global_attention(q, k, v)
+        e1.record()
+        parts = ctx.call_times()
+        torch.cuda.synchronize()
+        assert ctx.launch_count() - before == 3 and torch.equal(out, ref)
+        assert [n for n, _ in parts] == ["match_direct", "merge_direct", "attention_unmerge"]
+        assert all(ms > 0 for _, ms in parts) and sum(ms for _, ms in parts) <= e0.elapsed_time(e1) * 1.001
+        ctx.set_outlier_fraction(0.05)
+        ctx.global_attention(q, k, v)
+        assert [n for n, _ in ctx.call_times()] == ["match_direct", "outlier_filter", "merge_direct", "attention", "unmerge"]
+        ctx.set_outlier_fraction(0.0)
+        ctx.set_call_timing(False)
+        assert torch.equal(ctx.global_attention(q, k, v), ref)
+    big = synth.Workload("timing_big", 4, 1, 230, 4, 1, 100, 0.9, 0.7, heads=2)
+    q, k, v = (hb.bf16_from_bits(x, DEV) for x in synth.make_qkv(big))
+    with hb.Httm(hb.HttmConfig.of(big)) as ctx:
+        ctx.set_call_timing(True)
+        ctx.global_attention(q, k, v)
+        assert [n for n, _ in ctx.call_times()] == ["reorder", "big_scores", "big_select", "merge", "attention", "unmerge"]
+
+
 def test_argument_errors_are_reported_before_any_launch():
     wl = synth.WORKLOADS["tiny"].replace(heads=2)
     with hb.Httm(hb.HttmConfig.of(wl)) as ctx:
