@@ -325,7 +325,7 @@ def run_ours(args, wl):
     # what a pair of events with nothing between them reads, in the same queue (the per-kernel figures include it)
     gap = [(ev(), ev()) for _ in range(20)]
     for a_, b_ in gap:
-        ctx.launch_stage(order[-1], dq, dk, dv, out)
+        ctx.launch_stage(order[0], dq, dk, dv, out)
         a_.record(stream)
         b_.record(stream)
     torch.cuda.synchronize()
